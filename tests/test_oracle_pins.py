@@ -1,0 +1,333 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle itself.
+
+Hand-worked cases (tests/golden), full attention at alpha = 0 against a library softmax, agreement with the literal
+bool-matrix form of Algorithm 1, brute force over all subsets on tiny inputs, closed-form special cases and
+per-step invariants. A dropped term, wrong sign/index or transposed operand in the oracle fails at least one.
+"""
+import itertools
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import CormOracle
+from oracle.alg1_literal import LiteralUnit
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_golden(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(line)
+    return rows
+
+
+def _logit_inputs(c, d=64):
+    """q, k_j with q.k_j/sqrt(d) = ln c_j up to one float32 rounding; v_j = j in every channel."""
+    q = np.zeros((d,), dtype=np.float32)
+    q[0] = np.sqrt(d)
+    k = np.zeros((len(c), d), dtype=np.float64)
+    k[:, 0] = np.log(np.asarray(c, dtype=np.float64))
+    v = np.tile(np.arange(1, len(c) + 1, dtype=np.float32)[:, None], (1, d))
+    return q, k.astype(np.float32), v
+
+
+def _empty_prompt(o, d):
+    o.compress_prompt(0, np.zeros((o.B, o.Hkv, 0, d), np.float32), None, None, [0] * o.B)
+
+
+def test_handworked_decode_case():
+    rows = _read_golden("handworked_decode.txt")
+    c = [int(x) for x in rows[0].split()[1:]]
+    q, k, v = _logit_inputs(c)
+    o = CormOracle(1, 1, 1, 1, 64, 16, 2, 1, 1.0)
+    _empty_prompt(o, 64)
+    for line in rows[1:]:
+        t, live, out, words = [x.strip() for x in line.split("|")]
+        t = int(t)
+        got = o.decode_step(0, q[None, None], k[t - 1][None, None], v[t - 1][None, None])
+        st = o.export_unit(0, 0, 0)
+        assert st["pos"].tolist() == [int(x) for x in live.split()], (t, st["pos"])
+        assert st["word"].tolist() == [int(x, 2) for x in words.split()], (t, st["word"])
+        # float32 storage of ln c_j perturbs the logits by ~1e-7, hence the tolerance on the fraction
+        assert np.allclose(got[0, 0], float(Fraction(out)), rtol=0, atol=2e-6), (t, got[0, 0, 0])
+        assert st["n_tokens"] == t and st["n_obs"] == min(t, 2)
+
+
+def test_handworked_prompt_case():
+    rows = dict((r.split()[0], r.split()[1:]) for r in _read_golden("handworked_prompt.txt"))
+    c = [int(x) for x in rows["c"]]
+    q, k, v = _logit_inputs(c)
+    o = CormOracle(1, 1, 1, 1, 64, 16, 2, 1, 1.0)
+    q_last = np.stack([q, q])[None, None]                      # the two recorded queries are equal
+    o.compress_prompt(0, k[None, None], v[None, None], q_last, [4])
+    st = o.export_unit(0, 0, 0)
+    assert st["pos"].tolist() == [int(x) for x in rows["live_after"]]
+    assert st["word"].tolist() == [int(x, 2) for x in rows["words_after"]]
+    # a window of 3 records positions 2,3,4: key1 111; key2 (1/9 < 1/2 at i=2, then minor twice) 000; key3 000;
+    # key4 001 -> same survivors
+    o2 = CormOracle(1, 1, 1, 1, 64, 16, 3, 1, 1.0)
+    o2.compress_prompt(0, k[None, None], v[None, None], np.stack([q, q, q])[None, None], [4])
+    st2 = o2.export_unit(0, 0, 0)
+    assert st2["pos"].tolist() == [1, 4] and st2["word"].tolist() == [0b111, 0b001]
+    # with a window not yet full (w=4 > 3 usable rows... P=4 gives 4 rows; use w=5) nothing is evicted and the
+    # pre-eviction words of the two newest rows show in the low bits
+    o3 = CormOracle(1, 1, 1, 1, 64, 16, 5, 1, 1.0)
+    o3.compress_prompt(0, k[None, None], v[None, None], np.stack([q] * 5)[None, None], [4])
+    st3 = o3.export_unit(0, 0, 0)
+    assert st3["pos"].tolist() == [1, 2, 3, 4] and st3["n_obs"] == 4
+    assert [int(x) & 3 for x in st3["word"]] == [int(x, 2) for x in rows["words_before_eviction"]]
+
+
+def _random_case(rng, B, Hq, Hkv, d, P, steps, w, scale=1.5):
+    G = Hq // Hkv
+    k = rng.standard_normal((B, Hkv, P + steps, d)).astype(np.float32) * scale
+    v = rng.standard_normal((B, Hkv, P + steps, d)).astype(np.float32)
+    q = rng.standard_normal((B, Hq, w + steps, d)).astype(np.float32) * scale
+    return k, v, q, G
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_alpha_zero_is_full_attention(seed):
+    """alpha = 0 makes every key important, nothing is evicted, and each step is plain softmax(qK^T/sqrt(d))V over
+    all tokens so far, checked against torch's softmax in fp64."""
+    rng = np.random.default_rng(seed)
+    B, Hq, Hkv, d, P, steps, w, r = 2, 4, 2, 8, 5, 12, 3, 2
+    k, v, q, G = _random_case(rng, B, Hq, Hkv, d, P, steps, w)
+    o = CormOracle(1, B, Hq, Hkv, d, P + steps, w, r, 0.0)
+    o.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], [P] * B)
+    for s in range(steps):
+        out = o.decode_step(0, q[:, :, w + s], k[:, :, P + s], v[:, :, P + s])
+        n = P + s + 1
+        K = torch.from_numpy(k[:, :, :n]).double().repeat_interleave(G, dim=1)
+        V = torch.from_numpy(v[:, :, :n]).double().repeat_interleave(G, dim=1)
+        Q = torch.from_numpy(q[:, :, w + s]).double()
+        ref = torch.einsum("bhn,bhnd->bhd", torch.softmax(torch.einsum("bhd,bhnd->bhn", Q, K) / d ** 0.5, -1), V)
+        assert np.allclose(out, ref.numpy(), rtol=1e-12, atol=1e-12)
+        assert (o.live_lens(0) == n).all()
+    assert o.counters()["evicted"] == 0
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_shift_register_equals_literal_algorithm(seed):
+    """C oracle (shift registers) against the literal bool-matrix routine on random tiny cases, prompt included."""
+    rng = np.random.default_rng(1000 + seed)
+    Hkv = int(rng.integers(1, 3))
+    G = int(rng.integers(1, 4))
+    Hq, B = Hkv * G, int(rng.integers(1, 3))
+    d, w, r = int(rng.integers(1, 5)), int(rng.integers(1, 6)), int(rng.integers(1, 5))
+    P, steps = int(rng.integers(0, 9)), int(rng.integers(4, 16))
+    alpha = float(rng.choice([0.5, 1.0, 1.0, 2.0]))
+    k, v, q, _ = _random_case(rng, B, Hq, Hkv, d, P, steps, w, scale=2.0)
+    o = CormOracle(1, B, Hq, Hkv, d, P + steps, w, r, alpha)
+    lens = [P] * B
+    if B == 2 and P > 0:
+        lens[1] = int(rng.integers(0, P + 1))                  # ragged prompts
+    units = {}
+    for b in range(B):
+        for h in range(Hkv):
+            u = LiteralUnit(d, w, r, alpha)
+            u.compress_prompt(k[b, h, :lens[b]], v[b, h, :lens[b]], q[b, h * G:(h + 1) * G, :w])
+            units[b, h] = u
+    o.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], lens)
+    for s in range(steps + 1):
+        for b in range(B):
+            for h in range(Hkv):
+                st, u = o.export_unit(0, b, h), units[b, h]
+                assert st["pos"].tolist() == u.pos.tolist(), (s, b, h)
+                assert st["word"].tolist() == u.words().tolist(), (s, b, h)
+                assert np.array_equal(st["k"], u.keys) and np.array_equal(st["v"], u.values)
+        if s == steps:
+            break
+        k_new = np.stack([k[b, :, lens[b] + s] for b in range(B)])
+        v_new = np.stack([v[b, :, lens[b] + s] for b in range(B)])
+        out = o.decode_step(0, q[:, :, w + s], k_new, v_new)
+        for b in range(B):
+            for h in range(Hkv):
+                ref = units[b, h].decode_step(q[b, h * G:(h + 1) * G, w + s], k_new[b, h], v_new[b, h])
+                assert np.allclose(out[b, h * G:(h + 1) * G], ref, rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_bruteforce_eviction_sets(seed):
+    """t <= 16: verdicts recomputed with a library softmax, and the kept set identified by enumerating all subsets of
+    the live keys for the one that satisfies 'kept <=> recent, or important for some query among the last w'
+    (Definition 4.1 with the window of the Approach paragraph)."""
+    rng = np.random.default_rng(2000 + seed)
+    d, w, r, G = 3, int(rng.integers(1, 4)), int(rng.integers(1, 4)), int(rng.integers(1, 3))
+    alpha, steps = 1.0, 16
+    o = CormOracle(1, 1, G, 1, d, steps, w, r, alpha)
+    _empty_prompt(o, d)
+    k = (rng.standard_normal((steps, d)) * 2).astype(np.float32)
+    v = rng.standard_normal((steps, d)).astype(np.float32)
+    q = (rng.standard_normal((steps, G, d)) * 2).astype(np.float32)
+    history = []                                               # per step: {pos: verdict}
+    live = []                                                  # positions
+    for t in range(1, steps + 1):
+        live = live + [t]
+        K = torch.tensor(np.stack([k[p - 1] for p in live])).double()
+        verdict = {p: False for p in live}
+        for g in range(G):
+            prob = torch.softmax(K @ torch.tensor(q[t - 1, g]).double() / d ** 0.5, 0)
+            assert abs(float(prob.sum()) - 1) < 1e-12
+            for p, pr in zip(live, prob.tolist()):
+                verdict[p] = verdict[p] or pr >= alpha / t
+        history.append(verdict)
+        _, imp = o.decode_step(0, q[t - 1][None], k[t - 1][None, None], v[t - 1][None, None], want_verdicts=True)
+        assert imp[0, 0, :len(live)].tolist() == [int(verdict[p]) for p in live]
+        if len(history) >= w:
+            recent_rows = history[-w:]
+
+            def needed(p):
+                return p > t - r or any(row.get(p, False) for row in recent_rows)
+
+            valid = [S for n in range(len(live) + 1) for S in itertools.combinations(live, n)
+                     if all((p in S) == needed(p) for p in live)]
+            assert len(valid) == 1
+            live = list(valid[0])
+        assert o.export_unit(0, 0, 0)["pos"].tolist() == live
+
+
+def test_invariants_on_generated_workload():
+    from paper_2404_15949_b200.workload import CONFIGS, generate
+    cfg = CONFIGS[1].with_(prompt_min=96, prompt_max=96, steps=48, recent_r=16)
+    g = generate(cfg)
+    o = CormOracle(1, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.max_tokens, cfg.window_w,
+                   cfg.recent_r, cfg.alpha)
+    o.compress_prompt(0, g.k_prompt, g.v_prompt, g.q_last, g.prompt_lens)
+    prev = {h: o.export_unit(0, 0, h) for h in range(cfg.n_kv_heads)}
+    evicted_any = False
+    for s in range(cfg.steps):
+        t = 96 + s + 1
+        o.decode_step(0, g.q[s], g.k_new[s], g.v_new[s])
+        for h in range(cfg.n_kv_heads):
+            st = o.export_unit(0, 0, h)
+            pos = st["pos"]
+            assert (np.diff(pos) > 0).all()                                  # order kept
+            assert set(range(t - cfg.recent_r + 1, t + 1)) <= set(pos.tolist())  # recent r always live
+            assert set(pos.tolist()) <= set(prev[h]["pos"].tolist()) | {t}   # eviction is permanent
+            old = pos <= t - cfg.recent_r
+            assert (st["word"][old] != 0).all()                              # survivors outside the window are needed
+            assert st["live_len"] <= prev[h]["live_len"] + 1
+            evicted_any |= st["live_len"] < prev[h]["live_len"] + 1
+            prev[h] = st
+    c = o.counters()
+    assert evicted_any and c["appended"] - c["evicted"] == int(o.live_lens(0).sum())
+
+
+def test_warmup_blocks_eviction_until_w_rows():
+    rng = np.random.default_rng(7)
+    d, w, r, steps = 4, 5, 1, 9
+    o = CormOracle(1, 1, 1, 1, d, steps, w, r, 1.0)
+    _empty_prompt(o, d)
+    for t in range(1, steps + 1):
+        o.decode_step(0, rng.standard_normal((1, 1, d)).astype(np.float32) * 3,
+                      rng.standard_normal((1, 1, d)).astype(np.float32) * 3,
+                      rng.standard_normal((1, 1, d)).astype(np.float32))
+        if t < w:
+            assert o.live_len(0, 0, 0) == t and o.n_obs(0, 0) == t
+    assert o.n_obs(0, 0) == w and o.live_len(0, 0, 0) < steps
+
+
+def test_identical_keys_are_never_minor():
+    """All keys equal: every probability is exactly 1/l >= 1/t, so nothing can be evicted at alpha = 1."""
+    d, steps = 4, 20
+    o = CormOracle(1, 1, 1, 1, d, steps, 2, 1, 1.0)
+    _empty_prompt(o, d)
+    kv = np.ones((1, 1, d), np.float32)
+    for t in range(1, steps + 1):
+        out = o.decode_step(0, np.full((1, 1, d), 0.37, np.float32), kv, kv * t)
+        assert o.live_len(0, 0, 0) == t
+        assert np.allclose(out, (t + 1) / 2, rtol=1e-13)          # mean of 1..t
+
+
+def test_dominant_key_leaves_only_itself_and_the_recent_window():
+    d, w, r, steps = 8, 3, 4, 30
+    o = CormOracle(1, 1, 1, 1, d, steps, w, r, 1.0)
+    _empty_prompt(o, d)
+    q = np.zeros((1, 1, d), np.float32)
+    q[0, 0, 0] = np.sqrt(d)
+    for t in range(1, steps + 1):
+        k = np.zeros((1, 1, d), np.float32)
+        k[0, 0, 0] = 40.0 if t == 2 else 0.0                      # logit +40 over the rest
+        o.decode_step(0, q, k, np.ones((1, 1, d), np.float32))
+        if t > r + w + 2:
+            assert o.export_unit(0, 0, 0)["pos"].tolist() == [2] + list(range(t - r + 1, t + 1))
+
+
+def test_group_of_identical_heads_equals_single_head_and_or_rule():
+    rng = np.random.default_rng(11)
+    d, w, r, P, steps = 6, 3, 2, 7, 14
+    k, v, q, _ = _random_case(rng, 1, 1, 1, d, P, steps, w, scale=2.0)
+    single = CormOracle(1, 1, 1, 1, d, P + steps, w, r, 1.0)
+    group = CormOracle(1, 1, 3, 1, d, P + steps, w, r, 1.0)
+    q3 = np.repeat(q, 3, axis=1)
+    single.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], [P])
+    group.compress_prompt(0, k[:, :, :P], v[:, :, :P], q3[:, :, :w], [P])
+    for s in range(steps):
+        a = single.decode_step(0, q[:, :, w + s], k[:, :, P + s], v[:, :, P + s])
+        b = group.decode_step(0, q3[:, :, w + s], k[:, :, P + s], v[:, :, P + s])
+        assert np.array_equal(np.repeat(a, 3, axis=1), b)
+        sa, sb = single.export_unit(0, 0, 0), group.export_unit(0, 0, 0)
+        assert sa["pos"].tolist() == sb["pos"].tolist() and sa["word"].tolist() == sb["word"].tolist()
+    # OR rule: a group's verdict is the union of what each head alone would say on the same cache
+    two = CormOracle(1, 1, 2, 1, d, 4, 8, 8, 1.0)
+    ones = [CormOracle(1, 1, 1, 1, d, 4, 8, 8, 1.0) for _ in range(2)]
+    for o in [two] + ones:
+        _empty_prompt(o, d)
+    qq = (rng.standard_normal((4, 1, 2, d)) * 3).astype(np.float32)
+    for t in range(4):
+        kn, vn = k[:, :, t], v[:, :, t]
+        _, imp = two.decode_step(0, qq[t], kn, vn, want_verdicts=True)
+        sep = [o.decode_step(0, qq[t][:, g:g + 1], kn, vn, want_verdicts=True)[1] for g, o in enumerate(ones)]
+        assert np.array_equal(imp, sep[0] | sep[1])
+
+
+def test_positive_query_scaling_keeps_the_ranking():
+    """Eq. 4: q and m*q (m > 0) rank the keys identically, so their important sets are nested."""
+    rng = np.random.default_rng(5)
+    d, n = 8, 12
+    k = rng.standard_normal((n, d)).astype(np.float32) * 2
+    q = rng.standard_normal((d,)).astype(np.float32)
+    sets = []
+    for m in (0.25, 1.0, 3.0):
+        o = CormOracle(1, 1, 1, 1, d, n, 32, 32, 1.0)
+        _empty_prompt(o, d)
+        for j in range(n - 1):                                      # fill the cache (r = 32: no evictions)
+            o.decode_step(0, np.zeros((1, 1, d), np.float32), k[j][None, None], k[j][None, None])
+        _, imp = o.decode_step(0, (m * q)[None, None], k[n - 1][None, None], k[n - 1][None, None], want_verdicts=True)
+        sets.append(set(np.nonzero(imp[0, 0])[0].tolist()))
+    ranked = sorted(sets, key=len)
+    assert ranked[0] <= ranked[1] <= ranked[2] and len(ranked[2]) >= 1
+
+
+def test_near_threshold_band_counter():
+    """Keys sitting exactly on the threshold (identical keys, l = t) are counted inside the band."""
+    d = 4
+    o = CormOracle(1, 1, 1, 1, d, 8, 2, 1, 1.0)
+    _empty_prompt(o, d)
+    kv = np.ones((1, 1, d), np.float32)
+    for _ in range(5):
+        o.decode_step(0, kv, kv, kv)
+    c = o.counters()
+    assert c["near_threshold"] == c["verdict_evals"] == 1 + 2 + 3 + 4 + 5
+
+
+def test_bad_arguments_and_capacity():
+    with pytest.raises(ValueError):
+        CormOracle(1, 1, 3, 2, 4, 8, 2, 1, 1.0)
+    with pytest.raises(ValueError):
+        CormOracle(1, 1, 1, 1, 4, 8, 2, 0, 1.0)                 # r = 0 is rejected (the slice [-0:] selects everything)
+    o = CormOracle(1, 1, 1, 1, 4, 2, 2, 1, 0.0)
+    _empty_prompt(o, 4)
+    x = np.ones((1, 1, 4), np.float32)
+    o.decode_step(0, x, x, x)
+    o.decode_step(0, x, x, x)
+    with pytest.raises(RuntimeError):
+        o.decode_step(0, x, x, x)
