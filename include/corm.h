@@ -1,0 +1,142 @@
+/*
+ * corm.h — C ABI of the CORM hot path for NVIDIA B200 (sm_100a).
+ *
+ * CORM ("Cache Optimization with Recent Message") evicts a cached key/value pair once the key has been judged
+ * minor by every one of the last w queries (Definition 4.1 with the window of the "Approach" paragraph), where a
+ * key is important for the query of step t iff its softmax probability is at least alpha/t (Definition 3.1; the
+ * paper uses alpha = 1), and never evicts the r most recent tokens (Algorithm 1). The policy runs per head and per
+ * layer; with grouped-query attention a shared KV head keeps a key while any query head of its group still needs
+ * it (Section 5, "Integrate into grouped-query attention").
+ *
+ * A "unit" is one (layer, sequence, kv head). Each unit owns a slab of max_tokens slots holding K rows, V rows,
+ * one w-bit verdict register per key (bit b = verdict of the query b steps ago) and the key's absolute 1-based
+ * token position. Live entries occupy slots [0, live_len); their slot ORDER IS NOT the token order once decode
+ * steps have evicted keys (holes are filled from the tail), so recency is always decided from the stored position.
+ *
+ * Conventions
+ *  - Every pointer argument says "device" or "host". Device buffers are owned by the caller, including the
+ *    arena; the library never allocates or frees device memory. corm_cache_t owns host metadata only.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Calls that enqueue work are
+ *    asynchronous; all calls on one cache must be issued in stream order (they share scratch inside the arena).
+ *  - Tensors are row-major and dense; kv_dtype is the element type of the cache, q, k_new, v_new and out.
+ *  - Host-detectable errors return a status and enqueue nothing. Device-detected ones (a unit that would exceed
+ *    max_tokens) set a sticky device status, skip that unit, never trap or hang, and show in corm_cache_stats.
+ */
+#ifndef CORM_H_
+#define CORM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct corm_cache corm_cache_t;
+
+typedef enum {
+    CORM_OK = 0,
+    CORM_ERR_INVALID_ARG = 1,
+    CORM_ERR_UNSUPPORTED = 2,
+    CORM_ERR_ARENA_TOO_SMALL = 3,
+    CORM_ERR_STATE = 4,
+    CORM_ERR_CUDA = 5,
+    CORM_ERR_CAPACITY = 6,
+    CORM_ERR_TIMEOUT = 7
+} corm_status_t;
+
+typedef enum { CORM_F32 = 0, CORM_BF16 = 1 } corm_dtype_t;
+
+typedef struct {
+    int32_t n_layers, batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group size in {1,2,4,8} */
+    int32_t head_dim;                                /* 64 or 128 */
+    int32_t max_tokens;                              /* slab capacity per unit: >= longest prompt + decode steps */
+    int32_t window_w;                                /* 1..32: one 32-bit register per key */
+    int32_t recent_r;                                /* >= 1 (Algorithm 1's slice of the last r entries) */
+    float   alpha;                                   /* >= 0; threshold alpha/t; 0 means nothing is ever evicted */
+    int32_t kv_dtype;                                /* corm_dtype_t */
+    int32_t device;                                  /* CUDA device ordinal of the arena */
+} corm_config_t;
+
+typedef struct {
+    int64_t live_keys, appended_keys, evicted_keys; /* summed over all units */
+    double  retention;                               /* live / appended (1 when nothing was appended) */
+    int64_t kv_bytes_live, aux_bytes_live;           /* K+V bytes; register + position bytes */
+    int64_t moved_rows;                              /* rows copied by hole-filling compaction so far */
+    int64_t attended_keys;                           /* sum over decode steps and units of the live length read */
+    int32_t device_status;                           /* first device-side error (corm_status_t), CORM_OK if none */
+} corm_stats_t;
+
+/* Bytes of device memory a cache with this configuration needs (host, pure). 0 if the configuration is invalid. */
+size_t corm_cache_arena_bytes(const corm_config_t* cfg);
+
+/* Builds the host object over a caller-allocated device arena (256-byte aligned, >= corm_cache_arena_bytes) and
+ * zeroes the bookkeeping part of the arena on the legacy default stream, synchronously.
+ * Errors: INVALID_ARG (null/invalid fields), UNSUPPORTED (head_dim, group, w > 32), ARENA_TOO_SMALL, CUDA. */
+corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, size_t arena_bytes,
+                                corm_cache_t** out);
+corm_status_t corm_cache_destroy(corm_cache_t* cache);
+
+/* Empties every unit (asynchronous on `stream`); a prompt pass is needed again before decoding. */
+corm_status_t corm_cache_reset(corm_cache_t* cache, void* stream);
+
+/* Prompt-end pass for one layer (the paper covers generation only; this applies Algorithm 1's recording and
+ * eviction to the causal attention rows, Eq. 2, of the last min(P, w) prompt queries over the full prompt: the
+ * query at position i uses threshold alpha/i, keys newer than a query get a 0 bit as Algorithm 1's zero padding
+ * prescribes, and one eviction with t = P follows when w rows exist).
+ *   k_prompt, v_prompt  device [batch, n_kv_heads, p_max, head_dim]; rows >= prompt_lens[b] are ignored
+ *   q_last              device [batch, n_q_heads, window_w, head_dim]: queries of positions P-w+1..P, oldest
+ *                       first; for P < w the first w-P rows are ignored
+ *   prompt_lens_host    host [batch], 0 <= P_b <= min(p_max, max_tokens); P_b = 0 leaves the unit empty
+ * Survivors are written to the slabs in token order. Produces no attention output. */
+corm_status_t corm_compress_prompt(corm_cache_t* cache, int32_t layer, const void* k_prompt, const void* v_prompt,
+                                   const void* q_last, const int32_t* prompt_lens_host, int32_t p_max,
+                                   void* stream);
+
+/* One decode step of one layer for all sequences (Algorithm 1 around Eq. 1/Eq. 2):
+ * appends (k_new, v_new) as token t = tokens_so_far + 1, computes out = softmax(q K^T / sqrt(head_dim)) V over the
+ * live keys including the new one, marks each key important iff its probability >= alpha/t for at least one query
+ * head of its group, shifts that verdict into the key's register, and, once w verdict rows exist, removes keys
+ * whose register is zero and whose position is <= t - r. The output uses the cache before this step's eviction.
+ *   q      device [batch, n_q_heads, head_dim]
+ *   k_new  device [batch, n_kv_heads, head_dim], v_new likewise
+ *   out    device [batch, n_q_heads, head_dim]
+ * Errors: STATE if the layer has had no corm_compress_prompt since create/reset; INVALID_ARG. */
+corm_status_t corm_decode_step(corm_cache_t* cache, int32_t layer, const void* q, const void* k_new,
+                               const void* v_new, void* out, void* stream);
+
+/* Same step with HOST buffers (pinned memory recommended): copies q, k_new, v_new to staging space inside the
+ * arena, runs the step and copies out back, all asynchronously on `stream`. */
+corm_status_t corm_decode_step_host(corm_cache_t* cache, int32_t layer, const void* q_host, const void* k_new_host,
+                                    const void* v_new_host, void* out_host, void* stream);
+
+/* Totals over all units ("compression rate" of Section 5). Synchronises `stream`. */
+corm_status_t corm_cache_stats(corm_cache_t* cache, corm_stats_t* out_host, void* stream);
+
+/* Live length of every unit of one layer: live_host [batch, n_kv_heads]. Synchronises `stream`. */
+corm_status_t corm_cache_live_lens(corm_cache_t* cache, int32_t layer, int32_t* live_host, void* stream);
+
+/* Test / checkpoint hooks. Host buffers hold max_tokens entries; entries come in SLOT order (see above).
+ * k_host, v_host: [max_tokens, head_dim] in kv_dtype; word_host, pos_host: [max_tokens]; scalars by pointer.
+ * n_tokens / n_obs are per (layer, sequence): tokens seen and verdict rows recorded (<= w). Synchronise `stream`. */
+corm_status_t corm_cache_export_state(corm_cache_t* cache, int32_t layer, int32_t seq, int32_t kv_head,
+                                      void* k_host, void* v_host, uint32_t* word_host, int32_t* pos_host,
+                                      int32_t* live_len, int32_t* n_tokens, int32_t* n_obs, void* stream);
+corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_t seq, int32_t kv_head,
+                                      const void* k_host, const void* v_host, const uint32_t* word_host,
+                                      const int32_t* pos_host, int32_t live_len, int32_t n_tokens, int32_t n_obs,
+                                      void* stream);
+
+/* Tuning knobs (performance only; results do not depend on them): keys per split of the decode kernel
+ * (multiple of 32, 0 = automatic) and whether the fast bf16/head_dim-128 kernel may be used. */
+corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
+
+/* Number of kernels this library has launched on behalf of `cache` since create. */
+int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
+
+const char* corm_status_string(corm_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CORM_H_ */

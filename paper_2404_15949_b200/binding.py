@@ -1,0 +1,224 @@
+"""Thin ctypes binding over ``libcorm.so`` — argument marshalling only, same names as ``include/corm.h``.
+
+PyTorch supplies device memory (the arena and the tensors) and the CUDA stream; every step of the path runs inside
+the library's kernels. There is no CPU fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+from .build import LIB_PATH
+
+CORM_OK = 0
+CORM_F32, CORM_BF16 = 0, 1
+STATUS_NAMES = {0: "CORM_OK", 1: "CORM_ERR_INVALID_ARG", 2: "CORM_ERR_UNSUPPORTED", 3: "CORM_ERR_ARENA_TOO_SMALL",
+                4: "CORM_ERR_STATE", 5: "CORM_ERR_CUDA", 6: "CORM_ERR_CAPACITY", 7: "CORM_ERR_TIMEOUT"}
+
+
+class CormConfig(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("max_tokens", ctypes.c_int32),
+                ("window_w", ctypes.c_int32), ("recent_r", ctypes.c_int32), ("alpha", ctypes.c_float),
+                ("kv_dtype", ctypes.c_int32), ("device", ctypes.c_int32)]
+
+
+class CormStats(ctypes.Structure):
+    _fields_ = [("live_keys", ctypes.c_int64), ("appended_keys", ctypes.c_int64), ("evicted_keys", ctypes.c_int64),
+                ("retention", ctypes.c_double), ("kv_bytes_live", ctypes.c_int64), ("aux_bytes_live", ctypes.c_int64),
+                ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32)]
+
+
+class CormError(RuntimeError):
+    def __init__(self, call, status):
+        self.status = status
+        super().__init__(f"{call} -> {STATUS_NAMES.get(status, status)}")
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen the in-tree library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run paper_2404_15949_b200.build.build_library() "
+                           "(or __graft_entry__.build()) first; the CORM path has no CPU fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    cfgp = ctypes.POINTER(CormConfig)
+    lib.corm_cache_arena_bytes.restype = sz
+    lib.corm_cache_arena_bytes.argtypes = [cfgp]
+    lib.corm_cache_create.restype = i32
+    lib.corm_cache_create.argtypes = [cfgp, vp, sz, ctypes.POINTER(vp)]
+    lib.corm_cache_destroy.restype = i32
+    lib.corm_cache_destroy.argtypes = [vp]
+    lib.corm_cache_reset.restype = i32
+    lib.corm_cache_reset.argtypes = [vp, vp]
+    lib.corm_compress_prompt.restype = i32
+    lib.corm_compress_prompt.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp]
+    lib.corm_decode_step.restype = i32
+    lib.corm_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.corm_decode_step_host.restype = i32
+    lib.corm_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.corm_cache_stats.restype = i32
+    lib.corm_cache_stats.argtypes = [vp, ctypes.POINTER(CormStats), vp]
+    lib.corm_cache_live_lens.restype = i32
+    lib.corm_cache_live_lens.argtypes = [vp, i32, vp, vp]
+    lib.corm_cache_export_state.restype = i32
+    lib.corm_cache_export_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.corm_cache_import_state.restype = i32
+    lib.corm_cache_import_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp]
+    lib.corm_cache_set_tuning.restype = i32
+    lib.corm_cache_set_tuning.argtypes = [vp, i32, i32]
+    lib.corm_cache_kernel_launches.restype = i64
+    lib.corm_cache_kernel_launches.argtypes = [vp]
+    lib.corm_status_string.restype = ctypes.c_char_p
+    lib.corm_status_string.argtypes = [i32]
+    _lib = lib
+    return lib
+
+
+def _check(call, rc):
+    if rc != CORM_OK:
+        raise CormError(call, rc)
+
+
+def _stream_ptr(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _torch_dtype(kv_dtype):
+    return torch.bfloat16 if kv_dtype == CORM_BF16 else torch.float32
+
+
+def _np_view_dtype(kv_dtype):
+    return np.uint16 if kv_dtype == CORM_BF16 else np.float32
+
+
+def corm_cache_arena_bytes(cfg: CormConfig) -> int:
+    return int(load_library().corm_cache_arena_bytes(ctypes.byref(cfg)))
+
+
+class CormCache:
+    """Owns the arena tensor (torch device memory) and the library's host object."""
+
+    def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, window_w, recent_r, alpha,
+                 kv_dtype="bf16", device=0):
+        self.lib = load_library()
+        code = {"bf16": CORM_BF16, "f32": CORM_F32}[kv_dtype]
+        self.cfg = CormConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, window_w, recent_r,
+                              float(alpha), code, device)
+        self.kv_dtype, self.dtype, self.device = code, _torch_dtype(code), torch.device("cuda", device)
+        nbytes = corm_cache_arena_bytes(self.cfg)
+        if nbytes == 0:
+            raise CormError("corm_cache_arena_bytes", 1)
+        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        handle = ctypes.c_void_p()
+        _check("corm_cache_create", self.lib.corm_cache_create(ctypes.byref(self.cfg), self.arena.data_ptr(), nbytes,
+                                                               ctypes.byref(handle)))
+        self.handle = handle
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.corm_cache_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    # ---- the four calls of the boundary -------------------------------------------------------------------------
+    def corm_compress_prompt(self, layer, k_prompt, v_prompt, q_last, prompt_lens, stream=None):
+        lens = np.ascontiguousarray(prompt_lens, dtype=np.int32)
+        assert lens.shape == (self.cfg.batch,)
+        p_max = int(k_prompt.shape[2]) if k_prompt is not None else 0
+        for t in (k_prompt, v_prompt, q_last):
+            assert t is None or (t.is_cuda and t.is_contiguous() and t.dtype == self.dtype)
+        if p_max:
+            assert tuple(k_prompt.shape) == (self.cfg.batch, self.cfg.n_kv_heads, p_max, self.cfg.head_dim)
+            assert tuple(v_prompt.shape) == tuple(k_prompt.shape)
+            assert tuple(q_last.shape) == (self.cfg.batch, self.cfg.n_q_heads, self.cfg.window_w, self.cfg.head_dim)
+        ptr = lambda t: t.data_ptr() if (t is not None and t.numel()) else None
+        _check("corm_compress_prompt", self.lib.corm_compress_prompt(
+            self.handle, layer, ptr(k_prompt), ptr(v_prompt), ptr(q_last), lens.ctypes.data, p_max,
+            _stream_ptr(stream)))
+
+    def corm_decode_step(self, layer, q, k_new, v_new, out=None, stream=None):
+        c = self.cfg
+        assert tuple(q.shape) == (c.batch, c.n_q_heads, c.head_dim) and q.dtype == self.dtype and q.is_contiguous()
+        assert tuple(k_new.shape) == (c.batch, c.n_kv_heads, c.head_dim) and k_new.is_contiguous()
+        assert tuple(v_new.shape) == tuple(k_new.shape) and v_new.is_contiguous()
+        assert k_new.dtype == self.dtype and v_new.dtype == self.dtype and q.is_cuda and k_new.is_cuda and v_new.is_cuda
+        if out is None:
+            out = torch.empty_like(q)
+        _check("corm_decode_step", self.lib.corm_decode_step(self.handle, layer, q.data_ptr(), k_new.data_ptr(),
+                                                             v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)))
+        return out
+
+    def corm_decode_step_host(self, layer, q, k_new, v_new, out, stream=None):
+        """Host (pinned) tensors in and out; the copies run inside the library on the same stream."""
+        for t in (q, k_new, v_new, out):
+            assert not t.is_cuda and t.is_contiguous() and t.dtype == self.dtype
+        _check("corm_decode_step_host", self.lib.corm_decode_step_host(
+            self.handle, layer, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)))
+        return out
+
+    def corm_cache_stats(self, stream=None):
+        st = CormStats()
+        _check("corm_cache_stats", self.lib.corm_cache_stats(self.handle, ctypes.byref(st), _stream_ptr(stream)))
+        return {name: getattr(st, name) for name, _ in CormStats._fields_}
+
+    # ---- helpers --------------------------------------------------------------------------------------------------
+    def corm_cache_reset(self, stream=None):
+        _check("corm_cache_reset", self.lib.corm_cache_reset(self.handle, _stream_ptr(stream)))
+
+    def corm_cache_live_lens(self, layer, stream=None):
+        out = np.empty((self.cfg.batch, self.cfg.n_kv_heads), dtype=np.int32)
+        _check("corm_cache_live_lens", self.lib.corm_cache_live_lens(self.handle, layer, out.ctypes.data,
+                                                                     _stream_ptr(stream)))
+        return out
+
+    def corm_cache_set_tuning(self, split_len=0, allow_fast_path=True):
+        _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
+
+    def corm_cache_kernel_launches(self):
+        return int(self.lib.corm_cache_kernel_launches(self.handle))
+
+    def corm_cache_export_state(self, layer, seq, kv_head, stream=None):
+        """Live entries of one unit in slot order: k, v as float32 arrays [live, d], word, pos, counters."""
+        c = self.cfg
+        vt = _np_view_dtype(self.kv_dtype)
+        k = np.empty((c.max_tokens, c.head_dim), dtype=vt)
+        v = np.empty((c.max_tokens, c.head_dim), dtype=vt)
+        word = np.empty((c.max_tokens,), dtype=np.uint32)
+        pos = np.empty((c.max_tokens,), dtype=np.int32)
+        live, n_tokens, n_obs = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        _check("corm_cache_export_state", self.lib.corm_cache_export_state(
+            self.handle, layer, seq, kv_head, k.ctypes.data, v.ctypes.data, word.ctypes.data, pos.ctypes.data,
+            ctypes.byref(live), ctypes.byref(n_tokens), ctypes.byref(n_obs), _stream_ptr(stream)))
+        n = live.value
+        widen = (lambda a: (a[:n].astype(np.uint32) << 16).view(np.float32)) if self.kv_dtype == CORM_BF16 else (
+            lambda a: a[:n].copy())
+        return dict(k=widen(k), v=widen(v), word=word[:n].copy(), pos=pos[:n].copy(), live_len=n,
+                    n_tokens=n_tokens.value, n_obs=n_obs.value)
+
+    def corm_cache_import_state(self, layer, seq, kv_head, k, v, word, pos, n_tokens, n_obs, stream=None):
+        """k, v: float arrays [live, d] whose values are representable in the cache dtype."""
+        k32 = np.ascontiguousarray(k, dtype=np.float32)
+        v32 = np.ascontiguousarray(v, dtype=np.float32)
+        if self.kv_dtype == CORM_BF16:
+            assert not (k32.view(np.uint32) & 0xffff).any() and not (v32.view(np.uint32) & 0xffff).any()
+            kk = np.ascontiguousarray((k32.view(np.uint32) >> 16).astype(np.uint16))
+            vv = np.ascontiguousarray((v32.view(np.uint32) >> 16).astype(np.uint16))
+        else:
+            kk, vv = k32, v32
+        word = np.ascontiguousarray(word, dtype=np.uint32)
+        pos = np.ascontiguousarray(pos, dtype=np.int32)
+        _check("corm_cache_import_state", self.lib.corm_cache_import_state(
+            self.handle, layer, seq, kv_head, kk.ctypes.data, vv.ctypes.data, word.ctypes.data, pos.ctypes.data,
+            int(kk.shape[0]), int(n_tokens), int(n_obs), _stream_ptr(stream)))

@@ -1,0 +1,462 @@
+// Host side of the C-ABI library: arena layout, argument checks, launch configuration. Every step of the hot
+// path runs in the kernels of corm_generic.cuh / corm_fast.cuh; nothing here touches tensor data on the CPU.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <type_traits>
+#include <vector>
+
+#include "../../include/corm.h"
+#include "corm_common.cuh"
+#include "corm_fast.cuh"
+#include "corm_generic.cuh"
+
+using namespace corm;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kMinSplit = 64;
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Layout {
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, stash, partials;
+    size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
+};
+
+bool config_ok(const corm_config_t* c, corm_status_t* why) {
+    *why = CORM_ERR_INVALID_ARG;
+    if (!c) return false;
+    if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return false;
+    if (c->n_q_heads % c->n_kv_heads) return false;
+    if (c->max_tokens < 1 || c->window_w < 1 || c->recent_r < 1) return false;
+    if (!(c->alpha >= 0.f) || !std::isfinite(c->alpha)) return false;
+    if (c->kv_dtype != CORM_F32 && c->kv_dtype != CORM_BF16) return false;
+    if (c->device < 0) return false;
+    *why = CORM_ERR_UNSUPPORTED;
+    const int G = c->n_q_heads / c->n_kv_heads;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return false;
+    if (c->window_w > 32) return false;
+    if ((long long)c->batch * c->n_kv_heads > 65535) return false;     // grid.y of the decode kernel
+    if (c->max_tokens > (1 << 22)) return false;
+    *why = CORM_OK;
+    return true;
+}
+
+int max_splits_of(const corm_config_t& c) { return (c.max_tokens + kMinSplit - 1) / kMinSplit; }
+
+Layout make_layout(const corm_config_t& c) {
+    Layout L{};
+    const size_t U = (size_t)c.batch * c.n_kv_heads, Ltot = c.n_layers, C = c.max_tokens, D = c.head_dim;
+    const size_t e = c.kv_dtype == CORM_BF16 ? 2 : 4, G = c.n_q_heads / c.n_kv_heads;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+    L.K = take(Ltot * U * C * D * e);
+    L.V = take(Ltot * U * C * D * e);
+    L.word = take(Ltot * U * C * 4);
+    L.pos = take(Ltot * U * C * 4);
+    L.bookkeeping_begin = off;
+    L.live = take(Ltot * 2 * U * 4);
+    L.base_tokens = take(Ltot * c.batch * 4);
+    L.base_obs = take(Ltot * c.batch * 4);
+    L.ticket = take(Ltot * U * 4);
+    L.counters = take(Ltot * CNT_COUNT * 8);
+    L.status = take(4);
+    L.bookkeeping_end = off;
+    L.stash = take(U * G * C * 8);
+    L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
+    L.stage_q = take((size_t)c.batch * c.n_q_heads * D * e);
+    L.stage_k = take(U * D * e);
+    L.stage_v = take(U * D * e);
+    L.stage_out = take((size_t)c.batch * c.n_q_heads * D * e);
+    L.total = off;
+    return L;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define CORM_CUDA(expr)                                                         \
+    do {                                                                        \
+        cudaError_t e_ = (expr);                                                \
+        if (e_ != cudaSuccess) {                                                \
+            std::fprintf(stderr, "corm: %s failed: %s\n", #expr, cudaGetErrorString(e_)); \
+            return CORM_ERR_CUDA;                                               \
+        }                                                                       \
+    } while (0)
+
+}  // namespace
+
+struct corm_cache {
+    corm_config_t cfg;
+    Layout lay;
+    unsigned char* arena;
+    int U, G;
+    size_t e;
+    std::vector<int> parity, steps, ready, live_upper;
+    int tune_split_len = 0, allow_fast = 1;
+    int sm_count = 148;
+    long long launches = 0;
+};
+
+namespace {
+
+template <typename F> corm_status_t dispatch(const corm_cache* c, F&& f) {
+    const bool bf = c->cfg.kv_dtype == CORM_BF16;
+    const int D = c->cfg.head_dim, G = c->G;
+#define CORM_CASE(TT, DD, GG) if (D == DD && G == GG) return f((TT*)nullptr, std::integral_constant<int, DD>(), std::integral_constant<int, GG>());
+    if (bf) {
+        CORM_CASE(bf16_t, 64, 1) CORM_CASE(bf16_t, 64, 2) CORM_CASE(bf16_t, 64, 4) CORM_CASE(bf16_t, 64, 8)
+        CORM_CASE(bf16_t, 128, 1) CORM_CASE(bf16_t, 128, 2) CORM_CASE(bf16_t, 128, 4) CORM_CASE(bf16_t, 128, 8)
+    } else {
+        CORM_CASE(float, 64, 1) CORM_CASE(float, 64, 2) CORM_CASE(float, 64, 4) CORM_CASE(float, 64, 8)
+        CORM_CASE(float, 128, 1) CORM_CASE(float, 128, 2) CORM_CASE(float, 128, 4) CORM_CASE(float, 128, 8)
+    }
+#undef CORM_CASE
+    return CORM_ERR_UNSUPPORTED;
+}
+
+unsigned char* layer_ptr(const corm_cache* c, size_t base, size_t per_layer_bytes, int layer) {
+    return c->arena + base + per_layer_bytes * (size_t)layer;
+}
+
+int32_t* live_buf(const corm_cache* c, int layer, int parity) {
+    return reinterpret_cast<int32_t*>(c->arena + c->lay.live) + ((size_t)layer * 2 + parity) * c->U;
+}
+
+bool layer_ok(const corm_cache* c, int layer) { return c && layer >= 0 && layer < c->cfg.n_layers; }
+
+double log_alpha_of(const corm_cache* c) { return c->cfg.alpha > 0.f ? std::log((double)c->cfg.alpha) : -INFINITY; }
+
+corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
+                            cudaStream_t st) {
+    const corm_config_t& cf = c->cfg;
+    const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
+    DecodeParams p{};
+    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
+    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
+    p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
+    p.live_in = live_buf(c, layer, c->parity[layer]);
+    p.live_out = live_buf(c, layer, c->parity[layer] ^ 1);
+    p.base_tokens = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer));
+    p.base_obs = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer));
+    p.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
+    p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
+    p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
+    p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
+    p.partials = c->arena + c->lay.partials;
+    p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
+    p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
+    p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
+    p.log_alpha = log_alpha_of(c);
+    const int upper = std::min(cf.max_tokens, c->live_upper[layer] + 1);   // no unit can hold more live keys
+
+    const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128;
+    corm_status_t rc;
+    if (fast) {
+        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st);
+    } else {
+        p.split_len = c->tune_split_len ? c->tune_split_len : 256;
+        const int n_splits = (upper + p.split_len - 1) / p.split_len;
+        rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
+            using T = std::remove_pointer_t<decltype(tp)>;
+            constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
+            const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
+            auto kern = decode_generic_kernel<T, DD, GG>;
+            if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
+            CORM_CUDA(cudaGetLastError());
+            return CORM_OK;
+        });
+    }
+    if (rc != CORM_OK) return rc;
+    c->launches += 1;
+    c->parity[layer] ^= 1;
+    c->steps[layer] += 1;
+    c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
+    return CORM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t corm_cache_arena_bytes(const corm_config_t* cfg) {
+    corm_status_t why;
+    if (!config_ok(cfg, &why)) return 0;
+    return make_layout(*cfg).total;
+}
+
+corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, size_t arena_bytes, corm_cache_t** out) {
+    corm_status_t why;
+    if (!out) return CORM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg, &why)) return why;
+    if (!arena_device || (reinterpret_cast<uintptr_t>(arena_device) % kAlign)) return CORM_ERR_INVALID_ARG;
+    Layout lay = make_layout(*cfg);
+    if (arena_bytes < lay.total) return CORM_ERR_ARENA_TOO_SMALL;
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    corm_cache* c = new (std::nothrow) corm_cache();
+    if (!c) return CORM_ERR_INVALID_ARG;
+    c->cfg = *cfg;
+    c->lay = lay;
+    c->arena = static_cast<unsigned char*>(arena_device);
+    c->U = cfg->batch * cfg->n_kv_heads;
+    c->G = cfg->n_q_heads / cfg->n_kv_heads;
+    c->e = cfg->kv_dtype == CORM_BF16 ? 2 : 4;
+    c->parity.assign(cfg->n_layers, 0);
+    c->steps.assign(cfg->n_layers, 0);
+    c->ready.assign(cfg->n_layers, 0);
+    c->live_upper.assign(cfg->n_layers, 0);
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) c->sm_count = sms;
+    cudaError_t e = cudaMemset(c->arena + lay.bookkeeping_begin, 0, lay.bookkeeping_end - lay.bookkeeping_begin);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        std::fprintf(stderr, "corm: clearing the arena failed: %s\n", cudaGetErrorString(e));
+        delete c;
+        return CORM_ERR_CUDA;
+    }
+    *out = c;
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_destroy(corm_cache_t* cache) {
+    if (!cache) return CORM_ERR_INVALID_ARG;
+    delete cache;
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
+    if (!c) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    CORM_CUDA(cudaMemsetAsync(c->arena + c->lay.bookkeeping_begin, 0, c->lay.bookkeeping_end - c->lay.bookkeeping_begin,
+                              static_cast<cudaStream_t>(stream)));
+    for (int l = 0; l < c->cfg.n_layers; ++l) { c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; }
+    return CORM_OK;
+}
+
+corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k_prompt, const void* v_prompt,
+                                   const void* q_last, const int32_t* prompt_lens_host, int32_t p_max, void* stream) {
+    if (!layer_ok(c, layer) || !prompt_lens_host || p_max < 0) return CORM_ERR_INVALID_ARG;
+    const corm_config_t& cf = c->cfg;
+    int max_p = 0;
+    std::vector<int32_t> obs(cf.batch);
+    for (int b = 0; b < cf.batch; ++b) {
+        const int P = prompt_lens_host[b];
+        if (P < 0 || P > p_max) return CORM_ERR_INVALID_ARG;
+        if (P > cf.max_tokens) return CORM_ERR_CAPACITY;
+        max_p = std::max(max_p, P);
+        obs[b] = std::min(P, cf.window_w);
+    }
+    if (max_p > 0 && (!k_prompt || !v_prompt || !q_last)) return CORM_ERR_INVALID_ARG;
+    if (max_p > 0 && ((reinterpret_cast<uintptr_t>(k_prompt) | reinterpret_cast<uintptr_t>(v_prompt) |
+                       reinterpret_cast<uintptr_t>(q_last)) % 16)) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(cf.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
+    int32_t* base_tokens = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer));
+    int32_t* base_obs = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer));
+    // pageable sources are staged by the runtime before these calls return
+    CORM_CUDA(cudaMemcpyAsync(base_tokens, prompt_lens_host, (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemcpyAsync(base_obs, obs.data(), (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket, U * 4, layer), 0, U * 4, st));
+    PromptParams p{};
+    p.k_prompt = k_prompt; p.v_prompt = v_prompt; p.q_last = q_last;
+    p.prompt_lens = base_tokens;
+    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
+    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
+    p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
+    p.live_out = live_buf(c, layer, 0);
+    p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
+    p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
+    p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
+    p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.p_max = p_max; p.w = cf.window_w; p.r = cf.recent_r;
+    p.log_alpha = log_alpha_of(c);
+    corm_status_t rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
+        using T = std::remove_pointer_t<decltype(tp)>;
+        constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
+        const size_t smem = prompt_smem(GG, cf.window_w, cf.max_tokens);
+        auto kern = prompt_generic_kernel<T, DD, GG>;
+        if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<(unsigned)U, kPromptThreads, smem, st>>>(p);
+        CORM_CUDA(cudaGetLastError());
+        return CORM_OK;
+    });
+    if (rc != CORM_OK) return rc;
+    c->launches += 1;
+    c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p;
+    return CORM_OK;
+}
+
+corm_status_t corm_decode_step(corm_cache_t* c, int32_t layer, const void* q, const void* k_new, const void* v_new,
+                               void* out, void* stream) {
+    if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return CORM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+         reinterpret_cast<uintptr_t>(out)) % 16) return CORM_ERR_INVALID_ARG;
+    if (!c->ready[layer]) return CORM_ERR_STATE;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    return launch_decode(c, layer, q, k_new, v_new, out, static_cast<cudaStream_t>(stream));
+}
+
+corm_status_t corm_decode_step_host(corm_cache_t* c, int32_t layer, const void* q_host, const void* k_new_host,
+                                    const void* v_new_host, void* out_host, void* stream) {
+    if (!layer_ok(c, layer) || !q_host || !k_new_host || !v_new_host || !out_host) return CORM_ERR_INVALID_ARG;
+    if (!c->ready[layer]) return CORM_ERR_STATE;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->cfg.head_dim * c->e;
+    const size_t kb = (size_t)c->U * c->cfg.head_dim * c->e;
+    unsigned char *dq = c->arena + c->lay.stage_q, *dk = c->arena + c->lay.stage_k, *dv = c->arena + c->lay.stage_v,
+                  *dout = c->arena + c->lay.stage_out;
+    CORM_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st));
+    corm_status_t rc = launch_decode(c, layer, dq, dk, dv, dout, st);
+    if (rc != CORM_OK) return rc;
+    CORM_CUDA(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st));
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_live_lens(corm_cache_t* c, int32_t layer, int32_t* live_host, void* stream) {
+    if (!layer_ok(c, layer) || !live_host) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CORM_CUDA(cudaMemcpyAsync(live_host, live_buf(c, layer, c->parity[layer]), (size_t)c->U * 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* stream) {
+    if (!c || !out_host) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int L = c->cfg.n_layers;
+    std::vector<int32_t> live((size_t)L * 2 * c->U);
+    std::vector<unsigned long long> cnt((size_t)L * CNT_COUNT);
+    int32_t status = 0;
+    CORM_CUDA(cudaMemcpyAsync(live.data(), c->arena + c->lay.live, live.size() * 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaMemcpyAsync(cnt.data(), c->arena + c->lay.counters, cnt.size() * 8, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaMemcpyAsync(&status, c->arena + c->lay.status, 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    corm_stats_t s{};
+    for (int l = 0; l < L; ++l) {
+        const int32_t* lv = live.data() + ((size_t)l * 2 + c->parity[l]) * c->U;
+        for (int u = 0; u < c->U; ++u) s.live_keys += lv[u];
+        s.appended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_APPENDED];
+        s.evicted_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_EVICTED];
+        s.moved_rows += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_MOVED];
+        s.attended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_ATTENDED];
+    }
+    s.retention = s.appended_keys ? (double)s.live_keys / (double)s.appended_keys : 1.0;
+    s.kv_bytes_live = s.live_keys * 2 * c->cfg.head_dim * (int64_t)c->e;
+    s.aux_bytes_live = s.live_keys * 8;
+    s.device_status = status;
+    *out_host = s;
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_export_state(corm_cache_t* c, int32_t layer, int32_t seq, int32_t kv_head, void* k_host,
+                                      void* v_host, uint32_t* word_host, int32_t* pos_host, int32_t* live_len,
+                                      int32_t* n_tokens, int32_t* n_obs, void* stream) {
+    if (!layer_ok(c, layer) || seq < 0 || seq >= c->cfg.batch || kv_head < 0 || kv_head >= c->cfg.n_kv_heads)
+        return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const corm_config_t& cf = c->cfg;
+    const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U, u = (size_t)seq * cf.n_kv_heads + kv_head;
+    const size_t row_bytes = C * D * c->e;
+    int32_t bt = 0, bo = 0, lv = 0;
+    if (k_host) CORM_CUDA(cudaMemcpyAsync(k_host, layer_ptr(c, c->lay.K, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
+    if (v_host) CORM_CUDA(cudaMemcpyAsync(v_host, layer_ptr(c, c->lay.V, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
+    if (word_host) CORM_CUDA(cudaMemcpyAsync(word_host, layer_ptr(c, c->lay.word, U * C * 4, layer) + u * C * 4, C * 4, cudaMemcpyDeviceToHost, st));
+    if (pos_host) CORM_CUDA(cudaMemcpyAsync(pos_host, layer_ptr(c, c->lay.pos, U * C * 4, layer) + u * C * 4, C * 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaMemcpyAsync(&lv, live_buf(c, layer, c->parity[layer]) + u, 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaMemcpyAsync(&bt, layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer) + (size_t)seq * 4, 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaMemcpyAsync(&bo, layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer) + (size_t)seq * 4, 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    if (live_len) *live_len = lv;
+    if (n_tokens) *n_tokens = bt + c->steps[layer];
+    if (n_obs) *n_obs = std::min(cf.window_w, bo + c->steps[layer]);
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t seq, int32_t kv_head, const void* k_host,
+                                      const void* v_host, const uint32_t* word_host, const int32_t* pos_host,
+                                      int32_t live_len, int32_t n_tokens, int32_t n_obs, void* stream) {
+    if (!layer_ok(c, layer) || seq < 0 || seq >= c->cfg.batch || kv_head < 0 || kv_head >= c->cfg.n_kv_heads)
+        return CORM_ERR_INVALID_ARG;
+    const corm_config_t& cf = c->cfg;
+    if (live_len < 0 || n_tokens < 0 || n_obs < 0 || n_obs > cf.window_w) return CORM_ERR_INVALID_ARG;
+    if (live_len > cf.max_tokens) return CORM_ERR_CAPACITY;
+    if (live_len > 0 && (!k_host || !v_host || !word_host || !pos_host)) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(cf.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U, u = (size_t)seq * cf.n_kv_heads + kv_head;
+    const size_t row_bytes = C * D * c->e, n = (size_t)live_len;
+    if (n) {
+        CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.K, U * row_bytes, layer) + u * row_bytes, k_host, n * D * c->e, cudaMemcpyHostToDevice, st));
+        CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.V, U * row_bytes, layer) + u * row_bytes, v_host, n * D * c->e, cudaMemcpyHostToDevice, st));
+        CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.word, U * C * 4, layer) + u * C * 4, word_host, n * 4, cudaMemcpyHostToDevice, st));
+        CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.pos, U * C * 4, layer) + u * C * 4, pos_host, n * 4, cudaMemcpyHostToDevice, st));
+    }
+    // the kernels see tokens = base + steps and rows = min(w, base + steps): rebase this sequence
+    const int32_t bt = n_tokens - c->steps[layer], bo = n_obs - c->steps[layer], lv = live_len;
+    CORM_CUDA(cudaMemcpyAsync(live_buf(c, layer, c->parity[layer]) + u, &lv, 4, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer) + (size_t)seq * 4, &bt, 4, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer) + (size_t)seq * 4, &bo, 4, cudaMemcpyHostToDevice, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    c->ready[layer] = 1;
+    c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
+    if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
+    c->tune_split_len = split_len;
+    c->allow_fast = allow_fast_path ? 1 : 0;
+    return CORM_OK;
+}
+
+int64_t corm_cache_kernel_launches(const corm_cache_t* c) { return c ? c->launches : 0; }
+
+const char* corm_status_string(corm_status_t s) {
+    switch (s) {
+        case CORM_OK: return "ok";
+        case CORM_ERR_INVALID_ARG: return "invalid argument";
+        case CORM_ERR_UNSUPPORTED: return "unsupported configuration";
+        case CORM_ERR_ARENA_TOO_SMALL: return "arena too small";
+        case CORM_ERR_STATE: return "call out of order (no prompt pass for this layer)";
+        case CORM_ERR_CUDA: return "CUDA runtime error";
+        case CORM_ERR_CAPACITY: return "slab capacity exceeded";
+        case CORM_ERR_TIMEOUT: return "bounded wait expired";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

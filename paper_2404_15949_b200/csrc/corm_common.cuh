@@ -1,0 +1,261 @@
+// Shared device-side definitions of the CORM kernels: parameter blocks, element access, and the per-unit
+// "finalize" phase (split reduction, verdict, register update, keep decision, hole-filling compaction) that the
+// last-arriving thread block of a unit runs inside the decode kernel.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/corm.h"
+
+namespace corm {
+
+// Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
+enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_COUNT = 4 };
+
+struct DecodeParams {
+    void* K;                  // [U][C][D] this layer's key slabs
+    void* V;                  // [U][C][D]
+    uint32_t* word;           // [U][C] verdict registers
+    int32_t* pos;             // [U][C] absolute 1-based token positions
+    const int32_t* live_in;   // [U] live length before this step
+    int32_t* live_out;        // [U] live length after this step (the other half of a double buffer)
+    const int32_t* base_tokens;  // [B] tokens seen when the step counter was last rebased
+    const int32_t* base_obs;     // [B] verdict rows recorded at that time
+    uint32_t* ticket;         // [U] arrival counters of the splits of a unit (zero between steps)
+    unsigned long long* counters;  // [CNT_COUNT]
+    int32_t* status;          // sticky device status
+    double* stash;            // [U*G][C] scaled logits of this step (scratch)
+    unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
+    const void* q;            // [B][Hq][D]
+    const void* k_new;        // [B][Hkv][D]
+    const void* v_new;        // [B][Hkv][D]
+    void* out;                // [B][Hq][D]
+    int32_t U, Hkv, C, split_len, max_splits, step, w, r;
+    double log_alpha;         // ln(alpha), -inf for alpha = 0
+};
+
+struct PromptParams {
+    const void* k_prompt;     // [B][Hkv][p_max][D]
+    const void* v_prompt;
+    const void* q_last;       // [B][Hq][w][D]
+    const int32_t* prompt_lens;  // [B] device copy
+    void* K;
+    void* V;
+    uint32_t* word;
+    int32_t* pos;
+    int32_t* live_out;        // [U]
+    unsigned long long* counters;
+    int32_t* status;
+    double* stash;            // scratch, reused for temporary registers
+    int32_t U, Hkv, C, p_max, w, r;
+    double log_alpha;
+};
+
+__host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D; }
+
+// ---- element access: the cache dtype is only a storage format; all logits are formed in fp64 ----
+struct bf16_t { uint16_t bits; };
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) { return __uint_as_float(bits16 << 16); }
+
+// round-to-nearest-even float -> bf16 bits (finite inputs; NaN stays NaN)
+__device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
+    uint32_t x = __float_as_uint(f);
+    if ((x & 0x7f800000u) == 0x7f800000u) return (uint16_t)((x >> 16) | ((x & 0xffffu) ? 0x40u : 0u));
+    x += 0x7fffu + ((x >> 16) & 1u);
+    return (uint16_t)(x >> 16);
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kBytes = 4;
+    static __device__ __forceinline__ float load(const float* p) { return *p; }
+    static __device__ __forceinline__ void store(float* p, float v) { *p = v; }
+};
+template <> struct Elem<bf16_t> {
+    static constexpr int kBytes = 2;
+    static __device__ __forceinline__ float load(const bf16_t* p) { return bf16_bits_to_float(p->bits); }
+    static __device__ __forceinline__ void store(bf16_t* p, float v) { p->bits = float_to_bf16_bits(v); }
+};
+
+// N contiguous elements starting at p (p aligned to N*sizeof(T)), widened to float.
+template <typename T, int N> __device__ __forceinline__ void load_slice(const T* p, float (&out)[N]);
+template <> __device__ __forceinline__ void load_slice<float, 4>(const float* p, float (&out)[4]) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <> __device__ __forceinline__ void load_slice<float, 2>(const float* p, float (&out)[2]) {
+    float2 v = *reinterpret_cast<const float2*>(p);
+    out[0] = v.x; out[1] = v.y;
+}
+template <> __device__ __forceinline__ void load_slice<bf16_t, 4>(const bf16_t* p, float (&out)[4]) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    out[0] = __uint_as_float(v.x << 16); out[1] = __uint_as_float(v.x & 0xffff0000u);
+    out[2] = __uint_as_float(v.y << 16); out[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+template <> __device__ __forceinline__ void load_slice<bf16_t, 2>(const bf16_t* p, float (&out)[2]) {
+    uint32_t v = *reinterpret_cast<const uint32_t*>(p);
+    out[0] = __uint_as_float(v << 16); out[1] = __uint_as_float(v & 0xffff0000u);
+}
+
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ uint32_t window_mask(int w) { return w >= 32 ? 0xffffffffu : ((1u << w) - 1u); }
+
+// Exclusive prefix sums of popc(mask[i]) into prefix[0..nwords], block-wide. scratch holds NT ints.
+template <int NT>
+__device__ void block_popc_scan(const uint32_t* mask, int* prefix, int nwords, int* scratch) {
+    const int tid = threadIdx.x;
+    const int per = (nwords + NT - 1) / NT;
+    const int lo = min(tid * per, nwords), hi = min(lo + per, nwords);
+    int sum = 0;
+    for (int i = lo; i < hi; ++i) sum += __popc(mask[i]);
+    scratch[tid] = sum;
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int i = 0; i < NT; ++i) { int v = scratch[i]; scratch[i] = run; run += v; }
+        prefix[nwords] = run;
+    }
+    __syncthreads();
+    int run = scratch[tid];
+    for (int i = lo; i < hi; ++i) { prefix[i] = run; run += __popc(mask[i]); }
+    __syncthreads();
+}
+
+__device__ __forceinline__ int kept_before(const uint32_t* mask, const int* prefix, int j) {
+    return prefix[j >> 5] + __popc(mask[j >> 5] & ((1u << (j & 31)) - 1u));
+}
+
+// Copies one K row and one V row (D elements each) plus register and position from slot src to slot dst of a unit;
+// executed by one warp. Rows are D*sizeof(T) bytes = a multiple of 16.
+template <typename T, int D>
+__device__ __forceinline__ void warp_move_row(T* Ku, T* Vu, uint32_t* wordu, int32_t* posu, int src, int dst,
+                                              int lane) {
+    constexpr int kChunks = D * Elem<T>::kBytes / 16;
+    const uint4* ks = reinterpret_cast<const uint4*>(Ku + (size_t)src * D);
+    const uint4* vs = reinterpret_cast<const uint4*>(Vu + (size_t)src * D);
+    uint4* kd = reinterpret_cast<uint4*>(Ku + (size_t)dst * D);
+    uint4* vd = reinterpret_cast<uint4*>(Vu + (size_t)dst * D);
+    for (int c = lane; c < 2 * kChunks; c += 32) {
+        if (c < kChunks) kd[c] = __ldcg(ks + c);
+        else vd[c - kChunks] = __ldcg(vs + (c - kChunks));
+    }
+    if (lane == 0) {
+        wordu[dst] = __ldcg(wordu + src);
+        posu[dst] = __ldcg(posu + src);
+    }
+}
+
+// Finalize phase of one unit, run by the whole block that arrived last (every split of the unit has published its
+// partial record and its logits). Steps, in the order of Algorithm 1:
+//   1. reduce the split partials -> out (Eq. 1) and lse_g = ln sum_j exp(s_gj) per query head (Eq. 2's denominator)
+//   2. verdict of every live key: OR over the group of [s_gj >= lse_g + ln(alpha) - ln(t)]  (Definition 3.1 in log
+//      form; GQA rule), shifted into the key's register
+//   3. once w rows exist: keep iff register != 0 or position > t - r; holes below the new length are filled with
+//      kept rows from above it (as many row copies as there are holes; sources and destinations are disjoint)
+// smem: 2*(ceil(C/32)+2) 32-bit words of dynamic shared memory.
+template <typename T, int D, int G, int NT>
+__device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_act, int t, unsigned char* smem) {
+    __shared__ double s_thr[G];
+    __shared__ int s_scan[NT];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cap_words = (p.C + 31) / 32 + 2;
+    uint32_t* keepmask = reinterpret_cast<uint32_t*>(smem);
+    int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
+    T* Ku = reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D;
+    T* Vu = reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D;
+    uint32_t* wordu = p.word + (size_t)u * p.C;
+    int32_t* posu = p.pos + (size_t)u * p.C;
+    const size_t pstride = partial_stride(D);
+
+    // 1. split reduction
+    for (int g = 0; g < G; ++g) {
+        const unsigned char* rec0 = p.partials + ((size_t)u * p.max_splits * G + g) * pstride;
+        double m = -INFINITY;
+        for (int s = 0; s < n_act; ++s)
+            m = fmax(m, __ldcg(reinterpret_cast<const double*>(rec0 + (size_t)s * G * pstride)));
+        double Z = 0.0;
+        float acc[(D + NT - 1) / NT];
+#pragma unroll
+        for (int i = 0; i < (D + NT - 1) / NT; ++i) acc[i] = 0.f;
+        for (int s = 0; s < n_act; ++s) {
+            const unsigned char* rec = rec0 + (size_t)s * G * pstride;
+            const double ms = __ldcg(reinterpret_cast<const double*>(rec));
+            const double sc = exp(ms - m);
+            Z += __ldcg(reinterpret_cast<const double*>(rec) + 1) * sc;
+            const float scf = (float)sc;
+            const float* a = reinterpret_cast<const float*>(rec + 16);
+#pragma unroll
+            for (int i = 0; i < (D + NT - 1) / NT; ++i) {
+                const int c = tid + i * NT;
+                if (c < D) acc[i] += __ldcg(a + c) * scf;
+            }
+        }
+        T* outp = reinterpret_cast<T*>(p.out) + ((size_t)u * G + g) * D;
+#pragma unroll
+        for (int i = 0; i < (D + NT - 1) / NT; ++i) {
+            const int c = tid + i * NT;
+            if (c < D) Elem<T>::store(outp + c, (float)((double)acc[i] / Z));
+        }
+        if (tid == 0) s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);
+    }
+    __syncthreads();
+
+    // 2. verdicts, register update, keep flags
+    const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
+    const bool evict_on = n_obs >= p.w;
+    const uint32_t wmask = window_mask(p.w);
+    const double* stash_u = p.stash + (size_t)u * G * p.C;
+    for (int base = 0; base < l; base += NT) {
+        const int j = base + tid;
+        bool keep = false;
+        if (j < l) {
+            bool imp = false;
+#pragma unroll
+            for (int g = 0; g < G; ++g) imp |= (__ldcg(stash_u + (size_t)g * p.C + j) >= s_thr[g]);
+            const uint32_t wd = ((__ldcg(wordu + j) << 1) | (imp ? 1u : 0u)) & wmask;
+            wordu[j] = wd;
+            keep = !evict_on || wd != 0u || __ldcg(posu + j) > t - p.r;
+        }
+        const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
+    }
+    __syncthreads();
+    int new_len = l, n_moved = 0;
+    if (evict_on) {
+        const int nwords = (l + 31) / 32;
+        block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
+        new_len = prefix[nwords];
+        if (new_len < l) {
+            // 3. hole filling: the k-th kept row at or above new_len moves into the k-th hole below it
+            int* holes = reinterpret_cast<int*>(const_cast<double*>(stash_u));   // the logits are consumed
+            int* movers = holes + p.C;
+            const int kept_below = kept_before(keepmask, prefix, new_len);   // kept rows already below new_len
+            n_moved = new_len - kept_below;
+            for (int j = tid; j < l; j += NT) {
+                const int kb = kept_before(keepmask, prefix, j);
+                const bool kept = (keepmask[j >> 5] >> (j & 31)) & 1u;
+                if (j < new_len && !kept) holes[j - kb] = j;
+                if (j >= new_len && kept) movers[kb - kept_below] = j;
+            }
+            __syncthreads();
+            for (int i = warp; i < n_moved; i += NT / 32)
+                warp_move_row<T, D>(Ku, Vu, wordu, posu, movers[i], holes[i], lane);
+        }
+    }
+    if (tid == 0) {
+        p.live_out[u] = new_len;
+        atomicAdd(p.counters + CNT_APPENDED, 1ull);
+        atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+        if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+        if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
+    }
+}
+
+}  // namespace corm

@@ -1,0 +1,171 @@
+"""GPU parity: the CUDA library against the CPU oracle through the C ABI, same seeded inputs on both sides.
+
+Outputs must agree within max-abs 2e-3 (fp32 caches) / 2e-2 (bf16 caches); verdict registers, live-index lists and
+cached rows must be bit-exact. The oracle's count of probabilities within 1e-6 (relative) of the threshold is
+asserted to be zero on the fixed seeds, so no verdict is excused.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_15949_b200.workload import CONFIGS, generate
+from parity_util import (OUT_TOL, assert_states_equal, make_gpu_cache, make_oracle, run_free, sorted_state, to_dev)
+
+pytestmark = pytest.mark.gpu
+
+
+def _pair(cfg, data, **kw):
+    nb, nh = len(data.seqs), len(data.kv_heads)
+    return make_gpu_cache(cfg, nb, nh, **kw), make_oracle(cfg, nb, nh, **kw)
+
+
+@pytest.mark.parametrize("split_len", [0, 64, 128])
+def test_config1_tiny_f32_free_run(split_len):
+    cfg = CONFIGS[1]
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    gpu.corm_cache_set_tuning(split_len, True)
+    run_free(cfg, data, gpu, orc)
+    c = orc.counters()
+    assert c["near_threshold"] == 0 and c["evicted"] > 0
+    st = gpu.corm_cache_stats()
+    assert st["appended_keys"] == c["appended"] and st["evicted_keys"] == c["evicted"]
+    assert st["live_keys"] == int(orc.live_lens(0).sum())
+
+
+@pytest.mark.parametrize("seed", [15950, 15951])
+def test_config1_other_seeds(seed):
+    cfg = CONFIGS[1].with_(seed=seed)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    run_free(cfg, data, gpu, orc, check_every=8)
+    assert orc.counters()["near_threshold"] == 0
+
+
+SMALL = [
+    # dtype, head_dim, group, n_kv, batch, prompt range, steps, w, r, split_len, fast
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, True),
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, False),
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True),
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, False),
+    ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True),
+    ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 64, True),
+    ("bf16", 64, 4, 2, 2, (100, 200), 24, 8, 16, 64, True),
+    ("f32", 64, 1, 2, 2, (60, 130), 24, 5, 7, 64, True),
+    ("f32", 128, 8, 1, 1, (90, 90), 16, 16, 4, 0, True),
+    ("f32", 128, 2, 2, 3, (0, 40), 40, 8, 3, 64, True),      # prompts shorter than w, including empty ones
+]
+
+
+@pytest.mark.parametrize("case", SMALL, ids=lambda c: "-".join(str(x) for x in c))
+def test_small_shapes(case):
+    dtype, d, G, nkv, B, (pmin, pmax), steps, w, r, split_len, fast = case
+    cfg = CONFIGS[1].with_(name="small", batch=B, n_q_heads=nkv * G, n_kv_heads=nkv, head_dim=d, dtype=dtype,
+                           prompt_min=pmin, prompt_max=pmax, steps=steps, window_w=w, recent_r=r,
+                           gqa_rho=0.7 if G > 1 else 0.0, hh_min=2, hh_max=6, seed=777)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    gpu.corm_cache_set_tuning(split_len, fast)
+    run_free(cfg, data, gpu, orc)
+    assert orc.counters()["near_threshold"] == 0
+
+
+def test_alpha_zero_never_evicts():
+    cfg = CONFIGS[1].with_(prompt_min=100, prompt_max=100, steps=20, alpha=0.0, dtype="bf16")
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    run_free(cfg, data, gpu, orc)
+    assert (gpu.corm_cache_live_lens(0) == 120).all()
+    assert gpu.corm_cache_stats()["evicted_keys"] == 0
+
+
+def test_lockstep_from_imported_state():
+    """Both sides start every step from the oracle's state (import hook), as the large configurations do."""
+    cfg = CONFIGS[1].with_(prompt_min=200, prompt_max=200, steps=24, dtype="bf16", n_q_heads=8, n_kv_heads=2,
+                           gqa_rho=0.7)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    orc.compress_prompt(0, data.k_prompt, data.v_prompt, data.q_last, data.prompt_lens)
+    dt = cfg.dtype
+    for s in range(cfg.steps):
+        for h in range(2):
+            st = orc.export_unit(0, 0, h)
+            perm = np.random.default_rng(s * 7 + h).permutation(st["live_len"])      # slot order is free
+            gpu.corm_cache_import_state(0, 0, h, st["k"][perm], st["v"][perm], st["word"][perm], st["pos"][perm],
+                                        st["n_tokens"], st["n_obs"])
+        out_g = gpu.corm_decode_step(0, to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt))
+        out_o = orc.decode_step(0, data.q[s], data.k_new[s], data.v_new[s])
+        assert np.abs(out_g.float().cpu().numpy() - out_o).max() <= OUT_TOL[dt]
+        assert_states_equal(gpu, orc, 0, 1, 2, f"step {s}")
+
+
+def test_multi_layer_independent_and_deterministic():
+    cfg = CONFIGS[2].with_(n_layers=3, n_q_heads=4, n_kv_heads=4, prompt_min=300, prompt_max=300, steps=12,
+                           recent_r=32, dense_layers=1)
+    gpu = make_gpu_cache(cfg, 1, 4, n_layers=3)
+    gpu2 = make_gpu_cache(cfg, 1, 4, n_layers=3)
+    orc = make_oracle(cfg, 1, 4, n_layers=3)
+    datas = [generate(cfg, layer=l) for l in range(3)]
+    dt = cfg.dtype
+    for l in (2, 0, 1):                                              # layers in any order
+        d = datas[l]
+        for g in (gpu, gpu2):
+            g.corm_compress_prompt(l, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+        orc.compress_prompt(l, d.k_prompt, d.v_prompt, d.q_last, d.prompt_lens)
+    for s in range(cfg.steps):
+        for l in (1, 2, 0):
+            d = datas[l]
+            a = gpu.corm_decode_step(l, to_dev(d.q[s], dt), to_dev(d.k_new[s], dt), to_dev(d.v_new[s], dt))
+            b = gpu2.corm_decode_step(l, to_dev(d.q[s], dt), to_dev(d.k_new[s], dt), to_dev(d.v_new[s], dt))
+            o = orc.decode_step(l, d.q[s], d.k_new[s], d.v_new[s])
+            assert torch.equal(a, b)                                  # same inputs twice -> identical bits
+            assert np.abs(a.float().cpu().numpy() - o).max() <= OUT_TOL[dt]
+    for l in range(3):
+        assert_states_equal(gpu, orc, l, 1, 4, f"layer {l}")
+        for h in range(4):
+            sa = sorted_state(gpu.corm_cache_export_state(l, 0, h))
+            sb = sorted_state(gpu2.corm_cache_export_state(l, 0, h))
+            assert all(np.array_equal(sa[k], sb[k]) for k in ("k", "v", "word", "pos"))
+    assert gpu.corm_cache_kernel_launches() == 3 + 3 * cfg.steps
+
+
+def test_host_buffer_entry_point_matches_device_one():
+    cfg = CONFIGS[1].with_(prompt_min=130, prompt_max=130, steps=10, dtype="bf16")
+    data = generate(cfg)
+    a, b = make_gpu_cache(cfg, 1, 8), make_gpu_cache(cfg, 1, 8)
+    dt = cfg.dtype
+    for g in (a, b):
+        g.corm_compress_prompt(0, to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt),
+                               data.prompt_lens)
+    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).pin_memory()
+    for s in range(cfg.steps):
+        ref = a.corm_decode_step(0, to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt))
+        out = torch.empty(ref.shape, dtype=torch.bfloat16).pin_memory()
+        b.corm_decode_step_host(0, pin(data.q[s]), pin(data.k_new[s]), pin(data.v_new[s]), out)
+        torch.cuda.synchronize()
+        assert torch.equal(ref.cpu(), out)
+
+
+def test_capacity_overflow_is_reported_not_fatal():
+    cfg = CONFIGS[1].with_(prompt_min=40, prompt_max=40, steps=8, alpha=0.0, n_q_heads=2, n_kv_heads=2)
+    data = generate(cfg)
+    gpu = make_gpu_cache(cfg, 1, 2, max_tokens=44)
+    dt = cfg.dtype
+    gpu.corm_compress_prompt(0, to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt),
+                             data.prompt_lens)
+    for s in range(6):
+        gpu.corm_decode_step(0, to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt))
+    st = gpu.corm_cache_stats()
+    assert st["device_status"] == 6 and (gpu.corm_cache_live_lens(0) == 44).all()
+
+
+def test_state_errors_on_gpu():
+    from paper_2404_15949_b200.binding import CormError
+    cfg = CONFIGS[1].with_(n_q_heads=2, n_kv_heads=2)
+    gpu = make_gpu_cache(cfg, 1, 2)
+    x = torch.zeros(1, 2, 128, device="cuda")
+    with pytest.raises(CormError) as e:
+        gpu.corm_decode_step(0, x, x, x)                             # no prompt pass yet
+    assert e.value.status == 4
+    with pytest.raises(CormError):
+        gpu.corm_decode_step(1, x, x, x)                             # layer out of range

@@ -1,0 +1,73 @@
+"""CPU-side checks of the C-ABI library: it loads without a GPU, exports every symbol the header declares, sizes its
+arena as documented and rejects bad arguments before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2404_15949_b200 import binding
+from paper_2404_15949_b200.build import build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_library()
+    return binding.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "corm.h")).read()
+    names = set(re.findall(r"\b(corm_[a-z_]+)\s*\(", header))
+    assert {"corm_cache_create", "corm_compress_prompt", "corm_decode_step", "corm_cache_stats"} <= names
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} is declared in corm.h but not exported"
+
+
+def _cfg(**kw):
+    base = dict(n_layers=1, batch=2, n_q_heads=8, n_kv_heads=2, head_dim=128, max_tokens=512, window_w=8, recent_r=32,
+                alpha=1.0, kv_dtype=binding.CORM_BF16, device=0)
+    base.update(kw)
+    return binding.CormConfig(*[base[k] for k, _ in binding.CormConfig._fields_])
+
+
+def test_arena_bytes_and_the_256_gb_example(lib):
+    # The introduction's example: a 7B model (32 layers x 32 heads x 128), batch 128, sequence 4096, 16-bit cache
+    # needs 256 GB for K and V: 2 * 32*32*128 * 2 B = 0.5 MiB per token, times 4096 * 128 tokens = 256 GiB.
+    kv = 2 * 32 * 32 * 128 * 2 * 4096 * 128
+    assert kv == 256 * 2 ** 30
+    total = binding.corm_cache_arena_bytes(_cfg(n_layers=32, batch=128, n_q_heads=32, n_kv_heads=32, max_tokens=4096))
+    assert kv < total < kv * 1.03                                      # registers, positions and scratch: < 3 %
+    assert binding.corm_cache_arena_bytes(_cfg(kv_dtype=binding.CORM_F32)) > binding.corm_cache_arena_bytes(_cfg())
+
+
+@pytest.mark.parametrize("bad", [dict(n_q_heads=7), dict(recent_r=0), dict(window_w=0), dict(alpha=-1.0),
+                                 dict(kv_dtype=5), dict(batch=0)])
+def test_invalid_configs_have_no_arena(lib, bad):
+    assert binding.corm_cache_arena_bytes(_cfg(**bad)) == 0
+
+
+def test_create_rejects_before_any_cuda_call(lib):
+    handle = ctypes.c_void_p()
+    fake = ctypes.c_void_p(0x10000)                                    # aligned, never dereferenced on these paths
+    cfg = _cfg()
+    need = binding.corm_cache_arena_bytes(cfg)
+    assert lib.corm_cache_create(ctypes.byref(cfg), fake, need - 1, ctypes.byref(handle)) == 3
+    assert lib.corm_cache_create(ctypes.byref(cfg), None, need, ctypes.byref(handle)) == 1
+    assert lib.corm_cache_create(ctypes.byref(cfg), ctypes.c_void_p(0x10001), need, ctypes.byref(handle)) == 1
+    for bad, code in [(dict(head_dim=96), 2), (dict(window_w=33), 2), (dict(n_q_heads=6, n_kv_heads=2), 2),
+                      (dict(n_q_heads=7), 1)]:
+        c = _cfg(**bad)
+        assert lib.corm_cache_create(ctypes.byref(c), fake, 1 << 40, ctypes.byref(handle)) == code
+    assert handle.value is None
+    assert lib.corm_status_string(6) == b"slab capacity exceeded"
+    assert lib.corm_cache_destroy(None) == 1 and lib.corm_cache_kernel_launches(None) == 0
+
+
+def test_binding_fails_loudly_without_library(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libcorm.so")
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        binding.load_library()
