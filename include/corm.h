@@ -110,6 +110,30 @@ corm_status_t corm_decode_step(corm_cache_t* cache, int32_t layer, const void* q
 corm_status_t corm_decode_step_host(corm_cache_t* cache, int32_t layer, const void* q_host, const void* k_new_host,
                                     const void* v_new_host, void* out_host, void* stream);
 
+/* corm_decode_step for callers that cannot allocate device memory. (The paper has no counterpart: this is a
+ * packaging variant of the same step, not a different method.)
+ * Who needs it: code that receives a fixed set of buffers and may not call cudaMalloc or a framework allocator
+ * where the step runs, for example a plugin inside a serving runtime whose memory plan was frozen at start-up, or
+ * an embedder that gave the cache only room for K, V, registers and positions. corm_decode_step keeps its per-step
+ * scratch (this step's logits, the split partial records, the per-unit arrival counters) in the caller's arena;
+ * this variant keeps it in a 16 MiB array built into the library, which every GPU that loads the library holds
+ * until the process exits. The caller still passes the cache and q / k_new / v_new / out exactly as for
+ * corm_decode_step, results are the same, and the two calls may be mixed freely on one cache.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   Limit: align256(batch*n_q_heads*max_tokens*8) + align256(batch*n_kv_heads*ceil(live_bound/256)*group*
+ *   (16 + 4*head_dim)) + align256(batch*n_kv_heads*4) bytes must fit in 16 MiB (live_bound = the longest prompt so
+ *   far + decode steps so far + 1, capped at max_tokens); otherwise CORM_ERR_CAPACITY is returned, a message
+ *   naming both sizes goes to stderr and nothing is enqueued.
+ *   First call on a device: looks up the array's device address (once per device, that device made current for
+ *   the lookup). Make this first call outside any stream capture.
+ *   Sharing: all caches and all calls on a device use the same array. It keeps the previous call's contents; the
+ *   arrival counters are cleared on `stream` at the start of every call, everything else is rewritten before it
+ *   is read. Two calls of this function that overlap on the GPU (different streams, no ordering) race on the
+ *   array and give wrong results: keep them stream-ordered.
+ * Errors otherwise as corm_decode_step. */
+corm_status_t corm_decode_step_static(corm_cache_t* cache, int32_t layer, const void* q, const void* k_new,
+                                      const void* v_new, void* out, void* stream);
+
 /* Totals over all units ("compression rate" of Section 5). Synchronises `stream`. */
 corm_status_t corm_cache_stats(corm_cache_t* cache, corm_stats_t* out_host, void* stream);
 

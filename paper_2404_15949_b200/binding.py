@@ -64,6 +64,8 @@ def load_library():
     lib.corm_compress_prompt.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp]
     lib.corm_decode_step.restype = i32
     lib.corm_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.corm_decode_step_static.restype = i32
+    lib.corm_decode_step_static.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.corm_decode_step_host.restype = i32
     lib.corm_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.corm_cache_stats.restype = i32
@@ -158,6 +160,16 @@ class CormCache:
             out = torch.empty_like(q)
         _check("corm_decode_step", self.lib.corm_decode_step(self.handle, layer, q.data_ptr(), k_new.data_ptr(),
                                                              v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)))
+        return out
+
+    def corm_decode_step_static(self, layer, q, k_new, v_new, out=None, stream=None):
+        """corm_decode_step for callers that must not allocate: the step's scratch sits in an array built into the
+        library (16 MiB, shared by every cache on the device) instead of the arena. Pass ``out`` to keep this
+        wrapper allocation-free as well; calls that overlap on the GPU race on the shared array."""
+        if out is None:
+            out = torch.empty_like(q)
+        _check("corm_decode_step_static", self.lib.corm_decode_step_static(
+            self.handle, layer, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)))
         return out
 
     def corm_decode_step_host(self, layer, q, k_new, v_new, out, stream=None):

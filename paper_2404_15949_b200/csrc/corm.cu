@@ -339,6 +339,96 @@ corm_status_t corm_decode_step_host(corm_cache_t* c, int32_t layer, const void* 
     return CORM_OK;
 }
 
+// ---- decode step for callers that cannot allocate device memory ------------------------------------------------
+// The scratch of the decode kernel (this step's logits, the split partial records and the per-unit arrival
+// counters) lives in one file-scope device array instead of caller memory. Every GPU that loads this library
+// holds the array until the process exits.
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+
+// The array's name is only a handle on the host; its device address must be asked for, once per device, with that
+// device current. The caller holds a DeviceGuard for `device`.
+corm_status_t static_scratch_address(int device, unsigned char** out) {
+    if (device < 0 || device >= kMaxDevices) return CORM_ERR_UNSUPPORTED;
+    if (!g_static_scratch_ptr[device]) {
+        void* ptr = nullptr;
+        CORM_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_scratch_ptr[device] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_scratch_ptr[device];
+    return CORM_OK;
+}
+}  // namespace
+
+corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void* q, const void* k_new,
+                                      const void* v_new, void* out, void* stream) {
+    if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return CORM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+         reinterpret_cast<uintptr_t>(out)) % 16) return CORM_ERR_INVALID_ARG;
+    if (!c->ready[layer]) return CORM_ERR_STATE;
+    const corm_config_t& cf = c->cfg;
+    const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U, G = c->G;
+    const int split_len = 256;
+    const int upper = std::min(cf.max_tokens, c->live_upper[layer] + 1);
+    const int n_splits = (upper + split_len - 1) / split_len;
+    const size_t stash_bytes = align_up(U * G * C * 8);
+    const size_t partial_bytes = align_up(U * (size_t)n_splits * G * partial_stride((int)D));
+    const size_t ticket_bytes = align_up(U * 4);
+    if (stash_bytes + partial_bytes + ticket_bytes > kStaticScratchBytes) {
+        std::fprintf(stderr, "corm_decode_step_static: this cache needs %zu bytes of scratch per step, the built-in "
+                             "scratch holds %zu; use corm_decode_step with an arena instead\n",
+                     stash_bytes + partial_bytes + ticket_bytes, kStaticScratchBytes);
+        return CORM_ERR_CAPACITY;
+    }
+    DeviceGuard guard(cf.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    corm_status_t rc = static_scratch_address(cf.device, &scratch);
+    if (rc != CORM_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DecodeParams p{};
+    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
+    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
+    p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
+    p.live_in = live_buf(c, layer, c->parity[layer]);
+    p.live_out = live_buf(c, layer, c->parity[layer] ^ 1);
+    p.base_tokens = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer));
+    p.base_obs = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer));
+    p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
+    p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
+    p.stash = reinterpret_cast<double*>(scratch);
+    p.partials = scratch + stash_bytes;
+    p.ticket = reinterpret_cast<uint32_t*>(scratch + stash_bytes + partial_bytes);
+    p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
+    p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = n_splits; p.split_len = split_len;
+    p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
+    p.log_alpha = log_alpha_of(c);
+    // the array keeps whatever the previous call (of any cache) left: the arrival counters must start at zero;
+    // logits and partial records are fully rewritten before they are read
+    CORM_CUDA(cudaMemsetAsync(p.ticket, 0, U * 4, st));
+    rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
+        using T = std::remove_pointer_t<decltype(tp)>;
+        constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
+        const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
+        auto kern = decode_generic_kernel<T, DD, GG>;
+        if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
+        CORM_CUDA(cudaGetLastError());
+        return CORM_OK;
+    });
+    if (rc != CORM_OK) return rc;
+    c->launches += 1;
+    c->parity[layer] ^= 1;
+    c->steps[layer] += 1;
+    c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
+    return CORM_OK;
+}
+
 corm_status_t corm_cache_live_lens(corm_cache_t* c, int32_t layer, int32_t* live_host, void* stream) {
     if (!layer_ok(c, layer) || !live_host) return CORM_ERR_INVALID_ARG;
     DeviceGuard guard(c->cfg.device);
