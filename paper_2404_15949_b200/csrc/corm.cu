@@ -166,7 +166,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.log_alpha = log_alpha_of(c);
     const int upper = std::min(cf.max_tokens, c->live_upper[layer] + 1);   // no unit can hold more live keys
 
-    const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128;
+    const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
     if (fast) {
         rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st);

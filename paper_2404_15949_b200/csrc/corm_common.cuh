@@ -32,6 +32,7 @@ struct DecodeParams {
     const void* v_new;        // [B][Hkv][D]
     void* out;                // [B][Hq][D]
     int32_t U, Hkv, C, split_len, max_splits, step, w, r;
+    int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
     double log_alpha;         // ln(alpha), -inf for alpha = 0
 };
 

@@ -1,7 +1,490 @@
-// placeholder until the bf16 / head_dim 128 kernel lands
+// Decode kernel for bf16 caches with head_dim 128 (group size 1, 2 or 4): the bandwidth path.
+//
+// One thread block per (unit, split of its live range); every warp streams 32-key tiles of K and V through its own
+// ring of shared-memory stages filled by bulk asynchronous copies (the TMA engine; a tile is one contiguous run of
+// 256-byte rows in the slab) that complete on mbarriers, so warps never synchronise with each other in the main
+// loop. Logits are formed in fp64: bf16 inputs widen exactly, a lane owns 8 channels of a key and 16 lanes share a
+// key; the 16 partial sums of 16 keys are folded with a transposing butterfly (15 exchanges for 16 keys, no
+// selects: each lane loads its keys in an order permuted by its lane bits so that every exchange step sends and
+// keeps fixed registers). After the fold each lane owns one key of the tile for softmax, verdict logit and
+// probability. P.V accumulates in fp32. A unit that fits one split keeps its logits, registers and positions in
+// shared memory and finishes entirely inside the block; longer units publish split partials and logits to global
+// scratch and the last-arriving block runs the shared finalize phase.
 #pragma once
+
 #include "corm_common.cuh"
+
 namespace corm {
-inline bool fast_path_available() { return false; }
-inline corm_status_t launch_decode_fast(DecodeParams&, int, int, int, int, cudaStream_t) { return CORM_ERR_UNSUPPORTED; }
+
+constexpr int kFastWarps = 4;
+constexpr int kFastThreads = kFastWarps * 32;
+constexpr int kTileKeys = 32;
+constexpr int kRowBytes = 256;                    // 128 bf16
+constexpr int kTileBytes = kTileKeys * kRowBytes; // 8 KiB
+constexpr int kKStages = 2, kVStages = 1;
+constexpr int kStagesPerWarp = kKStages + kVStages;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits (about 2 s)
+
+inline bool fast_path_available() { return true; }
+
+// ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
+struct FastSmem {
+    int tiles, qs, psm, stash, word, pos, bars, total;
+};
+__host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
+    FastSmem s;
+    int off = 0;
+    auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
+    s.tiles = take(kFastWarps * kStagesPerWarp * kTileBytes);   // later reused: merge area, finalize lists
+    s.qs = take(G * 128 * 8);
+    s.psm = take(kFastWarps * kTileKeys * G * 4);
+    s.stash = take(single_cap * G * 8);
+    s.word = take(single_cap * 4);
+    s.pos = take(single_cap * 4);
+    s.bars = take(kFastWarps * kStagesPerWarp * 8);
+    s.total = off;
+    return s;
 }
+
+// ---- PTX wrappers ----
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Waits for the phase with the given parity; gives up after kWaitLimitCycles and reports false.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long start = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - start > kWaitLimitCycles) return false;
+    return true;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src_gmem, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src_gmem), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+// exp(x) for x <= ~0 (small positive arguments are fine), 0 below the normal range. Argument reduction by ln 2 in
+// two pieces, degree-11 Taylor polynomial on |r| <= ln2/2 (truncation ~6e-15 relative), scaling through the exponent.
+__device__ __forceinline__ double exp_nonpos(double x) {
+    if (!(x > -708.0)) return 0.0;
+    const double t = fma(x, 1.4426950408889634074, 6755399441055744.0);   // round(x / ln 2) in the low word
+    const int n = __double2loint(t);
+    const double nf = t - 6755399441055744.0;
+    double r = fma(nf, -6.93147180369123816490e-01, x);
+    r = fma(nf, -1.90821492927058770002e-10, r);
+    double p = 2.505210838544172e-08;            // 1/11!
+    p = fma(p, r, 2.755731922398589e-07);        // 1/10!
+    p = fma(p, r, 2.755731922398589e-06);        // 1/9!
+    p = fma(p, r, 2.48015873015873e-05);         // 1/8!
+    p = fma(p, r, 1.984126984126984e-04);        // 1/7!
+    p = fma(p, r, 1.388888888888889e-03);        // 1/6!
+    p = fma(p, r, 8.333333333333333e-03);        // 1/5!
+    p = fma(p, r, 4.166666666666666e-02);        // 1/4!
+    p = fma(p, r, 1.666666666666667e-01);        // 1/3!
+    p = fma(p, r, 0.5);
+    p = fma(p, r, 1.0);
+    p = fma(p, r, 1.0);
+    return p * __hiloint2double((1023 + n) << 20, 0);
+}
+
+__device__ __forceinline__ void unpack8_to_double(const uint4& raw, double (&kd)[8]) {
+    kd[0] = (double)__uint_as_float(raw.x << 16); kd[1] = (double)__uint_as_float(raw.x & 0xffff0000u);
+    kd[2] = (double)__uint_as_float(raw.y << 16); kd[3] = (double)__uint_as_float(raw.y & 0xffff0000u);
+    kd[4] = (double)__uint_as_float(raw.z << 16); kd[5] = (double)__uint_as_float(raw.z & 0xffff0000u);
+    kd[6] = (double)__uint_as_float(raw.w << 16); kd[7] = (double)__uint_as_float(raw.w & 0xffff0000u);
+}
+__device__ __forceinline__ void unpack8_to_float(const uint4& raw, float (&v)[8]) {
+    v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xffff0000u);
+    v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xffff0000u);
+    v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xffff0000u);
+    v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xffff0000u);
+}
+
+// Unscaled q.k sums of one 32-key tile. Lane (h = lane>>4, i = lane&15) reads channel chunk i of the keys of half h;
+// on return the lane holds, per query head, the full sum of tile key  16h + 8(i&1) + (i>>1).
+// Pass it in {0,1} and register slot s in 0..7 load key 16h + 8(it ^ (i&1)) + (s ^ (i>>1)): with that order every
+// butterfly step keeps the low slots and sends the high ones, whatever the lane.
+template <int G>
+__device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double (&qd)[G][8], int lane,
+                                        double (&sown)[G]) {
+    const int h = lane >> 4, i = lane & 15, m = i >> 1, b0 = i & 1;
+    double r[2][G];
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        double a[G][8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const int key = 16 * h + 8 * (it ^ b0) + (s ^ m);
+            const uint4 raw = *reinterpret_cast<const uint4*>(ktile + key * kRowBytes + i * 16);
+            double kd[8];
+            unpack8_to_double(raw, kd);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                double acc = qd[g][0] * kd[0];
+#pragma unroll
+                for (int e = 1; e < 8; ++e) acc = fma(qd[g][e], kd[e], acc);
+                a[g][s] = acc;
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 4], 8);
+#pragma unroll
+            for (int s = 0; s < 2; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 2], 4);
+            a[g][0] += __shfl_xor_sync(0xffffffffu, a[g][1], 2);
+            r[it][g] = a[g][0];
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
+}
+
+// Single-split finalize: logits, registers and positions of the whole unit are in shared memory.
+// lists: scratch for the keep mask, its prefix sums and the hole / mover lists (ints).
+template <int G, int NT>
+__device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int t, const double* thr,
+                                const double* stash_sm, int stash_ld, uint32_t* word_sm, const int32_t* pos_sm,
+                                unsigned char* lists) {
+    __shared__ int s_scan1[NT];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cap_words = (l + 31) / 32 + 2;
+    uint32_t* keepmask = reinterpret_cast<uint32_t*>(lists);
+    int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
+    int* holes = prefix + cap_words;
+    int* movers = holes + l;
+    bf16_t* Ku = reinterpret_cast<bf16_t*>(p.K) + (size_t)u * p.C * 128;
+    bf16_t* Vu = reinterpret_cast<bf16_t*>(p.V) + (size_t)u * p.C * 128;
+    uint32_t* wordu = p.word + (size_t)u * p.C;
+    int32_t* posu = p.pos + (size_t)u * p.C;
+    const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
+    const bool evict_on = n_obs >= p.w;
+    const uint32_t wmask = window_mask(p.w);
+    for (int base = 0; base < l; base += NT) {
+        const int j = base + tid;
+        bool keep = false;
+        if (j < l) {
+            bool imp = false;
+#pragma unroll
+            for (int g = 0; g < G; ++g) imp |= (stash_sm[g * stash_ld + j] >= thr[g]);
+            const uint32_t wd = ((word_sm[j] << 1) | (imp ? 1u : 0u)) & wmask;
+            wordu[j] = wd;
+            keep = !evict_on || wd != 0u || pos_sm[j] > t - p.r;
+        }
+        const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
+    }
+    __syncthreads();
+    int new_len = l, n_moved = 0;
+    if (evict_on) {
+        const int nwords = (l + 31) / 32;
+        block_popc_scan<NT>(keepmask, prefix, nwords, s_scan1);
+        new_len = prefix[nwords];
+        if (new_len < l) {
+            const int kept_below = kept_before(keepmask, prefix, new_len);
+            n_moved = new_len - kept_below;
+            for (int j = tid; j < l; j += NT) {
+                const int kb = kept_before(keepmask, prefix, j);
+                const bool kept = (keepmask[j >> 5] >> (j & 31)) & 1u;
+                if (j < new_len && !kept) holes[j - kb] = j;
+                if (j >= new_len && kept) movers[kb - kept_below] = j;
+            }
+            __syncthreads();
+            for (int i = warp; i < n_moved; i += NT / 32)
+                warp_move_row<bf16_t, 128>(Ku, Vu, wordu, posu, movers[i], holes[i], lane);
+        }
+    }
+    if (tid == 0) {
+        p.live_out[u] = new_len;
+        atomicAdd(p.counters + CNT_APPENDED, 1ull);
+        atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+        if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+        if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
+    }
+}
+
+template <int G>
+__global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int s_last;
+    __shared__ int s_failed;
+    __shared__ double s_thr1[G];
+    constexpr int NT = kFastThreads, NW = kFastWarps;
+    const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = u / p.Hkv;
+    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    if (l > p.C) {
+        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; }
+        return;
+    }
+    const int n_act = (l + p.split_len - 1) / p.split_len;
+    if (split >= n_act) return;
+    const bool single = (n_act == 1 && l <= p.single_cap);
+    const int t = __ldg(p.base_tokens + b) + p.step + 1;
+    const int begin = split * p.split_len, end = min(l, begin + p.split_len);
+    const int n_tiles = (end - begin + kTileKeys - 1) / kTileKeys;
+    const FastSmem lay = fast_smem_layout(G, p.single_cap);
+    unsigned char* my_tiles = smem + lay.tiles + warp * kStagesPerWarp * kTileBytes;
+    const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kStagesPerWarp * 8;
+    double* qs = reinterpret_cast<double*>(smem + lay.qs);
+    float* psm = reinterpret_cast<float*>(smem + lay.psm) + warp * kTileKeys * G;
+    double* stash_sm = reinterpret_cast<double*>(smem + lay.stash);
+    uint32_t* word_sm = reinterpret_cast<uint32_t*>(smem + lay.word);
+    int32_t* pos_sm = reinterpret_cast<int32_t*>(smem + lay.pos);
+    const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.K) + (size_t)u * p.C * kRowBytes;
+    const unsigned char* Vu = reinterpret_cast<const unsigned char*>(p.V) + (size_t)u * p.C * kRowBytes;
+    uint32_t* wordu = p.word + (size_t)u * p.C;
+    int32_t* posu = p.pos + (size_t)u * p.C;
+
+    if (tid == 0) s_failed = 0;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kStagesPerWarp; ++s) mbar_init(my_bars + s * 8, 1);
+        fence_mbar_init();
+        fence_async_smem();
+    }
+    __syncthreads();
+
+    // this warp's tiles: warp, warp + NW, ... (tile index inside the split)
+    const int my_n = (n_tiles > warp) ? (n_tiles - warp + NW - 1) / NW : 0;
+    auto tile_keys = [&](int it) { return min(kTileKeys, end - (begin + (warp + it * NW) * kTileKeys)); };
+    auto issue_k = [&](int it) {
+        const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kKStages;
+        const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
+        mbar_expect_tx(my_bars + slot * 8, bytes);
+        bulk_load(smem_addr(my_tiles + slot * kTileBytes), Ku + (size_t)k0 * kRowBytes, bytes, my_bars + slot * 8);
+    };
+    auto issue_v = [&](int it) {
+        const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kVStages;
+        const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
+        mbar_expect_tx(my_bars + (kKStages + slot) * 8, bytes);
+        bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vu + (size_t)k0 * kRowBytes, bytes,
+                  my_bars + (kKStages + slot) * 8);
+    };
+    if (lane == 0) {
+        for (int it = 0; it < min(my_n, kKStages); ++it) issue_k(it);
+        for (int it = 0; it < min(my_n, kVStages); ++it) issue_v(it);
+    }
+
+    // queries widened to fp64 once per block; registers and positions of a single-split unit staged on chip
+    {
+        const bf16_t* qg = reinterpret_cast<const bf16_t*>(p.q) + (size_t)u * G * 128;
+        for (int x = tid; x < G * 128; x += NT) qs[x] = (double)Elem<bf16_t>::load(qg + x);
+        if (single) {
+            for (int j = tid; j < l_old; j += NT) { word_sm[j] = __ldcg(wordu + j); pos_sm[j] = __ldcg(posu + j); }
+            if (tid == 0) { word_sm[l_old] = 0u; pos_sm[l_old] = t; }
+        }
+    }
+    __syncthreads();
+
+    const int h = lane >> 4, ci = lane & 15;
+    const int key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);     // tile key this lane owns after the fold
+    double qd[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) qd[g][e] = qs[g * 128 + ci * 8 + e];
+    double M[G], Zl[G];
+    float acc[G][8];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        M[g] = -INFINITY; Zl[g] = 0.0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
+    }
+    const double inv_root_d = 0.088388347648318440550;          // 1/sqrt(128)
+    bool failed = false;
+
+    for (int it = 0; it < my_n; ++it) {
+        const int k0 = begin + (warp + it * NW) * kTileKeys;
+        const int n_valid = min(kTileKeys, end - k0);
+        const bool has_new = (l_old >= k0 && l_old < k0 + kTileKeys);   // this tile holds the appended token
+        const int kslot = it % kKStages, vslot = it % kVStages;
+        unsigned char* ktile = my_tiles + kslot * kTileBytes;
+        unsigned char* vtile = my_tiles + (kKStages + vslot) * kTileBytes;
+        if (!mbar_wait(my_bars + kslot * 8, (it / kKStages) & 1)) failed = true;
+        if (has_new) {   // append: the new row goes to the slab and replaces whatever the copy fetched for that slot
+            const uint4* kn = reinterpret_cast<const uint4*>(p.k_new) + (size_t)u * 16;
+            if (lane < 16) {
+                const uint4 x = kn[lane];
+                *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = x;
+                reinterpret_cast<uint4*>(const_cast<unsigned char*>(Ku) + (size_t)l_old * kRowBytes)[lane] = x;
+            }
+            if (lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
+            __syncwarp();
+        }
+        double sown[G];
+        qk_tile<G>(ktile, qd, lane, sown);
+        __syncwarp();
+        if (lane == 0 && it + kKStages < my_n) { fence_async_smem(); issue_k(it + kKStages); }
+
+        const bool valid = key_own < n_valid;
+        const int j_own = k0 + key_own;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            const double s = valid ? sown[g] * inv_root_d : -INFINITY;     // Eq. 2's exponent
+            if (valid) {
+                if (single) stash_sm[g * p.single_cap + j_own] = s;
+                else p.stash[((size_t)u * G + g) * p.C + j_own] = s;
+            }
+            float mt = (float)s;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, o));
+            const double mtd = (double)mt;
+            if (mtd > M[g]) {                                              // warp-uniform
+                const double sc = exp_nonpos(M[g] - mtd);
+                const float scf = (float)sc;
+                Zl[g] *= sc;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] *= scf;
+                M[g] = mtd;
+            }
+            const double ex = valid ? exp_nonpos(s - M[g]) : 0.0;
+            Zl[g] += ex;
+            psm[key_own * G + g] = (float)ex;
+        }
+        __syncwarp();
+
+        if (!mbar_wait(my_bars + (kKStages + vslot) * 8, (it / kVStages) & 1)) failed = true;
+        if (has_new) {
+            const uint4* vn = reinterpret_cast<const uint4*>(p.v_new) + (size_t)u * 16;
+            if (lane < 16) {
+                const uint4 x = vn[lane];
+                *reinterpret_cast<uint4*>(vtile + (l_old - k0) * kRowBytes + lane * 16) = x;
+                reinterpret_cast<uint4*>(const_cast<unsigned char*>(Vu) + (size_t)l_old * kRowBytes)[lane] = x;
+            }
+        }
+        if (n_valid < kTileKeys)     // rows the copy did not fetch: make them harmless for 0 * v
+            for (int x = lane; x < (kTileKeys - n_valid) * 16; x += 32)
+                *reinterpret_cast<uint4*>(vtile + n_valid * kRowBytes + x * 16) = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+#pragma unroll 4
+        for (int n = 0; n < 16; ++n) {
+            const int key = 16 * h + n;
+            const uint4 raw = *reinterpret_cast<const uint4*>(vtile + key * kRowBytes + ci * 16);
+            float v[8];
+            unpack8_to_float(raw, v);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float pj = psm[key * G + g];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(pj, v[e], acc[g][e]);     // Eq. 1
+            }
+        }
+        __syncwarp();
+        if (lane == 0 && it + kVStages < my_n) { fence_async_smem(); issue_v(it + kVStages); }
+    }
+    if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
+
+    // fold the warp: lane-private sums of Z, the two halves of acc
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        Zl[g] = warp_sum(Zl[g]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], 16);
+    }
+    __syncthreads();                       // every warp is done with its tiles: the tile area becomes scratch
+    if (s_failed) return;                  // a bounded wait expired: reported through the status word, unit left as is
+    unsigned char* merge = smem + lay.tiles;                      // [NW][G] records {double M, double Z, float acc[128]}
+    constexpr int kRec = 16 + 4 * 128;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+        unsigned char* rec = merge + (warp * G + g) * kRec;
+        if (lane == 0) { reinterpret_cast<double*>(rec)[0] = M[g]; reinterpret_cast<double*>(rec)[1] = Zl[g]; }
+        if (lane < 16) {
+            float4* a = reinterpret_cast<float4*>(rec + 16 + ci * 32);
+            a[0] = make_float4(acc[g][0], acc[g][1], acc[g][2], acc[g][3]);
+            a[1] = make_float4(acc[g][4], acc[g][5], acc[g][6], acc[g][7]);
+        }
+    }
+    __syncthreads();
+    // block-level merge: thread c owns channel c (NT == 128)
+    const size_t pstride = partial_stride(128);
+    for (int g = 0; g < G; ++g) {
+        double Mb = -INFINITY;
+        for (int w = 0; w < NW; ++w) Mb = fmax(Mb, reinterpret_cast<const double*>(merge + (w * G + g) * kRec)[0]);
+        double Zb = 0.0;
+        float a = 0.f;
+        for (int w = 0; w < NW; ++w) {
+            const unsigned char* rec = merge + (w * G + g) * kRec;
+            const double sc = exp_nonpos(reinterpret_cast<const double*>(rec)[0] - Mb);
+            Zb += reinterpret_cast<const double*>(rec)[1] * sc;
+            a += reinterpret_cast<const float*>(rec + 16)[tid] * (float)sc;
+        }
+        if (single) {
+            bf16_t* outp = reinterpret_cast<bf16_t*>(p.out) + ((size_t)u * G + g) * 128;
+            Elem<bf16_t>::store(outp + tid, (float)((double)a / Zb));
+            if (tid == 0) s_thr1[g] = Mb + log(Zb) + p.log_alpha - log((double)t);
+        } else {
+            unsigned char* rec = p.partials + (((size_t)u * p.max_splits + split) * G + g) * pstride;
+            reinterpret_cast<float*>(rec + 16)[tid] = a;
+            if (tid == 0) { reinterpret_cast<double*>(rec)[0] = Mb; reinterpret_cast<double*>(rec)[1] = Zb; }
+        }
+    }
+    if (single) {
+        __syncthreads();
+        finalize_single<G, NT>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, word_sm, pos_sm, merge + NW * G * kRec);
+        return;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned prev = atomicAdd(p.ticket + u, 1u);
+        s_last = (prev == (unsigned)(n_act - 1));
+        if (s_last) p.ticket[u] = 0u;
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_last) return;
+    finalize_unit<bf16_t, 128, G, NT>(p, u, b, l, n_act, t, smem);
+}
+
+// Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
+inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int tune_split_len, int sm_count,
+                                        cudaStream_t st) {
+    (void)sm_count;
+    if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
+    int split_len = tune_split_len ? tune_split_len : (G == 1 ? 512 : 256);
+    split_len = (split_len + kFastWarps * kTileKeys - 1) / (kFastWarps * kTileKeys) * (kFastWarps * kTileKeys);
+    p.split_len = split_len;
+    const int n_splits = (upper + split_len - 1) / split_len;
+    if (n_splits > p.max_splits) return CORM_ERR_UNSUPPORTED;
+    // on-chip finish for units of one split, as long as two blocks still fit on an SM
+    p.single_cap = split_len;
+    while (p.single_cap > 0 && fast_smem_layout(G, p.single_cap).total > 110 * 1024) p.single_cap -= kFastWarps * kTileKeys;
+    const FastSmem lay = fast_smem_layout(G, p.single_cap);
+    size_t smem = (size_t)lay.total;
+    const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // multi-split finalize lists
+    const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
+                        (size_t)2 * p.single_cap * 4;
+    if (fin > smem) smem = fin;
+    if (fin1 > (size_t)kFastWarps * kStagesPerWarp * kTileBytes) return CORM_ERR_UNSUPPORTED;
+    if (smem > 227 * 1024) return CORM_ERR_UNSUPPORTED;
+    auto launch = [&](auto kern) -> corm_status_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        kern<<<dim3(n_splits, (unsigned)p.U), kFastThreads, smem, st>>>(p);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        return CORM_OK;
+    };
+    if (G == 1) return launch(decode_fast_kernel<1>);
+    if (G == 2) return launch(decode_fast_kernel<2>);
+    return launch(decode_fast_kernel<4>);
+}
+
+}  // namespace corm

@@ -20,7 +20,7 @@ __host__ __device__ inline size_t generic_decode_smem(int D, int G, int C) {
 // Decode step, one block per (split of a unit's live range, unit).
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const __grid_constant__ DecodeParams p) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_last;
     constexpr int NT = kGenericThreads, NW = NT / 32, NPL = D / 32;
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -147,7 +147,7 @@ __host__ __device__ inline size_t prompt_smem(int G, int w, int C) {
 // every key for those rows -> registers; then keep flags, prefix sums and an ordered gather into the slab.
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __grid_constant__ PromptParams p) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_scan[kPromptThreads];
     constexpr int NT = kPromptThreads, NW = NT / 32, NPL = D / 32;
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
