@@ -155,9 +155,12 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=384)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
+    ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
+    if args.alpha is not None:
+        cfg = cfg.with_(alpha=args.alpha, name=cfg.name + f"_alpha{args.alpha:g}")
     if args.impl == "reference":
         return run_reference(args, cfg)
 

@@ -6,7 +6,7 @@ import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
-LIB_PATH = os.path.join(_HERE, "libcorm.so")
+LIB_PATH = os.environ.get("CORM_LIB_PATH", os.path.join(_HERE, "libcorm.so"))   # override: load another build
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-O3", "-lineinfo", "--shared",
               "-Xcompiler", "-fPIC"]
 

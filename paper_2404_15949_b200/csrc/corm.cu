@@ -26,7 +26,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, stash, partials;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -69,6 +69,7 @@ Layout make_layout(const corm_config_t& c) {
     L.ticket = take(Ltot * U * 4);
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
+    L.maxlive = take(Ltot * 8);
     L.bookkeeping_end = off;
     L.stash = take(U * G * C * 8);
     L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
@@ -108,6 +109,10 @@ struct corm_cache {
     int U, G;
     size_t e;
     std::vector<int> parity, steps, ready, live_upper;
+    // sizing feedback: the kernels publish the longest live length, the host reads it back without ever waiting
+    unsigned long long* maxlive_host = nullptr;   // pinned, [n_layers]
+    std::vector<cudaEvent_t> readback_ev;
+    std::vector<int> readback_pending, last_readback_step;
     int tune_split_len = 0, allow_fast = 1;
     int sm_count = 148;
     long long launches = 0;
@@ -142,8 +147,33 @@ bool layer_ok(const corm_cache* c, int layer) { return c && layer >= 0 && layer 
 
 double log_alpha_of(const corm_cache* c) { return c->cfg.alpha > 0.f ? std::log((double)c->cfg.alpha) : -INFINITY; }
 
+unsigned long long* maxlive_ptr(const corm_cache* c, int layer) {
+    return reinterpret_cast<unsigned long long*>(c->arena + c->lay.maxlive) + layer;
+}
+
+// If an earlier read-back has landed, tighten the bound on this layer's longest unit: a unit grows by at most one
+// key per step, so (length after step s) + (steps since s) bounds every unit now.
+void poll_live_bound(corm_cache* c, int layer) {
+    if (!c->readback_pending[layer] || cudaEventQuery(c->readback_ev[layer]) != cudaSuccess) return;
+    c->readback_pending[layer] = 0;
+    const unsigned long long v = c->maxlive_host[layer];
+    const int steps_done = (int)(v >> 32), len = (int)(v & 0xffffffffu);
+    if (steps_done > c->steps[layer]) return;   // stale word from before a reset / new prompt
+    const int bound = len + (c->steps[layer] - steps_done);
+    if (bound < c->live_upper[layer]) c->live_upper[layer] = bound;
+}
+
+void schedule_live_readback(corm_cache* c, int layer, cudaStream_t st) {
+    if (c->readback_pending[layer] || !c->maxlive_host) return;
+    if (cudaMemcpyAsync(c->maxlive_host + layer, maxlive_ptr(c, layer), 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return;
+    if (cudaEventRecord(c->readback_ev[layer], st) != cudaSuccess) return;
+    c->readback_pending[layer] = 1;
+    c->last_readback_step[layer] = c->steps[layer];
+}
+
 corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                             cudaStream_t st) {
+    poll_live_bound(c, layer);
     const corm_config_t& cf = c->cfg;
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
     DecodeParams p{};
@@ -158,6 +188,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
     p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
     p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
+    p.maxlive = maxlive_ptr(c, layer);
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.partials = c->arena + c->lay.partials;
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
@@ -189,6 +220,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     c->parity[layer] ^= 1;
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
+    if (c->steps[layer] - c->last_readback_step[layer] >= 8) schedule_live_readback(c, layer, st);
     return CORM_OK;
 }
 
@@ -224,12 +256,28 @@ corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, si
     c->steps.assign(cfg->n_layers, 0);
     c->ready.assign(cfg->n_layers, 0);
     c->live_upper.assign(cfg->n_layers, 0);
+    c->readback_pending.assign(cfg->n_layers, 0);
+    c->last_readback_step.assign(cfg->n_layers, 0);
+    c->readback_ev.assign(cfg->n_layers, nullptr);
+    bool host_ok = cudaHostAlloc(reinterpret_cast<void**>(&c->maxlive_host), sizeof(unsigned long long) * cfg->n_layers,
+                                 cudaHostAllocDefault) == cudaSuccess;   // pinned HOST memory; device memory stays the caller's
+    for (int l = 0; host_ok && l < cfg->n_layers; ++l)
+        host_ok = cudaEventCreateWithFlags(&c->readback_ev[l], cudaEventDisableTiming) == cudaSuccess;
+    if (!host_ok) {
+        std::fprintf(stderr, "corm: could not set up the host-side read-back buffer\n");
+        for (cudaEvent_t ev : c->readback_ev) if (ev) cudaEventDestroy(ev);
+        if (c->maxlive_host) cudaFreeHost(c->maxlive_host);
+        delete c;
+        return CORM_ERR_CUDA;
+    }
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) c->sm_count = sms;
     cudaError_t e = cudaMemset(c->arena + lay.bookkeeping_begin, 0, lay.bookkeeping_end - lay.bookkeeping_begin);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         std::fprintf(stderr, "corm: clearing the arena failed: %s\n", cudaGetErrorString(e));
+        for (cudaEvent_t ev : c->readback_ev) if (ev) cudaEventDestroy(ev);
+        cudaFreeHost(c->maxlive_host);
         delete c;
         return CORM_ERR_CUDA;
     }
@@ -239,6 +287,11 @@ corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, si
 
 corm_status_t corm_cache_destroy(corm_cache_t* cache) {
     if (!cache) return CORM_ERR_INVALID_ARG;
+    {
+        DeviceGuard guard(cache->cfg.device);
+        for (cudaEvent_t ev : cache->readback_ev) if (ev) cudaEventDestroy(ev);
+        if (cache->maxlive_host) cudaFreeHost(cache->maxlive_host);
+    }
     delete cache;
     return CORM_OK;
 }
@@ -249,7 +302,10 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
     if (!guard.ok) return CORM_ERR_CUDA;
     CORM_CUDA(cudaMemsetAsync(c->arena + c->lay.bookkeeping_begin, 0, c->lay.bookkeeping_end - c->lay.bookkeeping_begin,
                               static_cast<cudaStream_t>(stream)));
-    for (int l = 0; l < c->cfg.n_layers; ++l) { c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; }
+    for (int l = 0; l < c->cfg.n_layers; ++l) {
+        c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0;
+        c->readback_pending[l] = 0; c->last_readback_step[l] = 0;
+    }
     return CORM_OK;
 }
 
@@ -279,6 +335,8 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     CORM_CUDA(cudaMemcpyAsync(base_tokens, prompt_lens_host, (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemcpyAsync(base_obs, obs.data(), (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket, U * 4, layer), 0, U * 4, st));
+    CORM_CUDA(cudaMemsetAsync(maxlive_ptr(c, layer), 0, 8, st));
+    c->readback_pending[layer] = 0;   // an older read-back no longer describes this layer
     PromptParams p{};
     p.k_prompt = k_prompt; p.v_prompt = v_prompt; p.q_last = q_last;
     p.prompt_lens = base_tokens;
@@ -289,6 +347,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     p.live_out = live_buf(c, layer, 0);
     p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
     p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
+    p.maxlive = maxlive_ptr(c, layer);
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.p_max = p_max; p.w = cf.window_w; p.r = cf.recent_r;
     p.log_alpha = log_alpha_of(c);
@@ -305,6 +364,8 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     if (rc != CORM_OK) return rc;
     c->launches += 1;
     c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p;
+    c->last_readback_step[layer] = 0;
+    schedule_live_readback(c, layer, st);
     return CORM_OK;
 }
 
@@ -522,6 +583,7 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer) + (size_t)seq * 4, &bo, 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaStreamSynchronize(st));
     c->ready[layer] = 1;
+    c->readback_pending[layer] = 0;   // a read-back enqueued before this import knows nothing of it
     c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
     return CORM_OK;
 }

@@ -25,6 +25,7 @@ struct DecodeParams {
     uint32_t* ticket;         // [U] arrival counters of the splits of a unit (zero between steps)
     unsigned long long* counters;  // [CNT_COUNT]
     int32_t* status;          // sticky device status
+    unsigned long long* maxlive;  // (steps done << 32 | longest live length after that step), atomicMax; may be null
     double* stash;            // [U*G][C] scaled logits of this step (scratch)
     unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
     const void* q;            // [B][Hq][D]
@@ -48,6 +49,7 @@ struct PromptParams {
     int32_t* live_out;        // [U]
     unsigned long long* counters;
     int32_t* status;
+    unsigned long long* maxlive;
     double* stash;            // scratch, reused for temporary registers
     int32_t U, Hkv, C, p_max, w, r;
     double log_alpha;
@@ -104,6 +106,12 @@ __device__ __forceinline__ double warp_sum(double x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
+}
+
+// Publishes a unit's new live length for the host's launch sizing: the word holds the latest step in its high half,
+// so the maximum over all units of the most recent step wins.
+__device__ __forceinline__ void publish_live(unsigned long long* maxlive, int steps_done, int live) {
+    if (maxlive) atomicMax(maxlive, ((unsigned long long)(unsigned)steps_done << 32) | (unsigned)live);
 }
 
 __device__ __forceinline__ uint32_t window_mask(int w) { return w >= 32 ? 0xffffffffu : ((1u << w) - 1u); }
@@ -252,6 +260,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     }
     if (tid == 0) {
         p.live_out[u] = new_len;
+        publish_live(p.maxlive, p.step + 1, new_len);
         atomicAdd(p.counters + CNT_APPENDED, 1ull);
         atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
         if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));

@@ -210,6 +210,7 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     }
     if (tid == 0) {
         p.live_out[u] = new_len;
+        publish_live(p.maxlive, p.step + 1, new_len);
         atomicAdd(p.counters + CNT_APPENDED, 1ull);
         atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
         if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
@@ -228,7 +229,7 @@ __global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __gr
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C) {
-        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; }
+        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
     const int n_act = (l + p.split_len - 1) / p.split_len;
@@ -456,9 +457,17 @@ __global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __gr
 // Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
 inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int tune_split_len, int sm_count,
                                         cudaStream_t st) {
-    (void)sm_count;
     if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
-    int split_len = tune_split_len ? tune_split_len : (G == 1 ? 512 : 256);
+    int split_len = tune_split_len;
+    if (!split_len) {
+        // enough blocks to fill the machine about four times over, but no smaller than one tile per warp and no
+        // larger than 2048 keys (long splits amortise the per-block prologue and merge)
+        const long long total_tiles = (long long)((upper + kTileKeys - 1) / kTileKeys) * p.U;
+        const long long target_blocks = 4ll * (sm_count > 0 ? sm_count : 148);
+        long long tiles_per_block = (total_tiles + target_blocks - 1) / target_blocks;
+        if (tiles_per_block < kFastWarps) tiles_per_block = kFastWarps;
+        split_len = (int)(tiles_per_block * kTileKeys > 2048 ? 2048 : tiles_per_block * kTileKeys);
+    }
     split_len = (split_len + kFastWarps * kTileKeys - 1) / (kFastWarps * kTileKeys) * (kFastWarps * kTileKeys);
     p.split_len = split_len;
     const int n_splits = (upper + split_len - 1) / split_len;

@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C) {   // the slab is full: report, leave the unit untouched
-        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; }
+        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
     const int n_act = (l + p.split_len - 1) / p.split_len;
@@ -261,6 +261,7 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     }
     if (tid == 0) {
         p.live_out[u] = kept_total;
+        publish_live(p.maxlive, 0, kept_total);
         atomicAdd(p.counters + CNT_APPENDED, (unsigned long long)P);
         if (kept_total < P) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(P - kept_total));
     }
