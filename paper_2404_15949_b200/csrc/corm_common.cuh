@@ -117,19 +117,31 @@ __device__ __forceinline__ void publish_live(unsigned long long* maxlive, int st
 __device__ __forceinline__ uint32_t window_mask(int w) { return w >= 32 ? 0xffffffffu : ((1u << w) - 1u); }
 
 // Exclusive prefix sums of popc(mask[i]) into prefix[0..nwords], block-wide. scratch holds NT ints.
+// Each thread sums a contiguous run of words; warp 0 scans the NT run totals with shuffles.
 template <int NT>
 __device__ void block_popc_scan(const uint32_t* mask, int* prefix, int nwords, int* scratch) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int per = (nwords + NT - 1) / NT;
     const int lo = min(tid * per, nwords), hi = min(lo + per, nwords);
     int sum = 0;
     for (int i = lo; i < hi; ++i) sum += __popc(mask[i]);
     scratch[tid] = sum;
     __syncthreads();
-    if (tid == 0) {
-        int run = 0;
-        for (int i = 0; i < NT; ++i) { int v = scratch[i]; scratch[i] = run; run += v; }
-        prefix[nwords] = run;
+    if (tid < 32) {
+        constexpr int kPer = NT / 32;
+        int v[kPer], tot = 0;
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) { v[k] = scratch[lane * kPer + k]; tot += v[k]; }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int run = incl - tot;
+#pragma unroll
+        for (int k = 0; k < kPer; ++k) { scratch[lane * kPer + k] = run; run += v[k]; }
+        if (lane == 31) prefix[nwords] = incl;
     }
     __syncthreads();
     int run = scratch[tid];
@@ -221,19 +233,40 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     const bool evict_on = n_obs >= p.w;
     const uint32_t wmask = window_mask(p.w);
     const double* stash_u = p.stash + (size_t)u * G * p.C;
-    for (int base = 0; base < l; base += NT) {
-        const int j = base + tid;
-        bool keep = false;
-        if (j < l) {
-            bool imp = false;
+    constexpr int kBatch = 4;                                      // slots per thread whose loads are issued together
+    for (int base0 = 0; base0 < l; base0 += kBatch * NT) {
+        double sv[kBatch][G];
+        uint32_t wv[kBatch];
+        int32_t pv[kBatch];
 #pragma unroll
-            for (int g = 0; g < G; ++g) imp |= (__ldcg(stash_u + (size_t)g * p.C + j) >= s_thr[g]);
-            const uint32_t wd = ((__ldcg(wordu + j) << 1) | (imp ? 1u : 0u)) & wmask;
-            wordu[j] = wd;
-            keep = !evict_on || wd != 0u || __ldcg(posu + j) > t - p.r;
+        for (int k = 0; k < kBatch; ++k) {
+            const int j = base0 + k * NT + tid;
+            wv[k] = 0u; pv[k] = 0;
+#pragma unroll
+            for (int g = 0; g < G; ++g) sv[k][g] = -INFINITY;
+            if (j < l) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) sv[k][g] = __ldcg(stash_u + (size_t)g * p.C + j);
+                wv[k] = __ldcg(wordu + j);
+                pv[k] = __ldcg(posu + j);
+            }
         }
-        const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+            const int base = base0 + k * NT, j = base + tid;
+            if (base >= l) break;                                  // uniform
+            bool keep = false;
+            if (j < l) {
+                bool imp = false;
+#pragma unroll
+                for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
+                const uint32_t wd = ((wv[k] << 1) | (imp ? 1u : 0u)) & wmask;
+                wordu[j] = wd;
+                keep = !evict_on || wd != 0u || pv[k] > t - p.r;
+            }
+            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
+        }
     }
     __syncthreads();
     int new_len = l, n_moved = 0;

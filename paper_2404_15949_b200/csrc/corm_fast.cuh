@@ -21,27 +21,32 @@ constexpr int kFastThreads = kFastWarps * 32;
 constexpr int kTileKeys = 32;
 constexpr int kRowBytes = 256;                    // 128 bf16
 constexpr int kTileBytes = kTileKeys * kRowBytes; // 8 KiB
-constexpr int kKStages = 2, kVStages = 1;
-constexpr int kStagesPerWarp = kKStages + kVStages;
+constexpr int kVStages = 1;
+// K stages per warp, resident blocks per SM and the shared-memory budget that allows them, by group size:
+// one query head per KV head leaves registers and shared memory for three blocks per SM; larger groups keep two.
+__host__ __device__ constexpr int fast_k_stages(int G) { return G == 1 ? 1 : 2; }
+__host__ __device__ constexpr int fast_stages(int G) { return fast_k_stages(G) + kVStages; }
+__host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? 3 : 2; }
+__host__ __device__ constexpr int fast_smem_budget(int G) { return G == 1 ? 74 * 1024 : 111 * 1024; }
 constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits (about 2 s)
+// longest unit that may finish inside one block (bounded by the registers that carry its verdict words)
+__host__ __device__ constexpr int fast_max_single_cap(int G) { return G == 1 ? 1024 : 256; }
 
 inline bool fast_path_available() { return true; }
 
 // ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
 struct FastSmem {
-    int tiles, qs, psm, stash, word, pos, bars, total;
+    int tiles, qs, psm, stash, bars, total;
 };
 __host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
     FastSmem s;
     int off = 0;
     auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
-    s.tiles = take(kFastWarps * kStagesPerWarp * kTileBytes);   // later reused: merge area, finalize lists
+    s.tiles = take(kFastWarps * fast_stages(G) * kTileBytes);   // later reused: merge area, finalize lists
     s.qs = take(G * 128 * 8);
     s.psm = take(kFastWarps * kTileKeys * G * 4);
     s.stash = take(single_cap * G * 8);
-    s.word = take(single_cap * 4);
-    s.pos = take(single_cap * 4);
-    s.bars = take(kFastWarps * kStagesPerWarp * 8);
+    s.bars = take(kFastWarps * fast_stages(G) * 8);
     s.total = off;
     return s;
 }
@@ -156,10 +161,11 @@ __device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double
 
 // Single-split finalize: logits, registers and positions of the whole unit are in shared memory.
 // lists: scratch for the keep mask, its prefix sums and the hole / mover lists (ints).
-template <int G, int NT>
+// wv / pv: registers and positions of slots tid, tid + NT, ... (loaded by the caller at block start).
+template <int G, int NT, int KPRE>
 __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int t, const double* thr,
-                                const double* stash_sm, int stash_ld, uint32_t* word_sm, const int32_t* pos_sm,
-                                unsigned char* lists) {
+                                const double* stash_sm, int stash_ld, const uint32_t (&wv)[KPRE],
+                                const int32_t (&pv)[KPRE], unsigned char* lists) {
     __shared__ int s_scan1[NT];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cap_words = (l + 31) / 32 + 2;
@@ -174,16 +180,18 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
     const bool evict_on = n_obs >= p.w;
     const uint32_t wmask = window_mask(p.w);
-    for (int base = 0; base < l; base += NT) {
-        const int j = base + tid;
+#pragma unroll
+    for (int k = 0; k < KPRE; ++k) {
+        const int base = k * NT, j = base + tid;
+        if (base >= l) break;                                     // uniform
         bool keep = false;
         if (j < l) {
             bool imp = false;
 #pragma unroll
             for (int g = 0; g < G; ++g) imp |= (stash_sm[g * stash_ld + j] >= thr[g]);
-            const uint32_t wd = ((word_sm[j] << 1) | (imp ? 1u : 0u)) & wmask;
+            const uint32_t wd = ((wv[k] << 1) | (imp ? 1u : 0u)) & wmask;
             wordu[j] = wd;
-            keep = !evict_on || wd != 0u || pos_sm[j] > t - p.r;
+            keep = !evict_on || wd != 0u || pv[k] > t - p.r;
         }
         const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
         if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
@@ -219,12 +227,13 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
 }
 
 template <int G>
-__global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
+__global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_last;
     __shared__ int s_failed;
     __shared__ double s_thr1[G];
     constexpr int NT = kFastThreads, NW = kFastWarps;
+    constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
@@ -244,8 +253,6 @@ __global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __gr
     double* qs = reinterpret_cast<double*>(smem + lay.qs);
     float* psm = reinterpret_cast<float*>(smem + lay.psm) + warp * kTileKeys * G;
     double* stash_sm = reinterpret_cast<double*>(smem + lay.stash);
-    uint32_t* word_sm = reinterpret_cast<uint32_t*>(smem + lay.word);
-    int32_t* pos_sm = reinterpret_cast<int32_t*>(smem + lay.pos);
     const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.K) + (size_t)u * p.C * kRowBytes;
     const unsigned char* Vu = reinterpret_cast<const unsigned char*>(p.V) + (size_t)u * p.C * kRowBytes;
     uint32_t* wordu = p.word + (size_t)u * p.C;
@@ -281,14 +288,28 @@ __global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __gr
         for (int it = 0; it < min(my_n, kVStages); ++it) issue_v(it);
     }
 
-    // queries widened to fp64 once per block; registers and positions of a single-split unit staged on chip
+    // queries widened to fp64 once per block; a single-split unit also fetches the registers and positions of the
+    // slots this thread will judge in the finalize phase (slots tid, tid + NT, ...) and keeps them in registers
+    constexpr int kPre = fast_max_single_cap(G) / NT;
+    uint32_t wv[kPre];
+    int32_t pv[kPre];
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) { wv[k] = 0u; pv[k] = 0; }
+    if (single) {
+#pragma unroll
+        for (int k = 0; k < kPre; ++k) {
+            const int j = tid + k * NT;
+            if (j < l_old) { wv[k] = __ldcg(wordu + j); pv[k] = __ldcg(posu + j); }
+            else if (j == l_old) { wv[k] = 0u; pv[k] = t; }          // the token appended by this step
+        }
+    }
     {
         const bf16_t* qg = reinterpret_cast<const bf16_t*>(p.q) + (size_t)u * G * 128;
-        for (int x = tid; x < G * 128; x += NT) qs[x] = (double)Elem<bf16_t>::load(qg + x);
-        if (single) {
-            for (int j = tid; j < l_old; j += NT) { word_sm[j] = __ldcg(wordu + j); pos_sm[j] = __ldcg(posu + j); }
-            if (tid == 0) { word_sm[l_old] = 0u; pos_sm[l_old] = t; }
-        }
+        float qv[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) qv[g] = Elem<bf16_t>::load(qg + g * 128 + tid);      // NT == 128 channels
+#pragma unroll
+        for (int g = 0; g < G; ++g) qs[g * 128 + tid] = (double)qv[g];
     }
     __syncthreads();
 
@@ -438,7 +459,7 @@ __global__ void __launch_bounds__(kFastThreads, 2) decode_fast_kernel(const __gr
     }
     if (single) {
         __syncthreads();
-        finalize_single<G, NT>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, word_sm, pos_sm, merge + NW * G * kRec);
+        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, merge + NW * G * kRec);
         return;
     }
     __threadfence();
@@ -473,15 +494,15 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     const int n_splits = (upper + split_len - 1) / split_len;
     if (n_splits > p.max_splits) return CORM_ERR_UNSUPPORTED;
     // on-chip finish for units of one split, as long as two blocks still fit on an SM
-    p.single_cap = split_len;
-    while (p.single_cap > 0 && fast_smem_layout(G, p.single_cap).total > 110 * 1024) p.single_cap -= kFastWarps * kTileKeys;
+    p.single_cap = split_len < fast_max_single_cap(G) ? split_len : fast_max_single_cap(G);
+    while (p.single_cap > 0 && fast_smem_layout(G, p.single_cap).total > fast_smem_budget(G)) p.single_cap -= kFastWarps * kTileKeys;
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
     size_t smem = (size_t)lay.total;
     const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // multi-split finalize lists
     const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
                         (size_t)2 * p.single_cap * 4;
     if (fin > smem) smem = fin;
-    if (fin1 > (size_t)kFastWarps * kStagesPerWarp * kTileBytes) return CORM_ERR_UNSUPPORTED;
+    if (fin1 > (size_t)kFastWarps * fast_stages(G) * kTileBytes) return CORM_ERR_UNSUPPORTED;
     if (smem > 227 * 1024) return CORM_ERR_UNSUPPORTED;
     auto launch = [&](auto kern) -> corm_status_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
