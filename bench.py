@@ -1,8 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the fused CORM decode+evict step (one JSON line on stdout).
 
-A "step" is one decode step of one layer for the whole batch: append, attention over every unit's live keys,
-verdicts, register update and compaction, all inside one kernel launch. Default workload: the batched-throughput
+A "step" is one decode step of the whole batch through every layer of the configuration (one layer for the default
+workload): append, attention over every unit's live keys, verdicts, register update and compaction, one kernel
+launch per layer. Default workload: the batched-throughput
 configuration (batch 32, 32 heads, head_dim 128, bf16, ragged prompts in [2048, 4096]).
 
     python bench.py --gpus 1 --steps 256 --warmup 16
@@ -139,7 +140,7 @@ def workload_config(cfg, args):
     return {"workload": f"{cfg.name} (BASELINE configs[{args.workload - 1}])", "batch": cfg.batch,
             "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
             "prompt_len": [cfg.prompt_min, cfg.prompt_max], "window_w": cfg.window_w, "recent_r": cfg.recent_r,
-            "alpha": cfg.alpha, "layers_per_step": 1, "seed": cfg.seed,
+            "alpha": cfg.alpha, "layers_per_step": cfg.n_layers, "seed": cfg.seed,
             "l2": "live K/V read per step exceeds the 126 MB L2 (no flush needed)"}
 
 
@@ -175,34 +176,43 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     # each rank owns an independent shard (its own batch, its own arena): no data-path collective
-    cfg_r = cfg.with_(seed=cfg.seed + rank)
+    from paper_2404_15949_b200.sharding import aggregate_throughput, shard_config
+    cfg_r = shard_config(cfg, rank, world)
     n_steps = args.warmup + args.steps + args.e2e_steps
     cfg_r = cfg_r.with_(steps=max(cfg.steps, n_steps))
-    L = 1
+    L = cfg.n_layers                     # a step = one token through every layer of the configuration
     t0 = time.perf_counter()
-    data = generate(cfg_r, n_steps=n_steps)
-    log(f"[rank {rank}] generated {cfg.name} inputs in {time.perf_counter() - t0:.1f} s")
+    data = [generate(cfg_r, layer=l, n_steps=n_steps) for l in range(L)]
+    log(f"[rank {rank}] generated {cfg.name} inputs ({L} layer(s)) in {time.perf_counter() - t0:.1f} s")
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
                       cfg.recent_r, cfg.alpha, cfg.dtype, local)
     cache.corm_cache_set_tuning(args.split_len, not args.no_fast)
-    kp, vp, ql = dev(data.k_prompt), dev(data.v_prompt), dev(data.q_last)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
-    torch.cuda.synchronize()
-    a.record()
-    cache.corm_compress_prompt(0, kp, vp, ql, data.prompt_lens)
-    b.record()
-    torch.cuda.synchronize()
-    prompt_ms = a.elapsed_time(b)
-    del kp, vp, ql
+    prompt_ms = 0.0
+    for l in range(L):
+        kp, vp, ql = dev(data[l].k_prompt), dev(data[l].v_prompt), dev(data[l].q_last)
+        torch.cuda.synchronize()
+        a.record()
+        cache.corm_compress_prompt(l, kp, vp, ql, data[l].prompt_lens)
+        b.record()
+        torch.cuda.synchronize()
+        prompt_ms += a.elapsed_time(b)
+        del kp, vp, ql
     st0 = cache.corm_cache_stats()
-    q_d, k_d, v_d = dev(data.q), dev(data.k_new), dev(data.v_new)
-    out = torch.empty_like(q_d[0])
+    q_d = [dev(d.q) for d in data]
+    k_d = [dev(d.k_new) for d in data]
+    v_d = [dev(d.v_new) for d in data]
+    out = torch.empty_like(q_d[0][0])
+
+    def step(s):
+        for l in range(L):
+            cache.corm_decode_step(l, q_d[l][s], k_d[l][s], v_d[l][s], out)
 
     for s in range(args.warmup):
-        cache.corm_decode_step(0, q_d[s], k_d[s], v_d[s], out)
+        step(s)
     torch.cuda.synchronize()
     st1 = cache.corm_cache_stats()
     launches0 = cache.corm_cache_kernel_launches()
@@ -213,7 +223,7 @@ def main():
     torch.cuda.synchronize()
     a.record()
     for s in range(args.warmup, args.warmup + args.steps):
-        cache.corm_decode_step(0, q_d[s], k_d[s], v_d[s], out)
+        step(s)
     b.record()
     torch.cuda.synchronize()
     if world > 1:
@@ -229,33 +239,32 @@ def main():
     if args.e2e_steps:
         base = args.warmup + args.steps
         pin = lambda t: t.cpu().pin_memory()
-        qh, kh, vh = pin(q_d[base:]), pin(k_d[base:]), pin(v_d[base:])
-        oh = torch.empty_like(qh[0]).pin_memory()
-        h2d = qh[0].numel() * qh.element_size() + 2 * kh[0].numel() * kh.element_size()
-        d2h = oh.numel() * oh.element_size()
+        qh = [pin(x[base:]) for x in q_d]
+        kh = [pin(x[base:]) for x in k_d]
+        vh = [pin(x[base:]) for x in v_d]
+        oh = torch.empty_like(qh[0][0]).pin_memory()
+        h2d = L * (qh[0][0].numel() + 2 * kh[0][0].numel()) * oh.element_size()
+        d2h = L * oh.numel() * oh.element_size()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         a.record()
         for s in range(args.e2e_steps):
-            cache.corm_decode_step_host(0, qh[s], kh[s], vh[s], oh)
+            for l in range(L):
+                cache.corm_decode_step_host(l, qh[l][s], kh[l][s], vh[l][s], oh)
         b.record()
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(b)
     st3 = cache.corm_cache_stats()
     assert st3["device_status"] == 0, f"device status {st3['device_status']}"
 
-    times = torch.tensor([ms, e2e_ms or 0.0], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_max, e2e_max = float(times[0]), float(times[1])
+    value, ms_max, _ = aggregate_throughput(ms, cfg.batch * args.steps, "cuda")
+    e2e_value = aggregate_throughput(e2e_ms, cfg.batch * args.e2e_steps, "cuda")[0] if e2e_ms else None
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-    tokens = cfg.batch * args.steps * world
-    value = tokens / (ms_max * 1e-3)
-    unit_steps = cfg.batch * cfg.n_kv_heads * args.steps
+    unit_steps = L * cfg.batch * cfg.n_kv_heads * args.steps
     attended = st2["attended_keys"] - st1["attended_keys"]
     moved = st2["moved_rows"] - st1["moved_rows"]
     abytes = algorithmic_bytes(cfg, attended, moved, unit_steps)
@@ -268,14 +277,14 @@ def main():
         "config": workload_config(cfg, args),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src, "traffic": None,
-                     "kernel": "decode step kernel (one launch per step)",
-                     "bytes_per_launch": abytes / args.steps, "us_per_launch": 1e3 * ms / args.steps},
-        "e2e": {"value": (cfg.batch * args.e2e_steps * world / (e2e_max * 1e-3)) if e2e_ms else None, "unit": UNIT,
+                     "kernel": "decode step kernel (one launch per layer per step)",
+                     "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * ms / (args.steps * L)},
+        "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "clocks": sampler.result(),
         "retention": st2["retention"],
-        "live_keys_per_unit": st2["live_keys"] / (cfg.batch * cfg.n_kv_heads),
+        "live_keys_per_unit": st2["live_keys"] / (L * cfg.batch * cfg.n_kv_heads),
         "evicted_keys_timed": st2["evicted_keys"] - st1["evicted_keys"], "moved_rows_timed": moved,
         "prompt_pass_ms": prompt_ms, "retention_after_prompt": st0["retention"],
         "paper_context": "paper reports KV memory only: up to 70% reduction (V100-32GB / A100-80GB), no throughput",
