@@ -30,6 +30,10 @@ from paper_2404_15949_b200.workload import CONFIGS, generate  # noqa: E402
 METRIC = "corm_decode_step_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per algorithmic byte of the decode kernel, from the ncu capture summarised in
+# profiles/decode_fast_kernel_batch32_bf16.md (323.9 MB moved for 313.1 MB algorithmic at the captured steps).
+# Set to None whenever the kernel changes until the counters are taken again.
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.034}
 
 
 def log(*a):
@@ -97,6 +101,7 @@ def oracle_baseline(cfg, n_seqs, n_steps):
     heads), n_steps decode steps from the post-prompt-compression state."""
     from oracle import CormOracle
     seqs = list(range(min(n_seqs, cfg.batch)))
+    n_steps = min(n_steps, cfg.steps)
     data = generate(cfg, seqs=seqs, n_steps=n_steps)
     orc = CormOracle(1, len(seqs), cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.max_tokens, cfg.window_w,
                      cfg.recent_r, cfg.alpha)
@@ -125,7 +130,7 @@ def run_reference(args, cfg):
         if total > 150:      # keep the whole run within a few minutes
             break
     timed = per_step[min(args.warmup, len(per_step) - 1):]
-    value = args.ref_seqs * args.ref_steps / float(np.mean(timed))
+    value = min(args.ref_seqs, cfg.batch) * min(args.ref_steps, cfg.steps) / float(np.mean(timed))
     base["value"] = value
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": len(timed), "warmup": len(per_step) - len(timed), "ms_per_step": 1e3 * float(np.mean(timed)),
@@ -152,8 +157,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--e2e-steps", type=int, default=64)
-    ap.add_argument("--ref-seqs", type=int, default=8)
-    ap.add_argument("--ref-steps", type=int, default=384)
+    ap.add_argument("--ref-seqs", type=int, default=32)
+    ap.add_argument("--ref-steps", type=int, default=512)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
@@ -276,7 +281,8 @@ def main():
         "dtype": "f64 logits / f32 accumulation over " + cfg.dtype + " cache", "data": "synthetic",
         "config": workload_config(cfg, args),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src, "traffic": None,
+                     "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src,
+                     "traffic": (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE.get(cfg.name) or 0) * abytes / (args.steps * L) or None,
                      "kernel": "decode step kernel (one launch per layer per step)",
                      "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * ms / (args.steps * L)},
         "e2e": {"value": e2e_value, "unit": UNIT,
