@@ -16,7 +16,13 @@
 
 namespace corm {
 
-constexpr int kFastWarps = 4;
+#ifndef CORM_FAST_WARPS
+#define CORM_FAST_WARPS 4
+#endif
+#ifndef CORM_FAST_BLOCKS_G1
+#define CORM_FAST_BLOCKS_G1 3
+#endif
+constexpr int kFastWarps = CORM_FAST_WARPS;
 constexpr int kFastThreads = kFastWarps * 32;
 constexpr int kTileKeys = 32;
 constexpr int kRowBytes = 256;                    // 128 bf16
@@ -26,11 +32,12 @@ constexpr int kVStages = 1;
 // one query head per KV head leaves registers and shared memory for three blocks per SM; larger groups keep two.
 __host__ __device__ constexpr int fast_k_stages(int G) { return G == 1 ? 1 : 2; }
 __host__ __device__ constexpr int fast_stages(int G) { return fast_k_stages(G) + kVStages; }
-__host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? 3 : 2; }
-__host__ __device__ constexpr int fast_smem_budget(int G) { return G == 1 ? 74 * 1024 : 111 * 1024; }
+__host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? CORM_FAST_BLOCKS_G1 : 2; }
+// 228 KB per SM, minus 1 KB the system reserves per block and ~1.2 KB of static shared memory
+__host__ __device__ constexpr int fast_smem_budget(int G) { return (228 * 1024) / fast_blocks_per_sm(G) - 2304; }
 constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits (about 2 s)
 // longest unit that may finish inside one block (bounded by the registers that carry its verdict words)
-__host__ __device__ constexpr int fast_max_single_cap(int G) { return G == 1 ? 1024 : 256; }
+__host__ __device__ constexpr int fast_max_single_cap(int G) { return (G == 1 ? 8 : 2) * kFastThreads; }
 
 inline bool fast_path_available() { return true; }
 
@@ -305,11 +312,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     }
     {
         const bf16_t* qg = reinterpret_cast<const bf16_t*>(p.q) + (size_t)u * G * 128;
-        float qv[G];
-#pragma unroll
-        for (int g = 0; g < G; ++g) qv[g] = Elem<bf16_t>::load(qg + g * 128 + tid);      // NT == 128 channels
-#pragma unroll
-        for (int g = 0; g < G; ++g) qs[g * 128 + tid] = (double)qv[g];
+        for (int x = tid; x < G * 128; x += NT) qs[x] = (double)Elem<bf16_t>::load(qg + x);
     }
     __syncthreads();
 
@@ -434,27 +437,36 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         }
     }
     __syncthreads();
-    // block-level merge: thread c owns channel c (NT == 128)
+    // block-level merge: thread tid owns channels tid, tid + NT, ...
     const size_t pstride = partial_stride(128);
     for (int g = 0; g < G; ++g) {
         double Mb = -INFINITY;
         for (int w = 0; w < NW; ++w) Mb = fmax(Mb, reinterpret_cast<const double*>(merge + (w * G + g) * kRec)[0]);
         double Zb = 0.0;
-        float a = 0.f;
+        float scw[NW];
         for (int w = 0; w < NW; ++w) {
             const unsigned char* rec = merge + (w * G + g) * kRec;
             const double sc = exp_nonpos(reinterpret_cast<const double*>(rec)[0] - Mb);
             Zb += reinterpret_cast<const double*>(rec)[1] * sc;
-            a += reinterpret_cast<const float*>(rec + 16)[tid] * (float)sc;
+            scw[w] = (float)sc;
         }
-        if (single) {
-            bf16_t* outp = reinterpret_cast<bf16_t*>(p.out) + ((size_t)u * G + g) * 128;
-            Elem<bf16_t>::store(outp + tid, (float)((double)a / Zb));
-            if (tid == 0) s_thr1[g] = Mb + log(Zb) + p.log_alpha - log((double)t);
-        } else {
-            unsigned char* rec = p.partials + (((size_t)u * p.max_splits + split) * G + g) * pstride;
-            reinterpret_cast<float*>(rec + 16)[tid] = a;
-            if (tid == 0) { reinterpret_cast<double*>(rec)[0] = Mb; reinterpret_cast<double*>(rec)[1] = Zb; }
+        for (int c = tid; c < 128; c += NT) {
+            float a = 0.f;
+            for (int w = 0; w < NW; ++w) a += reinterpret_cast<const float*>(merge + (w * G + g) * kRec + 16)[c] * scw[w];
+            if (single) {
+                bf16_t* outp = reinterpret_cast<bf16_t*>(p.out) + ((size_t)u * G + g) * 128;
+                Elem<bf16_t>::store(outp + c, (float)((double)a / Zb));
+            } else {
+                unsigned char* rec = p.partials + (((size_t)u * p.max_splits + split) * G + g) * pstride;
+                reinterpret_cast<float*>(rec + 16)[c] = a;
+            }
+        }
+        if (tid == 0) {
+            if (single) s_thr1[g] = Mb + log(Zb) + p.log_alpha - log((double)t);
+            else {
+                unsigned char* rec = p.partials + (((size_t)u * p.max_splits + split) * G + g) * pstride;
+                reinterpret_cast<double*>(rec)[0] = Mb; reinterpret_cast<double*>(rec)[1] = Zb;
+            }
         }
     }
     if (single) {
