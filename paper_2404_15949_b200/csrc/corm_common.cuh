@@ -233,7 +233,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     const bool evict_on = n_obs >= p.w;
     const uint32_t wmask = window_mask(p.w);
     const double* stash_u = p.stash + (size_t)u * G * p.C;
-    constexpr int kBatch = 4;                                      // slots per thread whose loads are issued together
+    constexpr int kBatch = (G >= 4 ? 4 : 8);                                      // slots per thread whose loads are issued together
     for (int base0 = 0; base0 < l; base0 += kBatch * NT) {
         double sv[kBatch][G];
         uint32_t wv[kBatch];

@@ -119,6 +119,25 @@ __device__ __forceinline__ void unpack8_to_double(const uint4& raw, double (&kd)
     kd[4] = (double)__uint_as_float(raw.z << 16); kd[5] = (double)__uint_as_float(raw.z & 0xffff0000u);
     kd[6] = (double)__uint_as_float(raw.w << 16); kd[7] = (double)__uint_as_float(raw.w & 0xffff0000u);
 }
+// Packed fp32 pairs (sm_100 has a two-wide fp32 FMA): helpers for the P.V accumulation.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void fma_f32x2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ void mul_f32x2(unsigned long long& acc, unsigned long long a) {
+    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(acc) : "l"(a));
+}
+// one 32-bit word holding two bf16 -> the two values as a packed fp32 pair (element 0 in the low half)
+__device__ __forceinline__ unsigned long long bf16x2_to_f32x2(uint32_t w) {
+    return pack_f32x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
 __device__ __forceinline__ void unpack8_to_float(const uint4& raw, float (&v)[8]) {
     v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xffff0000u);
     v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xffff0000u);
@@ -324,12 +343,12 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 #pragma unroll
         for (int e = 0; e < 8; ++e) qd[g][e] = qs[g * 128 + ci * 8 + e];
     double M[G], Zl[G];
-    float acc[G][8];
+    unsigned long long acc2[G][4];                                // P.V accumulators: channel pairs (2e, 2e+1) of this lane's 8
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         M[g] = -INFINITY; Zl[g] = 0.0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[g][e] = 0.f;
+        for (int e = 0; e < 4; ++e) acc2[g][e] = 0ull;
     }
     const double inv_root_d = 0.088388347648318440550;          // 1/sqrt(128)
     bool failed = false;
@@ -374,8 +393,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
                 const double sc = exp_nonpos(M[g] - mtd);
                 const float scf = (float)sc;
                 Zl[g] *= sc;
+                const unsigned long long sc2 = pack_f32x2(scf, scf);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[g][e] *= scf;
+                for (int e = 0; e < 4; ++e) mul_f32x2(acc2[g][e], sc2);
                 M[g] = mtd;
             }
             const double ex = valid ? exp_nonpos(s - M[g]) : 0.0;
@@ -401,13 +421,14 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         for (int n = 0; n < 16; ++n) {
             const int key = 16 * h + n;
             const uint4 raw = *reinterpret_cast<const uint4*>(vtile + key * kRowBytes + ci * 16);
-            float v[8];
-            unpack8_to_float(raw, v);
+            const unsigned long long v2[4] = {bf16x2_to_f32x2(raw.x), bf16x2_to_f32x2(raw.y), bf16x2_to_f32x2(raw.z),
+                                              bf16x2_to_f32x2(raw.w)};
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float pj = psm[key * G + g];
+                const unsigned long long p2 = pack_f32x2(pj, pj);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) acc[g][e] = fmaf(pj, v[e], acc[g][e]);     // Eq. 1
+                for (int e = 0; e < 4; ++e) fma_f32x2(acc2[g][e], p2, v2[e]);           // Eq. 1
             }
         }
         __syncwarp();
@@ -416,9 +437,12 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
 
     // fold the warp: lane-private sums of Z, the two halves of acc
+    float acc[G][8];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
         Zl[g] = warp_sum(Zl[g]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) unpack_f32x2(acc2[g][e], acc[g][2 * e], acc[g][2 * e + 1]);
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], 16);
     }
