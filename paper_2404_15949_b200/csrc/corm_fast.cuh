@@ -91,8 +91,9 @@ __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier
 
 // exp(x) for x <= ~0 (small positive arguments are fine), 0 below the normal range. Argument reduction by ln 2 in
 // two pieces, degree-11 Taylor polynomial on |r| <= ln2/2 (truncation ~6e-15 relative), scaling through the exponent.
-__device__ __forceinline__ double exp_nonpos(double x) {
-    if (!(x > -708.0)) return 0.0;
+// Branch-free, so that several independent calls interleave.
+__device__ __forceinline__ double exp_nonpos(double x0) {
+    const double x = fmax(x0, -708.0);
     const double t = fma(x, 1.4426950408889634074, 6755399441055744.0);   // round(x / ln 2) in the low word
     const int n = __double2loint(t);
     const double nf = t - 6755399441055744.0;
@@ -110,7 +111,8 @@ __device__ __forceinline__ double exp_nonpos(double x) {
     p = fma(p, r, 0.5);
     p = fma(p, r, 1.0);
     p = fma(p, r, 1.0);
-    return p * __hiloint2double((1023 + n) << 20, 0);
+    const double y = p * __hiloint2double((1023 + n) << 20, 0);
+    return x0 > -708.0 ? y : 0.0;
 }
 
 __device__ __forceinline__ void unpack8_to_double(const uint4& raw, double (&kd)[8]) {
@@ -378,29 +380,44 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
         const bool valid = key_own < n_valid;
         const int j_own = k0 + key_own;
+        // softmax bookkeeping for all heads at once: the per-head chains (shuffles, exponentials) are independent
+        double sv[G], Mn[G], sc[G], ex[G];
+        float mt[G];
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-            const double s = valid ? sown[g] * inv_root_d : -INFINITY;     // Eq. 2's exponent
-            if (valid) {
-                if (single) stash_sm[g * p.single_cap + j_own] = s;
-                else p.stash[((size_t)u * G + g) * p.C + j_own] = s;
-            }
-            float mt = (float)s;
+            sv[g] = valid ? sown[g] * inv_root_d : -INFINITY;             // Eq. 2's exponent
+            mt[g] = (float)sv[g];
+        }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, o));
-            const double mtd = (double)mt;
-            if (mtd > M[g]) {                                              // warp-uniform
-                const double sc = exp_nonpos(M[g] - mtd);
-                const float scf = (float)sc;
-                Zl[g] *= sc;
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int g = 0; g < G; ++g) mt[g] = fmaxf(mt[g], __shfl_xor_sync(0xffffffffu, mt[g], o));
+#pragma unroll
+        for (int g = 0; g < G; ++g) Mn[g] = fmax(M[g], (double)mt[g]);   // new reference: warp-uniform, >= every logit so far (up to fp32 rounding)
+#pragma unroll
+        for (int g = 0; g < G; ++g) sc[g] = exp_nonpos(M[g] - Mn[g]);    // exactly 1 when the reference did not move
+#pragma unroll
+        for (int g = 0; g < G; ++g) ex[g] = valid ? exp_nonpos(sv[g] - Mn[g]) : 0.0;
+        bool moved = false;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            moved |= (Mn[g] != M[g]);
+            Zl[g] = fma(Zl[g], sc[g], ex[g]);
+            M[g] = Mn[g];
+            psm[key_own * G + g] = (float)ex[g];
+            if (valid) {
+                if (single) stash_sm[g * p.single_cap + j_own] = sv[g];
+                else p.stash[((size_t)u * G + g) * p.C + j_own] = sv[g];
+            }
+        }
+        if (moved) {                                                       // warp-uniform
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float scf = (float)sc[g];
                 const unsigned long long sc2 = pack_f32x2(scf, scf);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) mul_f32x2(acc2[g][e], sc2);
-                M[g] = mtd;
             }
-            const double ex = valid ? exp_nonpos(s - M[g]) : 0.0;
-            Zl[g] += ex;
-            psm[key_own * G + g] = (float)ex;
         }
         __syncwarp();
 
