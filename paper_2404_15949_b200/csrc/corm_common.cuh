@@ -34,6 +34,8 @@ struct DecodeParams {
     void* out;                // [B][Hq][D]
     int32_t U, Hkv, C, split_len, max_splits, step, w, r;
     int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
+    int32_t n_splits;         // streaming kernel: work items are (unit, split) pairs, split < n_splits
+    uint32_t* queue;          // streaming kernel: {next work item, finished blocks}, both zero between launches
     double log_alpha;         // ln(alpha), -inf for alpha = 0
 };
 
@@ -153,23 +155,48 @@ __device__ __forceinline__ int kept_before(const uint32_t* mask, const int* pref
     return prefix[j >> 5] + __popc(mask[j >> 5] & ((1u << (j & 31)) - 1u));
 }
 
-// Copies one K row and one V row (D elements each) plus register and position from slot src to slot dst of a unit;
-// executed by one warp. Rows are D*sizeof(T) bytes = a multiple of 16.
-template <typename T, int D>
-__device__ __forceinline__ void warp_move_row(T* Ku, T* Vu, uint32_t* wordu, int32_t* posu, int src, int dst,
-                                              int lane) {
-    constexpr int kChunks = D * Elem<T>::kBytes / 16;
-    const uint4* ks = reinterpret_cast<const uint4*>(Ku + (size_t)src * D);
-    const uint4* vs = reinterpret_cast<const uint4*>(Vu + (size_t)src * D);
-    uint4* kd = reinterpret_cast<uint4*>(Ku + (size_t)dst * D);
-    uint4* vd = reinterpret_cast<uint4*>(Vu + (size_t)dst * D);
-    for (int c = lane; c < 2 * kChunks; c += 32) {
-        if (c < kChunks) kd[c] = __ldcg(ks + c);
-        else vd[c - kChunks] = __ldcg(vs + (c - kChunks));
-    }
-    if (lane == 0) {
-        wordu[dst] = __ldcg(wordu + src);
-        posu[dst] = __ldcg(posu + src);
+// Hole filling: row movers[i] (K row, V row, register, position) is copied to slot holes[i], i < n_moved, by the whole
+// block. Sources lie at or above the new length, destinations below it, so copies never overlap. Each warp takes
+// four rows at a time and issues all their loads before the first store (the copies are latency-, not
+// bandwidth-limited). Rows are D*sizeof(T) bytes = a multiple of 16.
+template <typename T, int D, int NT>
+__device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, int32_t* posu, const int* movers,
+                                                const int* holes, int n_moved) {
+    constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = 4, NW = NT / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i0 = warp * kRows; i0 < n_moved; i0 += NW * kRows) {
+        int src[kRows], dst[kRows];
+        uint4 buf[kRows][kIter];
+        uint32_t wd = 0u;
+        int32_t ps = 0;
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            const bool on = i0 + r < n_moved;
+            src[r] = on ? movers[i0 + r] : -1;
+            dst[r] = on ? holes[i0 + r] : -1;
+        }
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            if (src[r] < 0) continue;
+#pragma unroll
+            for (int x = 0; x < kIter; ++x) {
+                const int c = lane + 32 * x;
+                if (c < kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Ku + (size_t)src[r] * D) + c);
+                else if (c < 2 * kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Vu + (size_t)src[r] * D) + (c - kChunks));
+            }
+            if (lane == r) { wd = __ldcg(wordu + src[r]); ps = __ldcg(posu + src[r]); }
+        }
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            if (src[r] < 0) continue;
+#pragma unroll
+            for (int x = 0; x < kIter; ++x) {
+                const int c = lane + 32 * x;
+                if (c < kChunks) reinterpret_cast<uint4*>(Ku + (size_t)dst[r] * D)[c] = buf[r][x];
+                else if (c < 2 * kChunks) reinterpret_cast<uint4*>(Vu + (size_t)dst[r] * D)[c - kChunks] = buf[r][x];
+            }
+            if (lane == r) { wordu[dst[r]] = wd; posu[dst[r]] = ps; }
+        }
     }
 }
 
@@ -287,8 +314,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            for (int i = warp; i < n_moved; i += NT / 32)
-                warp_move_row<T, D>(Ku, Vu, wordu, posu, movers[i], holes[i], lane);
+            block_move_rows<T, D, NT>(Ku, Vu, wordu, posu, movers, holes, n_moved);
         }
     }
     if (tid == 0) {

@@ -193,14 +193,12 @@ __device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double
 template <int G, int NT, int KPRE>
 __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int t, const double* thr,
                                 const double* stash_sm, int stash_ld, const uint32_t (&wv)[KPRE],
-                                const int32_t (&pv)[KPRE], unsigned char* lists) {
+                                const int32_t (&pv)[KPRE], unsigned char* lists, int* holes, int* movers) {
     __shared__ int s_scan1[NT];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cap_words = (l + 31) / 32 + 2;
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(lists);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
-    int* holes = prefix + cap_words;
-    int* movers = holes + l;
     bf16_t* Ku = reinterpret_cast<bf16_t*>(p.K) + (size_t)u * p.C * 128;
     bf16_t* Vu = reinterpret_cast<bf16_t*>(p.V) + (size_t)u * p.C * 128;
     uint32_t* wordu = p.word + (size_t)u * p.C;
@@ -240,8 +238,7 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            for (int i = warp; i < n_moved; i += NT / 32)
-                warp_move_row<bf16_t, 128>(Ku, Vu, wordu, posu, movers[i], holes[i], lane);
+            block_move_rows<bf16_t, 128, NT>(Ku, Vu, wordu, posu, movers, holes, n_moved);
         }
     }
     if (tid == 0) {
@@ -512,7 +509,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     }
     if (single) {
         __syncthreads();
-        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, merge + NW * G * kRec);
+        unsigned char* lists = merge + NW * G * kRec;
+        int* holes = reinterpret_cast<int*>(lists + 2 * ((l + 31) / 32 + 2) * 4);
+        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l);
         return;
     }
     __threadfence();
