@@ -161,8 +161,6 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=512)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "stream", "split"],
-                    help="bf16/d128 decode kernel: persistent streaming or one block per split (auto = library default)")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -195,8 +193,7 @@ def main():
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
                       cfg.recent_r, cfg.alpha, cfg.dtype, local)
-    mode = 0 if args.no_fast else {"auto": 1, "stream": 1, "split": 2}[args.kernel]
-    cache.corm_cache_set_tuning(args.split_len, mode)
+    cache.corm_cache_set_tuning(args.split_len, not args.no_fast)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
     prompt_ms = 0.0

@@ -152,8 +152,7 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
                                       void* stream);
 
 /* Tuning knobs (performance only; results do not depend on them): keys per split of the decode kernel
- * (multiple of 32, 0 = automatic) and which kernel serves bf16 / head_dim-128 caches: 0 = the generic kernel,
- * 1 = the persistent streaming kernel (default), 2 = the one-block-per-split kernel. */
+ * (multiple of 32, 0 = automatic) and whether the fast bf16/head_dim-128 kernel may be used. */
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Number of kernels this library has launched on behalf of `cache` since create. */

@@ -196,7 +196,6 @@ class CormCache:
         return out
 
     def corm_cache_set_tuning(self, split_len=0, allow_fast_path=True):
-        """allow_fast_path: False/0 generic kernel, True/1 streaming kernel (default), 2 one-block-per-split kernel."""
         _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
 
     def corm_cache_kernel_launches(self):

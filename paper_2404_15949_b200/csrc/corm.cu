@@ -15,7 +15,6 @@
 #include "corm_common.cuh"
 #include "corm_fast.cuh"
 #include "corm_generic.cuh"
-#include "corm_stream.cuh"
 
 using namespace corm;
 
@@ -27,7 +26,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, queue, stash, partials;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -71,7 +70,6 @@ Layout make_layout(const corm_config_t& c) {
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
-    L.queue = take(8);
     L.bookkeeping_end = off;
     L.stash = take(U * G * C * 8);
     L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
@@ -191,7 +189,6 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
     p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
     p.maxlive = maxlive_ptr(c, layer);
-    p.queue = reinterpret_cast<uint32_t*>(c->arena + c->lay.queue);
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.partials = c->arena + c->lay.partials;
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
@@ -203,8 +200,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
     if (fast) {
-        rc = c->allow_fast == 2 ? launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st)
-                                : launch_decode_stream(p, c->G, upper, c->tune_split_len, c->sm_count, st);
+        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st);
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
         const int n_splits = (upper + p.split_len - 1) / p.split_len;
@@ -595,7 +591,7 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
 corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
-    c->allow_fast = allow_fast_path < 0 ? 0 : (allow_fast_path > 2 ? 2 : allow_fast_path);
+    c->allow_fast = allow_fast_path ? 1 : 0;
     return CORM_OK;
 }
 

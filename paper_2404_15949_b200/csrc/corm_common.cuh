@@ -34,8 +34,6 @@ struct DecodeParams {
     void* out;                // [B][Hq][D]
     int32_t U, Hkv, C, split_len, max_splits, step, w, r;
     int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
-    int32_t n_splits;         // streaming kernel: work items are (unit, split) pairs, split < n_splits
-    uint32_t* queue;          // streaming kernel: {next work item, finished blocks}, both zero between launches
     double log_alpha;         // ln(alpha), -inf for alpha = 0
 };
 

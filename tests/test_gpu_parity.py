@@ -48,8 +48,6 @@ SMALL = [
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, False),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, False),
-    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, 2),      # 2 = one-block-per-split kernel
-    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, 2),
     ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True),
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 64, True),
     ("bf16", 64, 4, 2, 2, (100, 200), 24, 8, 16, 64, True),
