@@ -15,6 +15,7 @@
 #include "corm_common.cuh"
 #include "corm_fast.cuh"
 #include "corm_generic.cuh"
+#include "corm_prompt_fast.cuh"
 
 using namespace corm;
 
@@ -351,18 +352,32 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.p_max = p_max; p.w = cf.window_w; p.r = cf.recent_r;
     p.log_alpha = log_alpha_of(c);
-    corm_status_t rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
-        using T = std::remove_pointer_t<decltype(tp)>;
-        constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
-        const size_t smem = prompt_smem(GG, cf.window_w, cf.max_tokens);
-        auto kern = prompt_generic_kernel<T, DD, GG>;
-        if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        kern<<<(unsigned)U, kPromptThreads, smem, st>>>(p);
-        CORM_CUDA(cudaGetLastError());
-        return CORM_OK;
-    });
+    corm_status_t rc = CORM_ERR_UNSUPPORTED;
+    int n_launched = 1;
+    if (cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->allow_fast) {     // two-launch tiled pass
+        PromptFastParams fp{};
+        fp.p = p;
+        fp.partials = c->arena + c->lay.partials;
+        fp.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
+        const size_t cap = U * (size_t)max_splits_of(cf) * c->G * partial_stride((int)D);
+        rc = launch_prompt_fast(fp, c->G, max_p, c->sm_count, cap, st);
+        n_launched = 2;
+    }
+    if (rc == CORM_ERR_UNSUPPORTED) {
+        n_launched = 1;
+        rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
+            using T = std::remove_pointer_t<decltype(tp)>;
+            constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
+            const size_t smem = prompt_smem(GG, cf.window_w, cf.max_tokens);
+            auto kern = prompt_generic_kernel<T, DD, GG>;
+            if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            kern<<<(unsigned)U, kPromptThreads, smem, st>>>(p);
+            CORM_CUDA(cudaGetLastError());
+            return CORM_OK;
+        });
+    }
     if (rc != CORM_OK) return rc;
-    c->launches += 1;
+    c->launches += n_launched;
     c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p;
     c->last_readback_step[layer] = 0;
     schedule_live_readback(c, layer, st);

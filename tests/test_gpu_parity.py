@@ -126,7 +126,7 @@ def test_multi_layer_independent_and_deterministic():
             sa = sorted_state(gpu.corm_cache_export_state(l, 0, h))
             sb = sorted_state(gpu2.corm_cache_export_state(l, 0, h))
             assert all(np.array_equal(sa[k], sb[k]) for k in ("k", "v", "word", "pos"))
-    assert gpu.corm_cache_kernel_launches() == 3 + 3 * cfg.steps
+    assert gpu.corm_cache_kernel_launches() == 2 * 3 + 3 * cfg.steps        # two launches per prompt pass, one per step
 
 
 def test_host_buffer_entry_point_matches_device_one():
