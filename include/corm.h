@@ -88,7 +88,8 @@ corm_status_t corm_cache_reset(corm_cache_t* cache, void* stream);
  *   q_last              device [batch, n_q_heads, window_w, head_dim]: queries of positions P-w+1..P, oldest
  *                       first; for P < w the first w-P rows are ignored
  *   prompt_lens_host    host [batch], 0 <= P_b <= min(p_max, max_tokens); P_b = 0 leaves the unit empty
- * Survivors are written to the slabs in token order. Produces no attention output. */
+ * Survivors are written to the slabs in token order. Produces no attention output. Whatever the layer held
+ * before is replaced and its counters (corm_cache_stats) restart. */
 corm_status_t corm_compress_prompt(corm_cache_t* cache, int32_t layer, const void* k_prompt, const void* v_prompt,
                                    const void* q_last, const int32_t* prompt_lens_host, int32_t p_max,
                                    void* stream);

@@ -337,6 +337,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     CORM_CUDA(cudaMemcpyAsync(base_obs, obs.data(), (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket, U * 4, layer), 0, U * 4, st));
     CORM_CUDA(cudaMemsetAsync(maxlive_ptr(c, layer), 0, 8, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer), 0, CNT_COUNT * 8, st));   // a new prompt restarts the layer's statistics
     c->readback_pending[layer] = 0;   // an older read-back no longer describes this layer
     PromptParams p{};
     p.k_prompt = k_prompt; p.v_prompt = v_prompt; p.q_last = q_last;
