@@ -77,6 +77,14 @@ class LiteralUnit:
                 verdict[:i] |= attn >= self.alpha / i           # keys newer than the query keep a 0 bit
             self._record_and_evict(verdict)                     # evicts only once w rows exist: at the last row
 
+    def ages(self):
+        """Per cached key: how many recorded queries ago it was last found important (0 = latest), -1 if never."""
+        m, l = self.message.shape
+        out = np.full((l,), -1, dtype=np.int32)
+        for b in range(m - 1, -1, -1):                    # oldest candidate first, newest overwrites
+            out[self.message[m - 1 - b]] = b
+        return out
+
     def words(self):
         """Shift-register view of the message: bit b = verdict of the query b steps ago."""
         m, l = self.message.shape

@@ -17,8 +17,8 @@
  * It shares no code with the CUDA library and never calls it.
  *
  * The recent-w verdict rows of Algorithm 1 (a bool matrix [m, l]) are held here as one w-bit shift register per
- * key: bit b of a key's word is the verdict of the query b steps ago. A literal bool-matrix version lives in
- * alg1_literal.py and is tested equal to this one.
+ * key (REG_WORDS 32-bit words, w <= 256): bit b of a key's register is the verdict of the query b steps ago. A
+ * literal bool-matrix version lives in alg1_literal.py and is tested equal to this one.
  *
  * Every function below is pinned by tests/test_oracle_pins.py (hand-worked cases, full attention at alpha=0,
  * brute force over subsets, closed forms, invariants); none is "parity unpinned".
@@ -36,7 +36,7 @@ typedef struct {
     double alpha;
     int     *live;   /* [L*B*Hkv]            live entries per unit            */
     int     *pos;    /* [L*B*Hkv][C]         absolute 1-based token position  */
-    uint32_t *word;  /* [L*B*Hkv][C]         w-bit verdict register           */
+    uint32_t *word;  /* [L*B*Hkv][C][REG_WORDS] w-bit verdict register (word 0 = newest 32 verdicts) */
     double  *k, *v;  /* [L*B*Hkv][C][d]                                       */
     int     *t;      /* [L*B]                tokens seen                      */
     int     *n_obs;  /* [L*B]                verdict rows recorded            */
@@ -45,6 +45,7 @@ typedef struct {
 } corm_oracle;
 
 enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1, ORACLE_CAPACITY = 6 };
+enum { REG_WORDS = 8, MAX_WINDOW = 32 * REG_WORDS };
 
 static size_t unit_index(const corm_oracle *o, int layer, int b, int h) {
     return ((size_t)layer * o->batch + b) * o->n_kv_heads + h;
@@ -53,7 +54,7 @@ static size_t unit_index(const corm_oracle *o, int layer, int b, int h) {
 corm_oracle *oracle_create(int n_layers, int batch, int n_q_heads, int n_kv_heads, int head_dim, int max_tokens,
                            int w, int r, double alpha) {
     if (n_layers < 1 || batch < 1 || n_kv_heads < 1 || n_q_heads < 1 || n_q_heads % n_kv_heads) return NULL;
-    if (head_dim < 1 || max_tokens < 1 || w < 1 || w > 32 || r < 1 || !(alpha >= 0.0)) return NULL;
+    if (head_dim < 1 || max_tokens < 1 || w < 1 || w > MAX_WINDOW || r < 1 || !(alpha >= 0.0)) return NULL;
     corm_oracle *o = (corm_oracle *)calloc(1, sizeof(corm_oracle));
     if (!o) return NULL;
     o->n_layers = n_layers; o->batch = batch; o->n_q_heads = n_q_heads; o->n_kv_heads = n_kv_heads;
@@ -62,7 +63,7 @@ corm_oracle *oracle_create(int n_layers, int batch, int n_q_heads, int n_kv_head
     size_t units = (size_t)n_layers * batch * n_kv_heads, C = (size_t)max_tokens, d = (size_t)head_dim;
     o->live = (int *)calloc(units, sizeof(int));
     o->pos = (int *)calloc(units * C, sizeof(int));
-    o->word = (uint32_t *)calloc(units * C, sizeof(uint32_t));
+    o->word = (uint32_t *)calloc(units * C * REG_WORDS, sizeof(uint32_t));
     o->k = (double *)calloc(units * C * d, sizeof(double));
     o->v = (double *)calloc(units * C * d, sizeof(double));
     o->t = (int *)calloc((size_t)n_layers * batch, sizeof(int));
@@ -76,7 +77,25 @@ void oracle_destroy(corm_oracle *o) {
     free(o->live); free(o->pos); free(o->word); free(o->k); free(o->v); free(o->t); free(o->n_obs); free(o);
 }
 
-static uint32_t window_mask(int w) { return w >= 32 ? 0xffffffffu : ((1u << w) - 1u); }
+/* register helpers: shift the newest verdict in at bit 0 and drop everything older than w verdicts */
+static void reg_shift_in(uint32_t *reg, int w, uint32_t bit) {
+    uint32_t carry = bit & 1u;
+    for (int i = 0; i < REG_WORDS; ++i) {
+        uint32_t next = reg[i] >> 31;
+        reg[i] = (reg[i] << 1) | carry;
+        carry = next;
+    }
+    for (int i = 0; i < REG_WORDS; ++i) {            /* keep bits [0, w) */
+        int lo = 32 * i;
+        if (w <= lo) reg[i] = 0u;
+        else if (w < lo + 32) reg[i] &= (1u << (w - lo)) - 1u;
+    }
+}
+static int reg_nonzero(const uint32_t *reg) {
+    for (int i = 0; i < REG_WORDS; ++i) if (reg[i]) return 1;
+    return 0;
+}
+static void reg_clear(uint32_t *reg) { memset(reg, 0, REG_WORDS * sizeof(uint32_t)); }
 
 /* Algorithm 1, the part after the message update: once w rows are recorded, a key stays iff some recent query
  * found it important (any over the window) or it is one of the r most recent tokens; survivors keep their order
@@ -87,11 +106,11 @@ static int evict_unit(corm_oracle *o, size_t u, int t, int n_obs) {
     size_t C = (size_t)o->max_tokens, d = (size_t)o->head_dim;
     int l = o->live[u], kept = 0;
     for (int j = 0; j < l; ++j) {
-        int keep = (o->word[u * C + j] != 0u) || (o->pos[u * C + j] > t - o->r);
+        int keep = reg_nonzero(o->word + (u * C + j) * REG_WORDS) || (o->pos[u * C + j] > t - o->r);
         if (!keep) continue;
         if (kept != j) {
             o->pos[u * C + kept] = o->pos[u * C + j];
-            o->word[u * C + kept] = o->word[u * C + j];
+            memcpy(o->word + (u * C + kept) * REG_WORDS, o->word + (u * C + j) * REG_WORDS, REG_WORDS * sizeof(uint32_t));
             memcpy(o->k + (u * C + kept) * d, o->k + (u * C + j) * d, d * sizeof(double));
             memcpy(o->v + (u * C + kept) * d, o->v + (u * C + j) * d, d * sizeof(double));
         }
@@ -159,7 +178,7 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
                 o->v[(u * C + l) * d + c] = (double)v_new[((size_t)b * Hkv + h) * d + c];
             }
             o->pos[u * C + l] = t;
-            o->word[u * C + l] = 0u;
+            reg_clear(o->word + (u * C + l) * REG_WORDS);
             l += 1;
             o->live[u] = l;
             ++appended;
@@ -179,9 +198,8 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
                 for (int j = 0; j < l; ++j)                           /* group rule: OR over the query heads */
                     if (important(o, p[j], t, &evals, &near)) imp[j] = 1;
             }
-            uint32_t mask = window_mask(o->w);
             for (int j = 0; j < l; ++j) {                             /* newest verdict enters at bit 0 */
-                o->word[u * C + j] = ((o->word[u * C + j] << 1) | (uint32_t)imp[j]) & mask;
+                reg_shift_in(o->word + (u * C + j) * REG_WORDS, o->w, (uint32_t)imp[j]);
                 if (imp_out) imp_out[((size_t)b * Hkv + h) * C + j] = imp[j];
             }
             evals_total += evals; near_total += near;
@@ -230,7 +248,7 @@ int oracle_compress_prompt(corm_oracle *o, int layer, const float *k_prompt, con
                     o->v[(u * C + j) * d + c] = (double)v_prompt[src + c];
                 }
                 o->pos[u * C + j] = j + 1;
-                o->word[u * C + j] = 0u;
+                reg_clear(o->word + (u * C + j) * REG_WORDS);
             }
             o->live[u] = P;
             appended += P;
@@ -238,7 +256,6 @@ int oracle_compress_prompt(corm_oracle *o, int layer, const float *k_prompt, con
             double *p = (double *)malloc((size_t)P * sizeof(double));
             double *qv = (double *)malloc((size_t)d * sizeof(double));
             unsigned char *imp = (unsigned char *)malloc((size_t)P);
-            uint32_t mask = window_mask(w);
             long long evals = 0, near = 0;
             for (int row = w - wp; row < w; ++row) {
                 int i = P - (w - 1 - row);                            /* absolute position of this query */
@@ -250,8 +267,7 @@ int oracle_compress_prompt(corm_oracle *o, int layer, const float *k_prompt, con
                     for (int j = 0; j < i; ++j)                       /* slot j holds position j+1 here */
                         if (important(o, p[j], i, &evals, &near)) imp[j] = 1;
                 }
-                for (int j = 0; j < P; ++j)
-                    o->word[u * C + j] = ((o->word[u * C + j] << 1) | (uint32_t)imp[j]) & mask;
+                for (int j = 0; j < P; ++j) reg_shift_in(o->word + (u * C + j) * REG_WORDS, w, (uint32_t)imp[j]);
             }
             free(p); free(qv); free(imp);
             evals_total += evals; near_total += near;
@@ -281,7 +297,7 @@ int oracle_export_unit(const corm_oracle *o, int layer, int b, int h, double *k,
     int l = o->live[u];
     if (k) memcpy(k, o->k + u * C * d, (size_t)l * d * sizeof(double));
     if (v) memcpy(v, o->v + u * C * d, (size_t)l * d * sizeof(double));
-    if (word) memcpy(word, o->word + u * C, (size_t)l * sizeof(uint32_t));
+    if (word) for (int j = 0; j < l; ++j) word[j] = o->word[(u * C + j) * REG_WORDS];   /* newest 32 verdicts */
     if (pos) memcpy(pos, o->pos + u * C, (size_t)l * sizeof(int));
     return l;
 }
@@ -293,12 +309,26 @@ int oracle_import_unit(corm_oracle *o, int layer, int b, int h, int live, const 
     size_t u = unit_index(o, layer, b, h), C = (size_t)o->max_tokens, d = (size_t)o->head_dim;
     memcpy(o->k + u * C * d, k, (size_t)live * d * sizeof(double));
     memcpy(o->v + u * C * d, v, (size_t)live * d * sizeof(double));
-    memcpy(o->word + u * C, word, (size_t)live * sizeof(uint32_t));
+    for (int j = 0; j < live; ++j) { reg_clear(o->word + (u * C + j) * REG_WORDS); o->word[(u * C + j) * REG_WORDS] = word[j]; }
     memcpy(o->pos + u * C, pos, (size_t)live * sizeof(int));
     o->live[u] = live;
     o->t[(size_t)layer * o->batch + b] = n_tokens;
     o->n_obs[(size_t)layer * o->batch + b] = n_obs;
     return ORACLE_OK;
+}
+
+/* For each live entry: how many queries ago it was last judged important (0 = by the latest query), -1 if by none
+ * of the last w. This is all of the register that can still influence an eviction. */
+int oracle_export_age(const corm_oracle *o, int layer, int b, int h, int *age) {
+    size_t u = unit_index(o, layer, b, h), C = (size_t)o->max_tokens;
+    int l = o->live[u];
+    for (int j = 0; j < l; ++j) {
+        const uint32_t *reg = o->word + (u * C + j) * REG_WORDS;
+        age[j] = -1;
+        for (int bit = 0; bit < o->w && age[j] < 0; ++bit)
+            if ((reg[bit >> 5] >> (bit & 31)) & 1u) age[j] = bit;
+    }
+    return l;
 }
 
 void oracle_counters(const corm_oracle *o, long long *appended, long long *evicted, long long *verdict_evals,

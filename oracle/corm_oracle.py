@@ -47,6 +47,8 @@ def _load():
     lib.oracle_export_unit.argtypes = [vp, c_int, c_int, c_int, vp, vp, vp, vp]
     lib.oracle_import_unit.restype = c_int
     lib.oracle_import_unit.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp, vp, vp, c_int, c_int]
+    lib.oracle_export_age.restype = c_int
+    lib.oracle_export_age.argtypes = [vp, c_int, c_int, c_int, vp]
     lib.oracle_counters.argtypes = [vp, vp, vp, vp, vp]
     lib.oracle_set_near_band.argtypes = [vp, c_dbl]
     _lib = lib
@@ -125,7 +127,9 @@ class CormOracle:
         pos = np.empty((l,), dtype=np.int32)
         self.lib.oracle_export_unit(self.h, layer, b, h, k.ctypes.data, v.ctypes.data, word.ctypes.data,
                                     pos.ctypes.data)
-        return dict(k=k, v=v, word=word, pos=pos, live_len=l, n_tokens=self.n_tokens(layer, b),
+        age = np.empty((l,), dtype=np.int32)
+        self.lib.oracle_export_age(self.h, layer, b, h, age.ctypes.data)
+        return dict(k=k, v=v, word=word, pos=pos, age=age, live_len=l, n_tokens=self.n_tokens(layer, b),
                     n_obs=self.n_obs(layer, b))
 
     def import_unit(self, layer, b, h, k, v, word, pos, n_tokens, n_obs):

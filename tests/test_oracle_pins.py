@@ -154,6 +154,33 @@ def test_shift_register_equals_literal_algorithm(seed):
                 assert np.allclose(out[b, h * G:(h + 1) * G], ref, rtol=1e-12, atol=1e-13)
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_wide_windows_equal_literal_algorithm(seed):
+    """Windows beyond 32 queries (the paper's experiments use up to 256): multi-word registers against the literal
+    bool-matrix routine, compared through the live lists and the age of each key's newest 'important' verdict."""
+    rng = np.random.default_rng(3000 + seed)
+    G = int(rng.integers(1, 3))
+    d, w, r = 3, int(rng.choice([33, 40, 64, 65, 100])), int(rng.integers(1, 20))
+    P, steps = int(rng.integers(0, 150)), int(rng.integers(40, 90))
+    k, v, q, _ = _random_case(rng, 1, G, 1, d, P, steps, w, scale=2.5)
+    o = CormOracle(1, 1, G, 1, d, P + steps, w, r, 1.0)
+    u = LiteralUnit(d, w, r, 1.0)
+    u.compress_prompt(k[0, 0, :P], v[0, 0, :P], q[0, :, :w])
+    o.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], [P])
+    evicted = False
+    for s in range(steps + 1):
+        st = o.export_unit(0, 0, 0)
+        assert st["pos"].tolist() == u.pos.tolist(), s
+        assert st["age"].tolist() == u.ages().tolist(), s
+        if s == steps:
+            break
+        out = o.decode_step(0, q[:, :, w + s], k[:, :, P + s], v[:, :, P + s])
+        ref = u.decode_step(q[0, :, w + s], k[0, 0, P + s], v[0, 0, P + s])
+        assert np.allclose(out[0], ref, rtol=1e-12, atol=1e-13)
+        evicted |= o.live_len(0, 0, 0) < P + s + 1
+    assert evicted or P + steps < w
+
+
 @pytest.mark.parametrize("seed", range(8))
 def test_bruteforce_eviction_sets(seed):
     """t <= 16: verdicts recomputed with a library softmax, and the kept set identified by enumerating all subsets of
