@@ -9,8 +9,10 @@
  * it (Section 5, "Integrate into grouped-query attention").
  *
  * A "unit" is one (layer, sequence, kv head). Each unit owns a slab of max_tokens slots holding K rows, V rows,
- * one w-bit verdict register per key (bit b = verdict of the query b steps ago) and the key's absolute 1-based
- * token position. Live entries occupy slots [0, live_len); their slot ORDER IS NOT the token order once decode
+ * one 32-bit verdict register per key and the key's absolute 1-based token position. Register encodings: for
+ * window_w <= 32 a shift register (bit b = verdict of the query b steps ago); for 33..256 (the paper's experiments
+ * use up to 256) the absolute step of the latest query that found the key important, 0 if none has, which decides
+ * Algorithm 1's any() over the last w rows as step_now - register < w. Live entries occupy slots [0, live_len); their slot ORDER IS NOT the token order once decode
  * steps have evicted keys (holes are filled from the tail), so recency is always decided from the stored position.
  *
  * Conventions
@@ -51,7 +53,7 @@ typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group size in {1,2,4,8} */
     int32_t head_dim;                                /* 64 or 128 */
     int32_t max_tokens;                              /* slab capacity per unit: >= longest prompt + decode steps */
-    int32_t window_w;                                /* 1..32: one 32-bit register per key */
+    int32_t window_w;                                /* 1..256 recent queries; see the register encodings below */
     int32_t recent_r;                                /* >= 1 (Algorithm 1's slice of the last r entries) */
     float   alpha;                                   /* >= 0; threshold alpha/t; 0 means nothing is ever evicted */
     int32_t kv_dtype;                                /* corm_dtype_t */
@@ -72,7 +74,7 @@ size_t corm_cache_arena_bytes(const corm_config_t* cfg);
 
 /* Builds the host object over a caller-allocated device arena (256-byte aligned, >= corm_cache_arena_bytes) and
  * zeroes the bookkeeping part of the arena on the legacy default stream, synchronously.
- * Errors: INVALID_ARG (null/invalid fields), UNSUPPORTED (head_dim, group, w > 32), ARENA_TOO_SMALL, CUDA. */
+ * Errors: INVALID_ARG (null/invalid fields), UNSUPPORTED (head_dim, group, w > 256), ARENA_TOO_SMALL, CUDA. */
 corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, size_t arena_bytes,
                                 corm_cache_t** out);
 corm_status_t corm_cache_destroy(corm_cache_t* cache);

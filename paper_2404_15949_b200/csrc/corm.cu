@@ -44,7 +44,7 @@ bool config_ok(const corm_config_t* c, corm_status_t* why) {
     const int G = c->n_q_heads / c->n_kv_heads;
     if (c->head_dim != 64 && c->head_dim != 128) return false;
     if (G != 1 && G != 2 && G != 4 && G != 8) return false;
-    if (c->window_w > 32) return false;
+    if (c->window_w > 256) return false;
     if ((long long)c->batch * c->n_kv_heads > 65535) return false;     // grid.y of the decode kernel
     if (c->max_tokens > (1 << 22)) return false;
     *why = CORM_OK;
@@ -362,7 +362,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
         fp.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
         const size_t cap = U * (size_t)max_splits_of(cf) * c->G * partial_stride((int)D);
         rc = launch_prompt_fast(fp, c->G, max_p, c->sm_count, cap, st);
-        n_launched = 2;
+        n_launched = prompt_fast_launches(c->G, cf.window_w);
     }
     if (rc == CORM_ERR_UNSUPPORTED) {
         n_launched = 1;

@@ -116,6 +116,17 @@ __device__ __forceinline__ void publish_live(unsigned long long* maxlive, int st
 
 __device__ __forceinline__ uint32_t window_mask(int w) { return w >= 32 ? 0xffffffffu : ((1u << w) - 1u); }
 
+// The per-key 32-bit register has two encodings. Windows of up to 32 queries: a shift register, bit b = verdict of
+// the query b steps ago (Algorithm 1's message column). Wider windows (the paper runs up to 256): the step t of the
+// latest query that found the key important, 0 if none has; "some query among the last w found it important" is
+// then t_now - stamp < w, which selects exactly the columns Algorithm 1's any() over the last w rows selects.
+__device__ __forceinline__ uint32_t update_register(uint32_t old, bool imp, int w, int t) {
+    return w <= 32 ? (((old << 1) | (imp ? 1u : 0u)) & window_mask(w)) : (imp ? (uint32_t)t : old);
+}
+__device__ __forceinline__ bool register_needed(uint32_t reg, int w, int t) {
+    return w <= 32 ? reg != 0u : (reg != 0u && t - (int)reg < w);
+}
+
 // Exclusive prefix sums of popc(mask[i]) into prefix[0..nwords], block-wide. scratch holds NT ints.
 // Each thread sums a contiguous run of words; warp 0 scans the NT run totals with shuffles.
 template <int NT>
@@ -256,7 +267,6 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     // 2. verdicts, register update, keep flags
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
     const bool evict_on = n_obs >= p.w;
-    const uint32_t wmask = window_mask(p.w);
     const double* stash_u = p.stash + (size_t)u * G * p.C;
     constexpr int kBatch = (G >= 4 ? 4 : 8);                                      // slots per thread whose loads are issued together
     for (int base0 = 0; base0 < l; base0 += kBatch * NT) {
@@ -285,9 +295,9 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 bool imp = false;
 #pragma unroll
                 for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
-                const uint32_t wd = ((wv[k] << 1) | (imp ? 1u : 0u)) & wmask;
+                const uint32_t wd = update_register(wv[k], imp, p.w, t);
                 wordu[j] = wd;
-                keep = !evict_on || wd != 0u || pv[k] > t - p.r;
+                keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
             }
             const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
             if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;

@@ -205,7 +205,6 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     int32_t* posu = p.pos + (size_t)u * p.C;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
     const bool evict_on = n_obs >= p.w;
-    const uint32_t wmask = window_mask(p.w);
 #pragma unroll
     for (int k = 0; k < KPRE; ++k) {
         const int base = k * NT, j = base + tid;
@@ -215,9 +214,9 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
             bool imp = false;
 #pragma unroll
             for (int g = 0; g < G; ++g) imp |= (stash_sm[g * stash_ld + j] >= thr[g]);
-            const uint32_t wd = ((wv[k] << 1) | (imp ? 1u : 0u)) & wmask;
+            const uint32_t wd = update_register(wv[k], imp, p.w, t);
             wordu[j] = wd;
-            keep = !evict_on || wd != 0u || pv[k] > t - p.r;
+            keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
         }
         const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
         if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;

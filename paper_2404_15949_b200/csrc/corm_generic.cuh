@@ -136,8 +136,11 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     finalize_unit<T, D, G, NT>(p, u, b, l, n_act, t, smem);
 }
 
+// window slots handled per pass of the generic prompt kernel (at most 64 (slot, head) rows at a time)
+__host__ __device__ inline int prompt_chunk_slots(int G, int w) { const int s = 64 / G; return s < w ? s : w; }
+
 __host__ __device__ inline size_t prompt_smem(int G, int w, int C) {
-    const size_t warps = kPromptThreads / 32, rows = (size_t)G * w;
+    const size_t warps = kPromptThreads / 32, rows = (size_t)G * prompt_chunk_slots(G, w);
     size_t a = warps * rows * 16 + rows * 8;
     size_t b = (size_t)2 * ((C + 31) / 32 + 2) * 4;
     return a + b;
@@ -158,8 +161,9 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
         return;
     }
     if (P == 0) { if (tid == 0) p.live_out[u] = 0; return; }
-    const int w = p.w, wp = min(P, w), rows = G * w;
-    double* sm_mz = reinterpret_cast<double*>(smem);                   // [NW][rows][2]
+    const int w = p.w, wp = min(P, w);
+    const int cs = prompt_chunk_slots(G, w), rows = G * cs;           // window slots per pass, rows per pass
+    double* sm_mz = reinterpret_cast<double*>(smem);                   // [NW][rows][2], row = g * cs + (slot - slot0)
     double* sm_thr = sm_mz + (size_t)NW * rows * 2;                    // [rows]
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(sm_thr + rows);
     int* prefix = reinterpret_cast<int*>(keepmask + (p.C + 31) / 32 + 2);
@@ -168,54 +172,20 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     const T* Q = reinterpret_cast<const T*>(p.q_last) + (size_t)u * G * w * D;   // [G][w][D]
     const int c0 = lane * NPL;
     const double root_d = sqrt((double)D);
-
-    for (int i = tid; i < NW * rows; i += NT) { sm_mz[2 * i] = -INFINITY; sm_mz[2 * i + 1] = 0.0; }
-    __syncthreads();
-    // pass 1: running max / sum of every row, per warp (only lane 0 owns the warp's entries)
-    for (int j = warp; j < P; j += NW) {
-        float kf[NPL];
-        load_slice<T, NPL>(Kp + (size_t)j * D + c0, kf);
-        for (int row = w - wp; row < w; ++row) {
-            const int i = P - (w - 1 - row);          // position of this query; it sees keys 1..i
-            if (j + 1 > i) continue;
-            for (int g = 0; g < G; ++g) {
-                float qf[NPL];
-                load_slice<T, NPL>(Q + ((size_t)g * w + row) * D + c0, qf);
-                double part = 0.0;
-#pragma unroll
-                for (int k = 0; k < NPL; ++k) part += (double)qf[k] * (double)kf[k];
-                const double s = warp_sum(part) / root_d;
-                if (lane == 0) {
-                    double* mz = sm_mz + ((size_t)warp * rows + g * w + row) * 2;
-                    if (s > mz[0]) { mz[1] = mz[1] * exp(mz[0] - s) + 1.0; mz[0] = s; }
-                    else mz[1] += exp(s - mz[0]);
-                }
-            }
-        }
-    }
-    __syncthreads();
-    for (int rr = tid; rr < rows; rr += NT) {
-        const int row = rr % w;
-        if (row < w - wp) { sm_thr[rr] = INFINITY; continue; }
-        double M = -INFINITY, Z = 0.0;
-        for (int x = 0; x < NW; ++x) M = fmax(M, sm_mz[((size_t)x * rows + rr) * 2]);
-        for (int x = 0; x < NW; ++x)
-            Z += sm_mz[((size_t)x * rows + rr) * 2 + 1] * exp(sm_mz[((size_t)x * rows + rr) * 2] - M);
-        const int i = P - (w - 1 - row);
-        sm_thr[rr] = M + log(Z) + p.log_alpha - log((double)i);      // Definition 3.1 in log form, threshold alpha/i
-    }
-    __syncthreads();
-    // pass 2: registers (oldest recorded row ends in the highest bit, the query at position P in bit 0)
     uint32_t* tmp_word = reinterpret_cast<uint32_t*>(p.stash + (size_t)u * G * p.C);
-    const uint32_t wmask = window_mask(w);
-    for (int j = warp; j < P; j += NW) {
-        float kf[NPL];
-        load_slice<T, NPL>(Kp + (size_t)j * D + c0, kf);
-        uint32_t wd = 0u;
-        for (int row = w - wp; row < w; ++row) {
-            const int i = P - (w - 1 - row);
-            uint32_t bit = 0u;
-            if (j + 1 <= i) {
+
+    // the recorded queries are taken oldest first, a few window slots per pass over the keys
+    for (int slot0 = w - wp; slot0 < w; slot0 += cs) {
+        const int slot1 = min(w, slot0 + cs);
+        for (int i = tid; i < NW * rows; i += NT) { sm_mz[2 * i] = -INFINITY; sm_mz[2 * i + 1] = 0.0; }
+        __syncthreads();
+        // pass 1: running max / sum of every row, per warp (only lane 0 owns the warp's entries)
+        for (int j = warp; j < P; j += NW) {
+            float kf[NPL];
+            load_slice<T, NPL>(Kp + (size_t)j * D + c0, kf);
+            for (int row = slot0; row < slot1; ++row) {
+                const int i = P - (w - 1 - row);          // position of this query; it sees keys 1..i
+                if (j + 1 > i) continue;
                 for (int g = 0; g < G; ++g) {
                     float qf[NPL];
                     load_slice<T, NPL>(Q + ((size_t)g * w + row) * D + c0, qf);
@@ -223,19 +193,57 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
 #pragma unroll
                     for (int k = 0; k < NPL; ++k) part += (double)qf[k] * (double)kf[k];
                     const double s = warp_sum(part) / root_d;
-                    bit |= (s >= sm_thr[g * w + row]) ? 1u : 0u;
+                    if (lane == 0) {
+                        double* mz = sm_mz + ((size_t)warp * rows + g * cs + (row - slot0)) * 2;
+                        if (s > mz[0]) { mz[1] = mz[1] * exp(mz[0] - s) + 1.0; mz[0] = s; }
+                        else mz[1] += exp(s - mz[0]);
+                    }
                 }
             }
-            wd = ((wd << 1) | bit) & wmask;
         }
-        if (lane == 0) tmp_word[j] = wd;
+        __syncthreads();
+        for (int rr = tid; rr < rows; rr += NT) {
+            const int row = slot0 + rr % cs;
+            if (row >= slot1) { sm_thr[rr] = INFINITY; continue; }
+            double M = -INFINITY, Z = 0.0;
+            for (int x = 0; x < NW; ++x) M = fmax(M, sm_mz[((size_t)x * rows + rr) * 2]);
+            for (int x = 0; x < NW; ++x)
+                Z += sm_mz[((size_t)x * rows + rr) * 2 + 1] * exp(sm_mz[((size_t)x * rows + rr) * 2] - M);
+            const int i = P - (w - 1 - row);
+            sm_thr[rr] = M + log(Z) + p.log_alpha - log((double)i);  // Definition 3.1 in log form, threshold alpha/i
+        }
+        __syncthreads();
+        // pass 2: verdicts of these queries enter the registers (shift register: the query at position P ends in
+        // bit 0; wide windows: the position of the newest query that found the key important)
+        for (int j = warp; j < P; j += NW) {
+            float kf[NPL];
+            load_slice<T, NPL>(Kp + (size_t)j * D + c0, kf);
+            uint32_t wd = slot0 == w - wp ? 0u : tmp_word[j];          // written by this same thread in the previous pass
+            for (int row = slot0; row < slot1; ++row) {
+                const int i = P - (w - 1 - row);
+                bool bit = false;
+                if (j + 1 <= i) {
+                    for (int g = 0; g < G; ++g) {
+                        float qf[NPL];
+                        load_slice<T, NPL>(Q + ((size_t)g * w + row) * D + c0, qf);
+                        double part = 0.0;
+#pragma unroll
+                        for (int k = 0; k < NPL; ++k) part += (double)qf[k] * (double)kf[k];
+                        const double s = warp_sum(part) / root_d;
+                        bit |= (s >= sm_thr[g * cs + (row - slot0)]);
+                    }
+                }
+                wd = update_register(wd, bit, w, i);
+            }
+            if (lane == 0) tmp_word[j] = wd;
+        }
+        __syncthreads();
     }
-    __syncthreads();
     const bool evict_on = wp >= w;
     for (int base = 0; base < P; base += NT) {
         const int j = base + tid;
         bool keep = false;
-        if (j < P) keep = !evict_on || tmp_word[j] != 0u || (j + 1) > P - p.r;
+        if (j < P) keep = !evict_on || register_needed(tmp_word[j], w, P) || (j + 1) > P - p.r;
         const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
         if (lane == 0 && base + warp * 32 < P) keepmask[(base >> 5) + warp] = ballot;
     }

@@ -24,7 +24,9 @@ struct PromptFastParams {
     PromptParams p;
     unsigned char* partials;      // scratch: [U][n_splits][rows] {double m, double Z}, then [U][rows] thresholds
     uint32_t* ticket;             // [U] arrival counters (zero between launches)
-    int32_t split_len, n_splits, rows;   // rows = w * G
+    int32_t split_len, n_splits;
+    int32_t slot0, slot1;         // window slots [slot0, slot1) recorded by this pair of launches (oldest slot = 0)
+    int32_t rows;                 // (slot1 - slot0) * G
 };
 
 __host__ __device__ inline size_t prompt_fast_smem(int rows, int C) {
@@ -71,8 +73,9 @@ __device__ __forceinline__ void qk_tile_clamped(const unsigned char* ktile, int 
     for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
 }
 
-// Rows are numbered r = rho * G + g (query slot rho of the window, head g); the query of slot rho sits at prompt
-// position P - (w - 1 - rho) and exists iff rho >= w - min(P, w).
+// Rows of one launch are numbered r = (rho - slot0) * G + g (query slot rho of the window, head g); the query of
+// slot rho sits at prompt position P - (w - 1 - rho) and exists iff rho >= w - min(P, w). Windows whose rows do not
+// fit one launch (more than 64 rows) are recorded by several launch pairs, oldest slots first.
 __device__ __forceinline__ void load_row_group(const uint16_t* q_sm, int group, int ci, double (&qd)[4][8]) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
@@ -82,12 +85,13 @@ __device__ __forceinline__ void load_row_group(const uint16_t* q_sm, int group, 
 }
 
 // Shared prologue of both kernels: stage the q rows (row-major r = rho*G + g, padded to a multiple of four rows).
-__device__ __forceinline__ void stage_q_rows(const PromptParams& p, int u, int G, int rows_pad, uint16_t* q_sm) {
+__device__ __forceinline__ void stage_q_rows(const PromptParams& p, int u, int G, int slot0, int rows, int rows_pad,
+                                             uint16_t* q_sm) {
     const uint16_t* Q = reinterpret_cast<const uint16_t*>(p.q_last) + (size_t)u * G * p.w * 128;   // [G][w][128]
     for (int x = threadIdx.x; x < rows_pad * 16; x += blockDim.x) {          // 16-byte chunks
-        const int r = x >> 4, c = x & 15, rho = r / G, g = r - rho * G;
+        const int r = x >> 4, c = x & 15, rho = slot0 + r / G, g = r % G;
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < p.w * G) v = __ldg(reinterpret_cast<const uint4*>(Q + ((size_t)g * p.w + rho) * 128) + c);
+        if (r < rows) v = __ldg(reinterpret_cast<const uint4*>(Q + ((size_t)g * p.w + rho) * 128) + c);
         reinterpret_cast<uint4*>(q_sm + (size_t)r * 128)[c] = v;
     }
 }
@@ -100,13 +104,13 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_lse_kernel(const __
     constexpr int NW = kPromptFastWarps;
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv, P = __ldg(p.prompt_lens + b), w = p.w, wp = min(P, w);
-    const int rows = w * G, rows_pad = (rows + 3) / 4 * 4, groups = rows_pad / 4;
+    const int rows = fp.rows, rows_pad = (rows + 3) / 4 * 4, groups = rows_pad / 4, slot0 = fp.slot0;
     const int begin = split * fp.split_len, end = min(P, begin + fp.split_len);
     const int n_act = (P + fp.split_len - 1) / fp.split_len;
     if (P == 0 || split >= n_act) return;
     uint16_t* q_sm = reinterpret_cast<uint16_t*>(smem);
     double* mz_sm = reinterpret_cast<double*>(smem + (size_t)rows_pad * 256);        // [NW][rows_pad][2]
-    stage_q_rows(p, u, G, rows_pad, q_sm);
+    stage_q_rows(p, u, G, slot0, rows, rows_pad, q_sm);
     __syncthreads();
     const unsigned char* Kp = reinterpret_cast<const unsigned char*>(p.k_prompt) + (size_t)u * p.p_max * kRowBytes;
     const int h = lane >> 4, ci = lane & 15, key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);
@@ -117,7 +121,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_lse_kernel(const __
         int qpos[4];
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
-            const int r = 4 * gi + x, rho = r / G;
+            const int r = 4 * gi + x, rho = slot0 + r / G;
             qpos[x] = (r < rows && rho >= w - wp) ? P - (w - 1 - rho) : 0;
         }
         double m[4], Z[4];
@@ -175,7 +179,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_lse_kernel(const __
     // thresholds of Definition 3.1 in log form: s >= lse + ln(alpha) - ln(position of the query)
     double* thr = reinterpret_cast<double*>(fp.partials) + (size_t)p.U * fp.n_splits * rows_pad * 2 + (size_t)u * rows_pad;
     for (int r = tid; r < rows_pad; r += kPromptFastThreads) {
-        const int rho = r / G;
+        const int rho = slot0 + r / G;
         const bool exists = r < rows && rho >= w - wp;
         double mb = -1e300, Zb = 0.0;
         const double* pu = reinterpret_cast<const double*>(fp.partials) + (size_t)u * fp.n_splits * rows_pad * 2;
@@ -195,12 +199,13 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     constexpr int NW = kPromptFastWarps, NT = kPromptFastThreads;
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv, P = __ldg(p.prompt_lens + b), w = p.w, wp = min(P, w);
+    const bool last_launch = fp.slot1 == w;
     if (P > p.C) {
-        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
+        if (last_launch && split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
         return;
     }
-    if (P == 0) { if (split == 0 && tid == 0) { p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); } return; }
-    const int rows = w * G, rows_pad = (rows + 3) / 4 * 4, groups = rows_pad / 4;
+    if (P == 0) { if (last_launch && split == 0 && tid == 0) { p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); } return; }
+    const int rows = fp.rows, rows_pad = (rows + 3) / 4 * 4, groups = rows_pad / 4, slot0 = fp.slot0;
     const int begin = split * fp.split_len, end = min(P, begin + fp.split_len);
     const int n_act = (P + fp.split_len - 1) / fp.split_len;
     if (split >= n_act) return;
@@ -208,7 +213,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     double* thr_sm = reinterpret_cast<double*>(smem + (size_t)rows_pad * 256 + (size_t)NW * rows_pad * 16);
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(thr_sm + rows_pad);
     int* prefix = reinterpret_cast<int*>(keepmask + (p.C + 31) / 32 + 2);
-    stage_q_rows(p, u, G, rows_pad, q_sm);
+    stage_q_rows(p, u, G, slot0, rows, rows_pad, q_sm);
     const double* thr = reinterpret_cast<const double*>(fp.partials) + (size_t)p.U * fp.n_splits * rows_pad * 2 + (size_t)u * rows_pad;
     for (int r = tid; r < rows_pad; r += NT) thr_sm[r] = __ldcg(thr + r);
     __syncthreads();
@@ -221,23 +226,33 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     for (int tix = warp; tix < n_tiles; tix += NW) {
         const int k0 = begin + tix * kTileKeys, n_valid = min(kTileKeys, end - k0);
         const int pos_own = k0 + key_own + 1;
-        uint32_t bits = 0u;                                 // bit (w-1-rho) = verdict of the query of window slot rho
+        // verdicts of this launch's queries for the lane's key: a bit per window slot (bit w-1-rho) when the window
+        // fits a shift register, else the position of the newest query that found the key important
+        uint32_t reg = 0u;
         for (int gi = 0; gi < groups; ++gi) {
-            if (4 * gi / G < w - wp && (4 * gi + 3) / G < w - wp) continue;      // none of these queries exists
+            if (slot0 + (4 * gi + 3) / G < w - wp) continue;                      // none of these queries exists
             double qd[4][8], sown[4];
             load_row_group(q_sm, gi, ci, qd);
             qk_tile_clamped<4>(Kp + (size_t)k0 * kRowBytes, n_valid, qd, lane, sown);
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
-                const int r = 4 * gi + x, rho = r / G;
+                const int r = 4 * gi + x, rho = slot0 + r / G;
                 const bool exists = r < rows && rho >= w - wp;
                 const int qpos = P - (w - 1 - rho);
                 // Definition 3.1 in log form; keys newer than the query keep a 0 bit (Algorithm 1's zero padding)
-                if (exists && pos_own <= qpos && sown[x] * inv_root_d >= thr_sm[r]) bits |= 1u << (w - 1 - rho);
+                if (exists && pos_own <= qpos && sown[x] * inv_root_d >= thr_sm[r]) {
+                    if (w <= 32) reg |= 1u << (w - 1 - rho);
+                    else reg = max(reg, (uint32_t)qpos);
+                }
             }
         }
-        if (key_own < n_valid) tmp_word[k0 + key_own] = bits;
+        if (key_own < n_valid) {
+            uint32_t* dst = tmp_word + k0 + key_own;
+            if (slot0 == 0) *dst = reg;                                            // first launch of the window
+            else *dst = w <= 32 ? (*dst | reg) : max(*dst, reg);                   // same lane wrote it last time
+        }
     }
+    if (!last_launch) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) {
@@ -254,7 +269,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     for (int base = 0; base < P; base += NT) {
         const int j = base + tid;
         bool keep = false;
-        if (j < P) keep = !evict_on || __ldcg(tmp_word + j) != 0u || (j + 1) > P - p.r;
+        if (j < P) keep = !evict_on || register_needed(__ldcg(tmp_word + j), w, P) || (j + 1) > P - p.r;
         const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
         if (lane == 0 && base + warp * 32 < P) keepmask[(base >> 5) + warp] = ballot;
     }
@@ -296,8 +311,8 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
 inline corm_status_t launch_prompt_fast(PromptFastParams& fp, int G, int max_p, int sm_count, size_t partial_capacity,
                                         cudaStream_t st) {
     const PromptParams& p = fp.p;
-    fp.rows = p.w * G;
-    const int rows_pad = (fp.rows + 3) / 4 * 4;
+    const int chunk_slots = 64 / G < p.w ? 64 / G : p.w;                 // at most 64 (slot, head) rows per launch pair
+    const int rows_pad = (chunk_slots * G + 3) / 4 * 4;
     // about four blocks per SM in flight, splits of whole tiles, at least 512 keys
     long long want_blocks = 4ll * (sm_count > 0 ? sm_count : 148);
     long long per_unit = (want_blocks + p.U - 1) / p.U;
@@ -314,8 +329,13 @@ inline corm_status_t launch_prompt_fast(PromptFastParams& fp, int G, int max_p, 
         if (e == cudaSuccess) e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         const dim3 grid(fp.n_splits, (unsigned)p.U);
-        k1<<<grid, kPromptFastThreads, smem, st>>>(fp);
-        k2<<<grid, kPromptFastThreads, smem, st>>>(fp);
+        for (int s0 = 0; s0 < p.w; s0 += chunk_slots) {                  // oldest window slots first
+            fp.slot0 = s0;
+            fp.slot1 = s0 + chunk_slots < p.w ? s0 + chunk_slots : p.w;
+            fp.rows = (fp.slot1 - fp.slot0) * G;
+            k1<<<grid, kPromptFastThreads, smem, st>>>(fp);
+            k2<<<grid, kPromptFastThreads, smem, st>>>(fp);
+        }
         e = cudaGetLastError();
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: prompt launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;
@@ -327,6 +347,12 @@ inline corm_status_t launch_prompt_fast(PromptFastParams& fp, int G, int max_p, 
         case 8: return run(prompt_lse_kernel<8>, prompt_verdict_kernel<8>);
     }
     return CORM_ERR_UNSUPPORTED;
+}
+
+// number of kernel launches launch_prompt_fast issues for this window and group size
+inline int prompt_fast_launches(int G, int w) {
+    const int chunk_slots = 64 / G < w ? 64 / G : w;
+    return 2 * ((w + chunk_slots - 1) / chunk_slots);
 }
 
 }  // namespace corm

@@ -129,6 +129,54 @@ def test_multi_layer_independent_and_deterministic():
     assert gpu.corm_cache_kernel_launches() == 2 * 3 + 3 * cfg.steps        # two launches per prompt pass, one per step
 
 
+WIDE = [
+    # dtype, d, G, n_kv, B, prompt range, steps, w, r, split_len, fast, alpha, seed
+    ("bf16", 128, 1, 4, 2, (300, 520), 80, 40, 16, 0, True, 1.0, 4242),      # tiled prompt pass, one launch pair
+    ("bf16", 128, 1, 2, 2, (20, 90), 150, 64, 8, 0, True, 1.0, 4245),        # prompts near the window size; it fills in decode
+    ("bf16", 128, 4, 2, 2, (400, 900), 60, 48, 32, 128, True, 2.0, 4242),    # GQA, three launch pairs, multi-split decode
+    ("bf16", 128, 1, 2, 1, (1500, 1500), 40, 256, 256, 0, True, 6.0, 4242),  # the paper's 256 + 256 budget
+    ("bf16", 128, 4, 1, 1, (700, 700), 300, 256, 64, 0, True, 6.0, 4243),    # 256-query window, 16 launch pairs
+    ("f32", 64, 2, 2, 2, (150, 260), 70, 100, 10, 64, False, 1.5, 4242),     # generic kernels, chunked prompt rows
+    ("bf16", 128, 8, 1, 1, (300, 300), 50, 33, 4, 0, True, 1.0, 4243),       # group of 8: generic decode, tiled prompt
+]
+
+
+@pytest.mark.parametrize("case", WIDE, ids=lambda c: "-".join(str(x) for x in c))
+def test_windows_beyond_32_queries(case):
+    """Windows of 33..256 queries keep, per key, the step of its latest important verdict instead of a shift register;
+    live lists, rows and the visible part of every register must still match the oracle's multi-word registers."""
+    dtype, d, G, nkv, B, (pmin, pmax), steps, w, r, split_len, fast, alpha, seed = case
+    cfg = CONFIGS[1].with_(name="wide", batch=B, n_q_heads=nkv * G, n_kv_heads=nkv, head_dim=d, dtype=dtype,
+                           prompt_min=pmin, prompt_max=pmax, steps=steps, window_w=w, recent_r=r, alpha=alpha,
+                           gqa_rho=0.7 if G > 1 else 0.0, hh_min=2, hh_max=6, seed=seed)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    gpu.corm_cache_set_tuning(split_len, fast)
+    run_free(cfg, data, gpu, orc, check_every=5)
+    assert orc.counters()["near_threshold"] == 0
+    assert gpu.corm_cache_stats()["evicted_keys"] > 0
+
+
+def test_wide_window_import_roundtrip():
+    """Importing the oracle's state (ages turned into stamps) and stepping gives the oracle's next state."""
+    from parity_util import ages_to_stamps
+    cfg = CONFIGS[1].with_(prompt_min=260, prompt_max=260, steps=30, dtype="bf16", n_q_heads=2, n_kv_heads=2,
+                           window_w=70, recent_r=12)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    orc.compress_prompt(0, data.k_prompt, data.v_prompt, data.q_last, data.prompt_lens)
+    dt = cfg.dtype
+    for s in range(cfg.steps):
+        for h in range(2):
+            st = orc.export_unit(0, 0, h)
+            gpu.corm_cache_import_state(0, 0, h, st["k"], st["v"], ages_to_stamps(st["age"], st["n_tokens"]),
+                                        st["pos"], st["n_tokens"], st["n_obs"])
+        out_g = gpu.corm_decode_step(0, to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt))
+        out_o = orc.decode_step(0, data.q[s], data.k_new[s], data.v_new[s])
+        assert np.abs(out_g.float().cpu().numpy() - out_o).max() <= OUT_TOL[dt]
+        assert_states_equal(gpu, orc, 0, 1, 2, f"step {s}")
+
+
 def test_host_buffer_entry_point_matches_device_one():
     cfg = CONFIGS[1].with_(prompt_min=130, prompt_max=130, steps=10, dtype="bf16")
     data = generate(cfg)

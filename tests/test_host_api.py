@@ -57,7 +57,7 @@ def test_create_rejects_before_any_cuda_call(lib):
     assert lib.corm_cache_create(ctypes.byref(cfg), fake, need - 1, ctypes.byref(handle)) == 3
     assert lib.corm_cache_create(ctypes.byref(cfg), None, need, ctypes.byref(handle)) == 1
     assert lib.corm_cache_create(ctypes.byref(cfg), ctypes.c_void_p(0x10001), need, ctypes.byref(handle)) == 1
-    for bad, code in [(dict(head_dim=96), 2), (dict(window_w=33), 2), (dict(n_q_heads=6, n_kv_heads=2), 2),
+    for bad, code in [(dict(head_dim=96), 2), (dict(window_w=257), 2), (dict(n_q_heads=6, n_kv_heads=2), 2),
                       (dict(n_q_heads=7), 1)]:
         c = _cfg(**bad)
         assert lib.corm_cache_create(ctypes.byref(c), fake, 1 << 40, ctypes.byref(handle)) == code
