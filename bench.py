@@ -163,10 +163,16 @@ def main():
     ap.add_argument("--no-fast", action="store_true")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--window", type=int, default=None, help="override the verdict window w (1..256)")
+    ap.add_argument("--recent", type=int, default=None, help="override the protected recent tokens r")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
     if args.alpha is not None:
         cfg = cfg.with_(alpha=args.alpha, name=cfg.name + f"_alpha{args.alpha:g}")
+    if args.window is not None:
+        cfg = cfg.with_(window_w=args.window, name=cfg.name + f"_w{args.window}")
+    if args.recent is not None:
+        cfg = cfg.with_(recent_r=args.recent, name=cfg.name + f"_r{args.recent}")
     if args.impl == "reference":
         return run_reference(args, cfg)
 
