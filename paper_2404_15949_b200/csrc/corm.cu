@@ -27,7 +27,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -74,6 +74,7 @@ Layout make_layout(const corm_config_t& c) {
     L.bookkeeping_end = off;
     L.stash = take(U * G * C * 8);
     L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
+    L.keepmask = take(U * (size_t)keepmask_words((int)C) * 4);
     L.stage_q = take((size_t)c.batch * c.n_q_heads * D * e);
     L.stage_k = take(U * D * e);
     L.stage_v = take(U * D * e);
@@ -192,6 +193,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.maxlive = maxlive_ptr(c, layer);
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.partials = c->arena + c->lay.partials;
+    p.keepmask = reinterpret_cast<uint32_t*>(c->arena + c->lay.keepmask);
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
     p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
@@ -200,8 +202,9 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
 
     const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
+    int n_launched = 1;
     if (fast) {
-        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st);
+        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st, &n_launched);
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
         const int n_splits = (upper + p.split_len - 1) / p.split_len;
@@ -217,7 +220,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
         });
     }
     if (rc != CORM_OK) return rc;
-    c->launches += 1;
+    c->launches += n_launched;
     c->parity[layer] ^= 1;
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);

@@ -28,6 +28,7 @@ struct DecodeParams {
     unsigned long long* maxlive;  // (steps done << 32 | longest live length after that step), atomicMax; may be null
     double* stash;            // [U*G][C] scaled logits of this step (scratch)
     unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
+    uint32_t* keepmask;       // [U][ceil(C/32)+2] keep bits of the verdict launch (scratch)
     const void* q;            // [B][Hq][D]
     const void* k_new;        // [B][Hkv][D]
     const void* v_new;        // [B][Hkv][D]

@@ -13,6 +13,7 @@
 #pragma once
 
 #include "corm_common.cuh"
+#include "corm_verdict.cuh"
 
 namespace corm {
 
@@ -32,6 +33,7 @@ constexpr int kVStages = 1;
 // one query head per KV head leaves registers and shared memory for three blocks per SM; larger groups keep two.
 __host__ __device__ constexpr int fast_k_stages(int G) { return G == 1 ? 1 : 2; }
 __host__ __device__ constexpr int fast_stages(int G) { return fast_k_stages(G) + kVStages; }
+__host__ __device__ constexpr int fast_warp_bytes(int G) { return fast_stages(G) * kTileBytes; }
 __host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? CORM_FAST_BLOCKS_G1 : 2; }
 // 228 KB per SM, minus 1 KB the system reserves per block and ~1.2 KB of static shared memory
 __host__ __device__ constexpr int fast_smem_budget(int G) { return (228 * 1024) / fast_blocks_per_sm(G) - 2304; }
@@ -49,7 +51,7 @@ __host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
     FastSmem s;
     int off = 0;
     auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
-    s.tiles = take(kFastWarps * fast_stages(G) * kTileBytes);   // later reused: merge area, finalize lists
+    s.tiles = take(kFastWarps * fast_warp_bytes(G));            // later reused: merge area, finalize lists
     s.qs = take(G * 128 * 8);
     s.psm = take(kFastWarps * kTileKeys * G * 4);
     s.stash = take(single_cap * G * 8);
@@ -253,13 +255,15 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
 template <int G>
 __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ int s_last;
     __shared__ int s_failed;
     __shared__ double s_thr1[G];
     constexpr int NT = kFastThreads, NW = kFastWarps;
     constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
+    // the verdict launch that may follow is allowed to become resident from here on (it waits for this grid to
+    // complete before it reads anything written here)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C) {
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
@@ -272,7 +276,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     const int begin = split * p.split_len, end = min(l, begin + p.split_len);
     const int n_tiles = (end - begin + kTileKeys - 1) / kTileKeys;
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
-    unsigned char* my_tiles = smem + lay.tiles + warp * kStagesPerWarp * kTileBytes;
+    unsigned char* my_tiles = smem + lay.tiles + warp * fast_warp_bytes(G);
     const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kStagesPerWarp * 8;
     double* qs = reinterpret_cast<double*>(smem + lay.qs);
     float* psm = reinterpret_cast<float*>(smem + lay.psm) + warp * kTileKeys * G;
@@ -513,29 +517,29 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l);
         return;
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned prev = atomicAdd(p.ticket + u, 1u);
-        s_last = (prev == (unsigned)(n_act - 1));
-        if (s_last) p.ticket[u] = 0u;
-        __threadfence();
-    }
-    __syncthreads();
-    if (!s_last) return;
-    finalize_unit<bf16_t, 128, G, NT>(p, u, b, l, n_act, t, smem);
+    // a unit of several splits: its partial records and logits are complete once this launch ends; the verdict
+    // launch that follows takes Algorithm 1 from there
 }
 
 // Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
 inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int tune_split_len, int sm_count,
-                                        cudaStream_t st) {
+                                        cudaStream_t st, int* n_launched) {
+    *n_launched = 0;
     if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
+    // longest unit that can finish inside one block: bounded by the verdict registers a thread carries and by the
+    // shared memory that holds the unit's logits
+    int cap = fast_max_single_cap(G);
+    while (cap > 0 && fast_smem_layout(G, cap).total > fast_smem_budget(G)) cap -= kFastWarps * kTileKeys;
+    const int sms = sm_count > 0 ? sm_count : 148;
     int split_len = tune_split_len;
-    if (!split_len) {
+    if (!split_len && upper <= cap && p.U >= 2 * sms) {
+        // enough units to fill the machine without splitting them: one launch, every unit finished on chip
+        split_len = upper;
+    } else if (!split_len) {
         // enough blocks to fill the machine about four times over, but no smaller than one tile per warp and no
         // larger than 2048 keys (long splits amortise the per-block prologue and merge)
         const long long total_tiles = (long long)((upper + kTileKeys - 1) / kTileKeys) * p.U;
-        const long long target_blocks = 4ll * (sm_count > 0 ? sm_count : 148);
+        const long long target_blocks = 4ll * sms;
         long long tiles_per_block = (total_tiles + target_blocks - 1) / target_blocks;
         if (tiles_per_block < kFastWarps) tiles_per_block = kFastWarps;
         split_len = (int)(tiles_per_block * kTileKeys > 2048 ? 2048 : tiles_per_block * kTileKeys);
@@ -545,15 +549,12 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     const int n_splits = (upper + split_len - 1) / split_len;
     if (n_splits > p.max_splits) return CORM_ERR_UNSUPPORTED;
     // on-chip finish for units of one split, as long as two blocks still fit on an SM
-    p.single_cap = split_len < fast_max_single_cap(G) ? split_len : fast_max_single_cap(G);
-    while (p.single_cap > 0 && fast_smem_layout(G, p.single_cap).total > fast_smem_budget(G)) p.single_cap -= kFastWarps * kTileKeys;
+    p.single_cap = split_len < cap ? split_len : cap;
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
-    size_t smem = (size_t)lay.total;
-    const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // multi-split finalize lists
+    const size_t smem = (size_t)lay.total;
     const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
                         (size_t)2 * p.single_cap * 4;
-    if (fin > smem) smem = fin;
-    if (fin1 > (size_t)kFastWarps * fast_stages(G) * kTileBytes) return CORM_ERR_UNSUPPORTED;
+    if (fin1 > (size_t)kFastWarps * fast_warp_bytes(G)) return CORM_ERR_UNSUPPORTED;
     if (smem > 227 * 1024) return CORM_ERR_UNSUPPORTED;
     auto launch = [&](auto kern) -> corm_status_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -563,9 +564,35 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;
     };
-    if (G == 1) return launch(decode_fast_kernel<1>);
-    if (G == 2) return launch(decode_fast_kernel<2>);
-    return launch(decode_fast_kernel<4>);
+    corm_status_t rc = G == 1 ? launch(decode_fast_kernel<1>) : G == 2 ? launch(decode_fast_kernel<2>) : launch(decode_fast_kernel<4>);
+    if (rc != CORM_OK) return rc;
+    *n_launched = 1;
+    if (n_splits == 1 && upper <= p.single_cap) return CORM_OK;          // every unit finishes inside the streaming kernel
+    // verdict launch for the units that do not
+    const size_t vsmem = verdict_smem(p.C, n_splits, G);
+    auto launch_v = [&](auto kern) -> corm_status_t {
+        cudaError_t e = cudaSuccess;
+        if (vsmem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vsmem);
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((upper + kVerdictChunk - 1) / kVerdictChunk, (unsigned)p.U);
+        cfg.blockDim = dim3(kVerdictThreads);
+        cfg.dynamicSmemBytes = vsmem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may overlap the streaming kernel's tail
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, p, n_splits);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: verdict launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        return CORM_OK;
+    };
+    rc = G == 1 ? launch_v(decode_verdict_kernel<bf16_t, 128, 1>) : G == 2 ? launch_v(decode_verdict_kernel<bf16_t, 128, 2>)
+                                                                           : launch_v(decode_verdict_kernel<bf16_t, 128, 4>);
+    if (rc == CORM_OK) *n_launched = 2;
+    return rc;
 }
 
 }  // namespace corm

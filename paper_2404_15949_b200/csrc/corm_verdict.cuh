@@ -1,0 +1,179 @@
+// Second launch of a decode step for units that span several splits: the work that follows the streaming pass
+// (Algorithm 1's verdict row, register update, keep decision, compaction), spread over many blocks instead of one.
+//
+// The streaming kernel leaves, per unit, one partial record {m, Z, acc[D]} per split and query head and the scaled
+// logits of every live key. Here a block owns 1024 consecutive slots of one unit:
+//   a. every block reduces the (m, Z) of the unit's splits to lse_g and the threshold of Definition 3.1 in log form
+//      (a few dozen values; the same arithmetic in the same order in every block, so all blocks agree bit for bit);
+//      block 0 of the unit also reduces the accumulators to the attention output of Eq. 1;
+//   b. verdicts of its slots (OR over the group), register update, keep flag -> one bit per slot in a global mask;
+//   c. the block that finishes last (arrival counter after a fence) scans the mask, fills the holes below the new
+//      length with kept rows from above it, and publishes the new length. No block waits for another.
+// The launch is programmatic-dependent on the streaming kernel: its blocks may become resident while the last
+// streaming blocks still run, read what the streaming kernel does not write (lengths, registers and positions of
+// the older slots), and only then wait for the streaming grid to complete.
+#pragma once
+
+#include "corm_common.cuh"
+
+namespace corm {
+
+constexpr int kVerdictThreads = 256;
+constexpr int kVerdictChunk = 1024;                       // slots per block
+constexpr int kVerdictPer = kVerdictChunk / kVerdictThreads;
+
+__host__ __device__ inline int keepmask_words(int C) { return (C + 31) / 32 + 2; }
+
+__host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G) {
+    return (size_t)G * n_splits * (8 + 8 + 4) + 16 + (size_t)2 * keepmask_words(C) * 4;
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
+                                                                         const int n_splits) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ double s_thr[G], s_Z[G];
+    __shared__ int s_scan[kVerdictThreads];
+    __shared__ int s_last;
+    constexpr int NT = kVerdictThreads;
+    const int u = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = u / p.Hkv;
+    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    if (l > p.C) return;                                                   // reported by the streaming kernel
+    const int n_act = (l + p.split_len - 1) / p.split_len;
+    if (n_act == 1 && l <= p.single_cap) return;                           // finished inside the streaming kernel
+    const int n_chunks = (l + kVerdictChunk - 1) / kVerdictChunk;
+    if (chunk >= n_chunks) return;
+    const int t = __ldg(p.base_tokens + b) + p.step + 1;
+    const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
+    const bool evict_on = n_obs >= p.w;
+    uint32_t* wordu = p.word + (size_t)u * p.C;
+    int32_t* posu = p.pos + (size_t)u * p.C;
+    const int base0 = chunk * kVerdictChunk;
+    uint32_t wv[kVerdictPer];
+    int32_t pv[kVerdictPer];
+#pragma unroll
+    for (int k = 0; k < kVerdictPer; ++k) {                                // the appended slot l_old starts as (0, t)
+        const int j = base0 + k * NT + tid;
+        wv[k] = j < l_old ? __ldcg(wordu + j) : 0u;
+        pv[k] = j < l_old ? __ldcg(posu + j) : t;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");                     // the streaming grid has completed
+    if (__ldcg(p.status) == (int)CORM_ERR_TIMEOUT) return;                 // a copy never arrived: leave the unit as is
+
+    double* sm_m = reinterpret_cast<double*>(smem);                        // [G][n_splits]
+    double* sm_Z = sm_m + (size_t)G * n_splits;
+    float* sm_sc = reinterpret_cast<float*>(sm_Z + (size_t)G * n_splits);
+    uint32_t* keep_sm = reinterpret_cast<uint32_t*>(smem + (((size_t)G * n_splits * 20 + 15) & ~(size_t)15));
+    int* prefix = reinterpret_cast<int*>(keep_sm + keepmask_words(p.C));
+    const size_t pstride = partial_stride(D);
+    const unsigned char* rec_u = p.partials + (size_t)u * p.max_splits * G * pstride;
+
+    // a. split reduction
+    for (int x = tid; x < G * n_act; x += NT) {
+        const int g = x / n_act, s = x - g * n_act;
+        const double* rec = reinterpret_cast<const double*>(rec_u + ((size_t)s * G + g) * pstride);
+        sm_m[g * n_splits + s] = __ldcg(rec);
+        sm_Z[g * n_splits + s] = __ldcg(rec + 1);
+    }
+    __syncthreads();
+    if (tid < G) {
+        const int g = tid;
+        double m = -INFINITY;
+        for (int s = 0; s < n_act; ++s) m = fmax(m, sm_m[g * n_splits + s]);
+        double Z = 0.0;
+        for (int s = 0; s < n_act; ++s) {
+            const double sc = exp(sm_m[g * n_splits + s] - m);
+            Z += sm_Z[g * n_splits + s] * sc;
+            sm_sc[g * n_splits + s] = (float)sc;
+        }
+        s_Z[g] = Z;
+        s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);             // Definition 3.1: s >= lse + ln(alpha) - ln(t)
+    }
+    __syncthreads();
+    if (chunk == 0) {
+        for (int x = tid; x < G * D; x += NT) {
+            const int g = x / D, c = x - g * D;
+            float acc = 0.f;
+            for (int s = 0; s < n_act; ++s)
+                acc += __ldcg(reinterpret_cast<const float*>(rec_u + ((size_t)s * G + g) * pstride + 16) + c) *
+                       sm_sc[g * n_splits + s];
+            Elem<T>::store(reinterpret_cast<T*>(p.out) + ((size_t)u * G + g) * D + c, (float)((double)acc / s_Z[g]));
+        }
+    }
+
+    // b. verdicts, register update, keep flags of this block's slots
+    const double* stash_u = p.stash + (size_t)u * G * p.C;
+    uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
+    {
+        double sv[kVerdictPer][G];
+#pragma unroll
+        for (int k = 0; k < kVerdictPer; ++k) {
+            const int j = base0 + k * NT + tid;
+#pragma unroll
+            for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
+        }
+#pragma unroll
+        for (int k = 0; k < kVerdictPer; ++k) {
+            const int base = base0 + k * NT, j = base + tid;
+            if (base >= l) break;                                          // uniform
+            bool keep = false;
+            if (j < l) {
+                bool imp = false;
+#pragma unroll
+                for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
+                const uint32_t wd = update_register(wv[k], imp, p.w, t);
+                wordu[j] = wd;
+                keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
+            }
+            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0 && base + warp * 32 < l) keep_g[(base >> 5) + warp] = ballot;
+        }
+    }
+
+    // c. the last block of the unit to get here compacts it
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned prev = atomicAdd(p.ticket + u, 1u);
+        s_last = (prev == (unsigned)(n_chunks - 1));
+        if (s_last) p.ticket[u] = 0u;
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_last) return;
+    int new_len = l, n_moved = 0;
+    if (evict_on) {
+        const int nwords = (l + 31) / 32;
+        for (int i = tid; i < nwords; i += NT) keep_sm[i] = __ldcg(keep_g + i);
+        __syncthreads();
+        block_popc_scan<NT>(keep_sm, prefix, nwords, s_scan);
+        new_len = prefix[nwords];
+        if (new_len < l) {
+            // the k-th kept row at or above new_len moves into the k-th hole below it
+            int* holes = reinterpret_cast<int*>(const_cast<double*>(stash_u));   // every block is done with the logits
+            int* movers = holes + p.C;
+            const int kept_below = kept_before(keep_sm, prefix, new_len);
+            n_moved = new_len - kept_below;
+            for (int j = tid; j < l; j += NT) {
+                const int kb = kept_before(keep_sm, prefix, j);
+                const bool kept = (keep_sm[j >> 5] >> (j & 31)) & 1u;
+                if (j < new_len && !kept) holes[j - kb] = j;
+                if (j >= new_len && kept) movers[kb - kept_below] = j;
+            }
+            __syncthreads();
+            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D,
+                                      reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D, wordu, posu, movers, holes, n_moved);
+        }
+    }
+    if (tid == 0) {
+        p.live_out[u] = new_len;
+        publish_live(p.maxlive, p.step + 1, new_len);
+        atomicAdd(p.counters + CNT_APPENDED, 1ull);
+        atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+        if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+        if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
+    }
+}
+
+}  // namespace corm

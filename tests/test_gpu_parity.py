@@ -126,7 +126,9 @@ def test_multi_layer_independent_and_deterministic():
             sa = sorted_state(gpu.corm_cache_export_state(l, 0, h))
             sb = sorted_state(gpu2.corm_cache_export_state(l, 0, h))
             assert all(np.array_equal(sa[k], sb[k]) for k in ("k", "v", "word", "pos"))
-    assert gpu.corm_cache_kernel_launches() == 2 * 3 + 3 * cfg.steps        # two launches per prompt pass, one per step
+    # two launches per prompt pass; per step one streaming launch, plus a verdict launch while units span several splits
+    n = gpu.corm_cache_kernel_launches()
+    assert 2 * 3 + 3 * cfg.steps <= n <= 2 * 3 + 2 * 3 * cfg.steps and n == gpu2.corm_cache_kernel_launches()
 
 
 WIDE = [
