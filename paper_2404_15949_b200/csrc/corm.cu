@@ -213,7 +213,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
             constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
             const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
             auto kern = decode_generic_kernel<T, DD, GG>;
-            if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
             kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
             CORM_CUDA(cudaGetLastError());
             return CORM_OK;
@@ -374,7 +374,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
             constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
             const size_t smem = prompt_smem(GG, cf.window_w, cf.max_tokens);
             auto kern = prompt_generic_kernel<T, DD, GG>;
-            if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
             kern<<<(unsigned)U, kPromptThreads, smem, st>>>(p);
             CORM_CUDA(cudaGetLastError());
             return CORM_OK;
@@ -496,7 +496,7 @@ corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void
         constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
         const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
         auto kern = decode_generic_kernel<T, DD, GG>;
-        if (smem > 48 * 1024) CORM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
         kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
         CORM_CUDA(cudaGetLastError());
         return CORM_OK;

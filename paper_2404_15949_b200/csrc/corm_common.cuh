@@ -6,9 +6,35 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/corm.h"
 
 namespace corm {
+
+// Raises a kernel's dynamic shared-memory limit on the current device when a launch needs more than any earlier one
+// did; the driver call is skipped otherwise (it costs more than a microsecond and decode launches are that short).
+inline cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+    struct Entry { const void* kernel; int device; size_t bytes; };
+    constexpr int kSlots = 256;                       // fixed table: nothing is allocated here, on host or device
+    static std::mutex mu;
+    static Entry seen[kSlots];
+    static int n_seen = 0;
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    int device = 0;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    Entry* slot = nullptr;
+    for (int i = 0; i < n_seen && !slot; ++i)
+        if (seen[i].kernel == kernel && seen[i].device == device) slot = &seen[i];
+    if (slot && bytes <= slot->bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    if (slot) slot->bytes = bytes;
+    else if (n_seen < kSlots) seen[n_seen++] = Entry{kernel, device, bytes};   // a full table only costs the shortcut
+    return e;
+}
 
 // Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
 enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_COUNT = 4 };

@@ -557,7 +557,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     if (fin1 > (size_t)kFastWarps * fast_warp_bytes(G)) return CORM_ERR_UNSUPPORTED;
     if (smem > 227 * 1024) return CORM_ERR_UNSUPPORTED;
     auto launch = [&](auto kern) -> corm_status_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         kern<<<dim3(n_splits, (unsigned)p.U), kFastThreads, smem, st>>>(p);
         e = cudaGetLastError();
@@ -571,8 +571,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     // verdict launch for the units that do not
     const size_t vsmem = verdict_smem(p.C, n_splits, G);
     auto launch_v = [&](auto kern) -> corm_status_t {
-        cudaError_t e = cudaSuccess;
-        if (vsmem > 48 * 1024) e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vsmem);
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), vsmem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((upper + kVerdictChunk - 1) / kVerdictChunk, (unsigned)p.U);

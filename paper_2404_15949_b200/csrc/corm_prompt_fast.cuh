@@ -325,8 +325,8 @@ inline corm_status_t launch_prompt_fast(PromptFastParams& fp, int G, int max_p, 
     const size_t smem = prompt_fast_smem(rows_pad, p.C);
     if (need > partial_capacity || smem > 200 * 1024 || p.U > 65535) return CORM_ERR_UNSUPPORTED;
     auto run = [&](auto k1, auto k2) -> corm_status_t {
-        cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(k1), smem);
+        if (e == cudaSuccess) e = ensure_dynamic_smem(reinterpret_cast<const void*>(k2), smem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         const dim3 grid(fp.n_splits, (unsigned)p.U);
         for (int s0 = 0; s0 < p.w; s0 += chunk_slots) {                  // oldest window slots first

@@ -29,13 +29,14 @@ __host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G) {
 }
 
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
+__global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
                                                                          const int n_splits) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ double s_thr[G], s_Z[G];
     __shared__ int s_scan[kVerdictThreads];
     __shared__ int s_last;
-    constexpr int NT = kVerdictThreads;
+    constexpr int NT = kVerdictThreads, kListCap = 512;
+    __shared__ int s_lists[2 * kListCap];
     const int u = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
@@ -59,7 +60,16 @@ __global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const _
         pv[k] = j < l_old ? __ldcg(posu + j) : t;
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");                     // the streaming grid has completed
-    if (__ldcg(p.status) == (int)CORM_ERR_TIMEOUT) return;                 // a copy never arrived: leave the unit as is
+    // everything this block needs from the streaming kernel is requested at once: status, split records, logits
+    const int status = __ldcg(p.status);
+    const double* stash_u = p.stash + (size_t)u * G * p.C;
+    double sv[kVerdictPer][G];
+#pragma unroll
+    for (int k = 0; k < kVerdictPer; ++k) {
+        const int j = base0 + k * NT + tid;
+#pragma unroll
+        for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
+    }
 
     double* sm_m = reinterpret_cast<double*>(smem);                        // [G][n_splits]
     double* sm_Z = sm_m + (size_t)G * n_splits;
@@ -76,43 +86,30 @@ __global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const _
         sm_m[g * n_splits + s] = __ldcg(rec);
         sm_Z[g * n_splits + s] = __ldcg(rec + 1);
     }
+    if (status == (int)CORM_ERR_TIMEOUT) return;                           // a copy never arrived: leave the unit as is
     __syncthreads();
-    if (tid < G) {
-        const int g = tid;
+    if (warp < G) {                                                        // warp g reduces head g, a split per lane
+        const int g = warp;
         double m = -INFINITY;
-        for (int s = 0; s < n_act; ++s) m = fmax(m, sm_m[g * n_splits + s]);
+        for (int s = lane; s < n_act; s += 32) m = fmax(m, sm_m[g * n_splits + s]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
         double Z = 0.0;
-        for (int s = 0; s < n_act; ++s) {
+        for (int s = lane; s < n_act; s += 32) {
             const double sc = exp(sm_m[g * n_splits + s] - m);
             Z += sm_Z[g * n_splits + s] * sc;
             sm_sc[g * n_splits + s] = (float)sc;
         }
-        s_Z[g] = Z;
-        s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);             // Definition 3.1: s >= lse + ln(alpha) - ln(t)
+        Z = warp_sum(Z);                                                   // fixed tree: every block gets the same bits
+        if (lane == 0) {
+            s_Z[g] = Z;
+            s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);         // Definition 3.1: s >= lse + ln(alpha) - ln(t)
+        }
     }
     __syncthreads();
-    if (chunk == 0) {
-        for (int x = tid; x < G * D; x += NT) {
-            const int g = x / D, c = x - g * D;
-            float acc = 0.f;
-            for (int s = 0; s < n_act; ++s)
-                acc += __ldcg(reinterpret_cast<const float*>(rec_u + ((size_t)s * G + g) * pstride + 16) + c) *
-                       sm_sc[g * n_splits + s];
-            Elem<T>::store(reinterpret_cast<T*>(p.out) + ((size_t)u * G + g) * D + c, (float)((double)acc / s_Z[g]));
-        }
-    }
-
     // b. verdicts, register update, keep flags of this block's slots
-    const double* stash_u = p.stash + (size_t)u * G * p.C;
     uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
     {
-        double sv[kVerdictPer][G];
-#pragma unroll
-        for (int k = 0; k < kVerdictPer; ++k) {
-            const int j = base0 + k * NT + tid;
-#pragma unroll
-            for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
-        }
 #pragma unroll
         for (int k = 0; k < kVerdictPer; ++k) {
             const int base = base0 + k * NT, j = base + tid;
@@ -141,6 +138,25 @@ __global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const _
         __threadfence();
     }
     __syncthreads();
+    {   // Eq. 1: the unit's G x D outputs are shared out over its blocks
+        const int per = (G * D + n_chunks - 1) / n_chunks, x_end = min(G * D, (chunk + 1) * per);
+        for (int x = chunk * per + tid; x < x_end; x += NT) {
+            const int g = x / D, c = x - g * D;
+            float acc = 0.f;
+            for (int s0 = 0; s0 < n_act; s0 += 8) {                       // eight loads in flight, summed in split order
+                float a[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    a[k] = s0 + k < n_act
+                               ? __ldcg(reinterpret_cast<const float*>(rec_u + ((size_t)(s0 + k) * G + g) * pstride + 16) + c)
+                               : 0.f;
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (s0 + k < n_act) acc += a[k] * sm_sc[g * n_splits + s0 + k];
+            }
+            Elem<T>::store(reinterpret_cast<T*>(p.out) + ((size_t)u * G + g) * D + c, (float)((double)acc / s_Z[g]));
+        }
+    }
     if (!s_last) return;
     int new_len = l, n_moved = 0;
     if (evict_on) {
@@ -150,16 +166,33 @@ __global__ void __launch_bounds__(kVerdictThreads) decode_verdict_kernel(const _
         block_popc_scan<NT>(keep_sm, prefix, nwords, s_scan);
         new_len = prefix[nwords];
         if (new_len < l) {
-            // the k-th kept row at or above new_len moves into the k-th hole below it
-            int* holes = reinterpret_cast<int*>(const_cast<double*>(stash_u));   // every block is done with the logits
-            int* movers = holes + p.C;
+            // the k-th kept row at or above new_len moves into the k-th hole below it; both lists are built word by
+            // word from the keep mask (few bits qualify), in shared memory when they are short
             const int kept_below = kept_before(keep_sm, prefix, new_len);
             n_moved = new_len - kept_below;
-            for (int j = tid; j < l; j += NT) {
-                const int kb = kept_before(keep_sm, prefix, j);
-                const bool kept = (keep_sm[j >> 5] >> (j & 31)) & 1u;
-                if (j < new_len && !kept) holes[j - kb] = j;
-                if (j >= new_len && kept) movers[kb - kept_below] = j;
+            int* holes = s_lists;
+            int* movers = s_lists + kListCap;
+            if (n_moved > kListCap) {
+                holes = reinterpret_cast<int*>(const_cast<double*>(stash_u));    // every block is done with the logits
+                movers = holes + p.C;
+            }
+            for (int i = tid; i < nwords; i += NT) {
+                const uint32_t m = keep_sm[i];
+                const int j0 = i * 32;
+                const uint32_t valid = l - j0 >= 32 ? 0xffffffffu : (1u << (l - j0)) - 1u;
+                const uint32_t below = new_len - j0 >= 32 ? 0xffffffffu : (new_len > j0 ? (1u << (new_len - j0)) - 1u : 0u);
+                uint32_t hm = ~m & valid & below;                  // evicted slots below the new length
+                while (hm) {
+                    const int bit = __ffs(hm) - 1;
+                    hm &= hm - 1u;
+                    holes[j0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = j0 + bit;
+                }
+                uint32_t km = m & ~below;                          // kept slots at or above it
+                while (km) {
+                    const int bit = __ffs(km) - 1;
+                    km &= km - 1u;
+                    movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = j0 + bit;
+                }
             }
             __syncthreads();
             block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D,
