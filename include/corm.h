@@ -108,8 +108,10 @@ corm_status_t corm_compress_prompt(corm_cache_t* cache, int32_t layer, const voi
 corm_status_t corm_decode_step(corm_cache_t* cache, int32_t layer, const void* q, const void* k_new,
                                const void* v_new, void* out, void* stream);
 
-/* Same step with HOST buffers (pinned memory recommended): copies q, k_new, v_new to staging space inside the
- * arena, runs the step and copies out back, all asynchronously on `stream`. */
+/* Same step with HOST buffers, asynchronous on `stream` (out_host is valid once the stream has been synchronised).
+ * Pinned buffers the device can address (cudaHostAlloc / cudaHostRegister, 16-byte aligned) are read and written by
+ * the kernels directly across the bus, with no copies; any other host memory is copied to staging space inside the
+ * arena before the step and out is copied back after it. */
 corm_status_t corm_decode_step_host(corm_cache_t* cache, int32_t layer, const void* q_host, const void* k_new_host,
                                     const void* v_new_host, void* out_host, void* stream);
 

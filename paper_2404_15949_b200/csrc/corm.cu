@@ -408,6 +408,22 @@ corm_status_t corm_decode_step_host(corm_cache_t* c, int32_t layer, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->cfg.head_dim * c->e;
     const size_t kb = (size_t)c->U * c->cfg.head_dim * c->e;
+    // Pinned, mapped host buffers are handed to the kernels as they are: each unit's 256-byte query, key and value
+    // rows cross the bus from inside the launch and the outputs are written straight to the host, so a step needs
+    // no copy engine work at all. Any other host memory goes through the staging buffers of the arena.
+    {
+        const void* in[3] = {q_host, k_new_host, v_new_host};
+        void* dev[4] = {nullptr, nullptr, nullptr, nullptr};
+        bool mapped = true;
+        for (int i = 0; i < 4 && mapped; ++i) {
+            const void* h = i < 3 ? in[i] : out_host;
+            cudaPointerAttributes at{};
+            if (cudaPointerGetAttributes(&at, h) != cudaSuccess) { (void)cudaGetLastError(); mapped = false; break; }
+            mapped = at.type == cudaMemoryTypeHost && at.devicePointer && reinterpret_cast<uintptr_t>(at.devicePointer) % 16 == 0;
+            dev[i] = at.devicePointer;
+        }
+        if (mapped) return launch_decode(c, layer, dev[0], dev[1], dev[2], dev[3], st);
+    }
     unsigned char *dq = c->arena + c->lay.stage_q, *dk = c->arena + c->lay.stage_k, *dv = c->arena + c->lay.stage_v,
                   *dout = c->arena + c->lay.stage_out;
     CORM_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st));
