@@ -179,7 +179,10 @@ def test_wide_window_import_roundtrip():
         assert_states_equal(gpu, orc, 0, 1, 2, f"step {s}")
 
 
-def test_host_buffer_entry_point_matches_device_one():
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned-in-place", "pageable-staged"])
+def test_host_buffer_entry_point_matches_device_one(pinned):
+    """Pinned buffers are read and written by the kernels in place; pageable ones go through the arena's staging
+    space. Either way the step equals the device-buffer call bit for bit."""
     cfg = CONFIGS[1].with_(prompt_min=130, prompt_max=130, steps=10, dtype="bf16")
     data = generate(cfg)
     a, b = make_gpu_cache(cfg, 1, 8), make_gpu_cache(cfg, 1, 8)
@@ -187,13 +190,20 @@ def test_host_buffer_entry_point_matches_device_one():
     for g in (a, b):
         g.corm_compress_prompt(0, to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt),
                                data.prompt_lens)
-    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).pin_memory()
+
+    def host(x):
+        t = torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16)
+        return t.pin_memory() if pinned else t
+
     for s in range(cfg.steps):
         ref = a.corm_decode_step(0, to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt))
-        out = torch.empty(ref.shape, dtype=torch.bfloat16).pin_memory()
-        b.corm_decode_step_host(0, pin(data.q[s]), pin(data.k_new[s]), pin(data.v_new[s]), out)
+        out = host(np.zeros(tuple(ref.shape), dtype=np.float32))
+        b.corm_decode_step_host(0, host(data.q[s]), host(data.k_new[s]), host(data.v_new[s]), out)
         torch.cuda.synchronize()
         assert torch.equal(ref.cpu(), out)
+    for h in range(8):
+        sa, sb = sorted_state(a.corm_cache_export_state(0, 0, h)), sorted_state(b.corm_cache_export_state(0, 0, h))
+        assert all(np.array_equal(sa[k], sb[k]) for k in ("k", "v", "word", "pos"))
 
 
 def test_capacity_overflow_is_reported_not_fatal():
