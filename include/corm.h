@@ -67,8 +67,6 @@ typedef struct {
     int64_t moved_rows;                              /* rows copied by hole-filling compaction so far */
     int64_t attended_keys;                           /* sum over decode steps and units of the live length read */
     int32_t device_status;                           /* first device-side error (corm_status_t), CORM_OK if none */
-    int64_t redone_units;                            /* unit-steps whose verdicts needed the exact fp64 redo (see
-                                                        corm_cache_set_bound_scale) */
 } corm_stats_t;
 
 /* Bytes of device memory a cache with this configuration needs (host, pure). 0 if the configuration is invalid. */
@@ -163,12 +161,6 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Number of kernels this library has launched on behalf of `cache` since create. */
-/* The bf16/head_dim-128 kernels form the logits of grouped query heads (n_q_heads > n_kv_heads) in fp32 and decide
- * a verdict from them only where a proven bound on the fp32 error allows it; units with an undecided key are redone
- * in fp64 by one more launch, so results never depend on this. `scale` >= 1 multiplies the bound (default 1): larger
- * values send more units through the redo, which is how the tests exercise it. Errors: INVALID_ARG. */
-corm_status_t corm_cache_set_bound_scale(corm_cache_t* cache, double scale);
-
 int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
 
 const char* corm_status_string(corm_status_t status);

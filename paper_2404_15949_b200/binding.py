@@ -29,8 +29,7 @@ class CormConfig(ctypes.Structure):
 class CormStats(ctypes.Structure):
     _fields_ = [("live_keys", ctypes.c_int64), ("appended_keys", ctypes.c_int64), ("evicted_keys", ctypes.c_int64),
                 ("retention", ctypes.c_double), ("kv_bytes_live", ctypes.c_int64), ("aux_bytes_live", ctypes.c_int64),
-                ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32),
-                ("redone_units", ctypes.c_int64)]
+                ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32)]
 
 
 class CormError(RuntimeError):
@@ -79,8 +78,6 @@ def load_library():
     lib.corm_cache_import_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.corm_cache_set_tuning.restype = i32
     lib.corm_cache_set_tuning.argtypes = [vp, i32, i32]
-    lib.corm_cache_set_bound_scale.restype = ctypes.c_int
-    lib.corm_cache_set_bound_scale.argtypes = [vp, ctypes.c_double]
     lib.corm_cache_kernel_launches.restype = i64
     lib.corm_cache_kernel_launches.argtypes = [vp]
     lib.corm_status_string.restype = ctypes.c_char_p
@@ -200,11 +197,6 @@ class CormCache:
 
     def corm_cache_set_tuning(self, split_len=0, allow_fast_path=True):
         _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
-
-    def corm_cache_set_bound_scale(self, scale):
-        """Multiplies the proven fp32 error bound of the grouped-query kernels (>= 1; results never change, only how
-        many units take the exact fp64 redo)."""
-        _check("corm_cache_set_bound_scale", self.lib.corm_cache_set_bound_scale(self.handle, float(scale)))
 
     def corm_cache_kernel_launches(self):
         return int(self.lib.corm_cache_kernel_launches(self.handle))

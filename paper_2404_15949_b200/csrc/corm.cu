@@ -14,7 +14,6 @@
 #include "../../include/corm.h"
 #include "corm_common.cuh"
 #include "corm_fast.cuh"
-#include "corm_redo.cuh"
 #include "corm_generic.cuh"
 #include "corm_prompt_fast.cuh"
 
@@ -28,7 +27,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, redo_flag, counters, status, maxlive, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -69,7 +68,6 @@ Layout make_layout(const corm_config_t& c) {
     L.base_tokens = take(Ltot * c.batch * 4);
     L.base_obs = take(Ltot * c.batch * 4);
     L.ticket = take(Ltot * U * 4);
-    L.redo_flag = take(U * 4);
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
@@ -118,7 +116,6 @@ struct corm_cache {
     std::vector<cudaEvent_t> readback_ev;
     std::vector<int> readback_pending, last_readback_step;
     int tune_split_len = 0, allow_fast = 1;
-    double delta_scale = 1.0;
     int sm_count = 148;
     long long launches = 0;
 };
@@ -197,8 +194,6 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.partials = c->arena + c->lay.partials;
     p.keepmask = reinterpret_cast<uint32_t*>(c->arena + c->lay.keepmask);
-    p.redo_flag = reinterpret_cast<int32_t*>(c->arena + c->lay.redo_flag);
-    p.delta_scale = c->delta_scale;
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
     p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
@@ -561,7 +556,6 @@ corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* st
         s.evicted_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_EVICTED];
         s.moved_rows += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_MOVED];
         s.attended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_ATTENDED];
-        s.redone_units += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_REDONE];
     }
     s.retention = s.appended_keys ? (double)s.live_keys / (double)s.appended_keys : 1.0;
     s.kv_bytes_live = s.live_keys * 2 * c->cfg.head_dim * (int64_t)c->e;
@@ -633,12 +627,6 @@ corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t 
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
     c->allow_fast = allow_fast_path ? 1 : 0;
-    return CORM_OK;
-}
-
-corm_status_t corm_cache_set_bound_scale(corm_cache_t* c, double scale) {
-    if (!c || !(scale >= 1.0) || !std::isfinite(scale)) return CORM_ERR_INVALID_ARG;
-    c->delta_scale = scale;
     return CORM_OK;
 }
 

@@ -36,15 +36,8 @@ inline cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
     return e;
 }
 
-// |fp32 dot - exact dot| <= kDotErr * |q| * |k| for the fast kernels' fp32 logits (bf16 x bf16 products are exact in
-// fp32): 7 roundings in a lane's 8-term FMA chain and 5 in the cross-lane fold make 12 * 2^-24 to first order;
-// 16 * 2^-24 leaves a third of slack for the higher-order terms and for the rounding of the fp32 key norm itself.
-constexpr double kDotErr = 16.0 / 16777216.0;
-// 1 / sqrt(head_dim), the scale of Eq. 2's exponent
-__host__ __device__ constexpr double inv_root_dim(int D) { return D == 128 ? 0.088388347648318440550 : 0.125; }
-
 // Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
-enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_REDONE = 4, CNT_COUNT = 5 };
+enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_COUNT = 4 };
 
 struct DecodeParams {
     void* K;                  // [U][C][D] this layer's key slabs
@@ -62,7 +55,6 @@ struct DecodeParams {
     double* stash;            // [U*G][C] scaled logits of this step (scratch)
     unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
     uint32_t* keepmask;       // [U][ceil(C/32)+2] keep bits of the verdict launch (scratch)
-    int32_t* redo_flag;       // [U] step + 1 of the last step whose fp32 logits could not certify every verdict (scratch)
     const void* q;            // [B][Hq][D]
     const void* k_new;        // [B][Hkv][D]
     const void* v_new;        // [B][Hkv][D]
@@ -70,7 +62,6 @@ struct DecodeParams {
     int32_t U, Hkv, C, split_len, max_splits, step, w, r;
     int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
     double log_alpha;         // ln(alpha), -inf for alpha = 0
-    double delta_scale;       // multiplies the certified fp32 error bound (1; tests raise it to force the exact redo)
 };
 
 struct PromptParams {
@@ -91,9 +82,7 @@ struct PromptParams {
     double log_alpha;
 };
 
-// split record: {double m, double Z, float acc[D], float kmax2, float qn2, 8 bytes unused}; the last two (largest
-// squared key norm of the split, squared query norm) are only written by the kernels that form fp32 logits
-__host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D + 16; }
+__host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D; }
 
 // ---- element access: the cache dtype is only a storage format; all logits are formed in fp64 ----
 struct bf16_t { uint16_t bits; };
@@ -160,10 +149,6 @@ __device__ __forceinline__ uint32_t window_mask(int w) { return w >= 32 ? 0xffff
 // then t_now - stamp < w, which selects exactly the columns Algorithm 1's any() over the last w rows selects.
 __device__ __forceinline__ uint32_t update_register(uint32_t old, bool imp, int w, int t) {
     return w <= 32 ? (((old << 1) | (imp ? 1u : 0u)) & window_mask(w)) : (imp ? (uint32_t)t : old);
-}
-// Corrects the newest verdict of a register that update_register(old, false-or-true, w, t) produced this step.
-__device__ __forceinline__ uint32_t patch_register(uint32_t reg, bool imp, int w, int t) {
-    return w <= 32 ? ((reg & ~1u) | (imp ? 1u : 0u)) : (imp ? (uint32_t)t : reg);
 }
 __device__ __forceinline__ bool register_needed(uint32_t reg, int w, int t) {
     return w <= 32 ? reg != 0u : (reg != 0u && t - (int)reg < w);
@@ -259,10 +244,7 @@ __device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, i
 //   3. once w rows exist: keep iff register != 0 or position > t - r; holes below the new length are filled with
 //      kept rows from above it (as many row copies as there are holes; sources and destinations are disjoint)
 // smem: 2*(ceil(C/32)+2) 32-bit words of dynamic shared memory.
-// kPatch: the outputs and speculative registers of this step already exist (written from certified fp32 logits, with
-// a 0 verdict wherever the bound could not decide); the logits and records now hold exact fp64 values, and step 2
-// only corrects the newest verdict of each register: bit 0, or the stamp when the window is wider than 32.
-template <typename T, int D, int G, int NT, bool kPatch = false>
+template <typename T, int D, int G, int NT>
 __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_act, int t, unsigned char* smem) {
     __shared__ double s_thr[G];
     __shared__ int s_scan[NT];
@@ -300,12 +282,10 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
             }
         }
         T* outp = reinterpret_cast<T*>(p.out) + ((size_t)u * G + g) * D;
-        if (!kPatch) {
 #pragma unroll
-            for (int i = 0; i < (D + NT - 1) / NT; ++i) {
-                const int c = tid + i * NT;
-                if (c < D) Elem<T>::store(outp + c, (float)((double)acc[i] / Z));
-            }
+        for (int i = 0; i < (D + NT - 1) / NT; ++i) {
+            const int c = tid + i * NT;
+            if (c < D) Elem<T>::store(outp + c, (float)((double)acc[i] / Z));
         }
         if (tid == 0) s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);
     }
@@ -342,7 +322,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 bool imp = false;
 #pragma unroll
                 for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
-                const uint32_t wd = kPatch ? patch_register(wv[k], imp, p.w, t) : update_register(wv[k], imp, p.w, t);
+                const uint32_t wd = update_register(wv[k], imp, p.w, t);
                 wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
             }

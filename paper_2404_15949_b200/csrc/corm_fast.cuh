@@ -38,13 +38,9 @@ __host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? CO
 // 228 KB per SM, minus 1 KB the system reserves per block and ~1.2 KB of static shared memory
 __host__ __device__ constexpr int fast_smem_budget(int G) { return (228 * 1024) / fast_blocks_per_sm(G) - 2304; }
 constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits (about 2 s)
-// Groups of several query heads form their logits in fp32 (bf16 x bf16 products are exact there) with a certified
-// bound on the accumulation error; the verdict launch decides every key the bound allows and flags the unit for an
-// exact fp64 redo otherwise. One query head per KV head keeps fp64 logits throughout.
-__host__ __device__ constexpr bool fast_f32_logits(int G) { return G > 1; }
-// longest unit that may finish inside one block (bounded by the registers that carry its verdict words); units with
-// fp32 logits always go through the verdict launch
-__host__ __device__ constexpr int fast_max_single_cap(int G) { return G == 1 ? 8 * kFastThreads : 0; }
+// longest unit that may finish inside one block (bounded by the registers that carry its verdict words)
+__host__ __device__ constexpr int fast_max_single_cap(int G) { return (G == 1 ? 8 : 2) * kFastThreads; }
+
 inline bool fast_path_available() { return true; }
 
 // ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
@@ -193,49 +189,6 @@ __device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double
     for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
 }
 
-// fp32 form of qk_tile for groups of query heads, same key order and fold. Also returns the squared norm of the
-// lane's key (the error bound of a logit is proportional to |q| |k|).
-template <int G>
-__device__ __forceinline__ void qk_tile32(const unsigned char* ktile, const float (&qf)[G][8], int lane,
-                                          float (&sown)[G], float& n2own) {
-    const int h = lane >> 4, i = lane & 15, m = i >> 1, b0 = i & 1;
-    float r[2][G + 1];
-#pragma unroll
-    for (int it = 0; it < 2; ++it) {
-        float a[G + 1][8];
-#pragma unroll
-        for (int s = 0; s < 8; ++s) {
-            const int key = 16 * h + 8 * (it ^ b0) + (s ^ m);
-            const uint4 raw = *reinterpret_cast<const uint4*>(ktile + key * kRowBytes + i * 16);
-            float kf[8];
-            unpack8_to_float(raw, kf);
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float acc = qf[g][0] * kf[0];
-#pragma unroll
-                for (int e = 1; e < 8; ++e) acc = fmaf(qf[g][e], kf[e], acc);
-                a[g][s] = acc;
-            }
-            float nn = kf[0] * kf[0];
-#pragma unroll
-            for (int e = 1; e < 8; ++e) nn = fmaf(kf[e], kf[e], nn);
-            a[G][s] = nn;
-        }
-#pragma unroll
-        for (int g = 0; g <= G; ++g) {
-#pragma unroll
-            for (int s = 0; s < 4; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 4], 8);
-#pragma unroll
-            for (int s = 0; s < 2; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 2], 4);
-            a[g][0] += __shfl_xor_sync(0xffffffffu, a[g][1], 2);
-            r[it][g] = a[g][0];
-        }
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
-    n2own = r[0][G] + __shfl_xor_sync(0xffffffffu, r[1][G], 1);
-}
-
 // Single-split finalize: logits, registers and positions of the whole unit are in shared memory.
 // lists: scratch for the keep mask, its prefix sums and the hole / mover lists (ints).
 // wv / pv: registers and positions of slots tid, tid + NT, ... (loaded by the caller at block start).
@@ -303,7 +256,6 @@ template <int G>
 __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_failed;
-    __shared__ unsigned s_kmax2_bits;
     __shared__ double s_thr1[G];
     constexpr int NT = kFastThreads, NW = kFastWarps;
     constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
@@ -334,7 +286,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
 
-    if (tid == 0) { s_failed = 0; s_kmax2_bits = 0u; }
+    if (tid == 0) s_failed = 0;
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kStagesPerWarp; ++s) mbar_init(my_bars + s * 8, 1);
@@ -366,7 +318,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
     // queries widened to fp64 once per block; a single-split unit also fetches the registers and positions of the
     // slots this thread will judge in the finalize phase (slots tid, tid + NT, ...) and keeps them in registers
-    constexpr int kPre = fast_max_single_cap(G) / NT > 0 ? fast_max_single_cap(G) / NT : 1;
+    constexpr int kPre = fast_max_single_cap(G) / NT;
     uint32_t wv[kPre];
     int32_t pv[kPre];
 #pragma unroll
@@ -387,18 +339,11 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
     const int h = lane >> 4, ci = lane & 15;
     const int key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);     // tile key this lane owns after the fold
-    constexpr bool kF32 = fast_f32_logits(G);
-    double qd[kF32 ? 1 : G][8];                                  // the lane's 8 channels of every query head
-    float qf[kF32 ? G : 1][8];
+    double qd[G][8];
 #pragma unroll
     for (int g = 0; g < G; ++g)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            if constexpr (kF32) qf[g][e] = (float)qs[g * 128 + ci * 8 + e];      // exact: the queries are bf16
-            else qd[g][e] = qs[g * 128 + ci * 8 + e];
-        }
-    float kmax2 = 0.f;                                           // largest squared key norm this lane has seen
-    float* stash32 = reinterpret_cast<float*>(p.stash) + (size_t)u * 2 * G * p.C;   // [G + 1][C]: raw fp32 dots, key norms
+        for (int e = 0; e < 8; ++e) qd[g][e] = qs[g * 128 + ci * 8 + e];
     double M[G], Zl[G];
     unsigned long long acc2[G][4];                                // P.V accumulators: channel pairs (2e, 2e+1) of this lane's 8
 #pragma unroll
@@ -429,14 +374,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             __syncwarp();
         }
         double sown[G];
-        float sown32[kF32 ? G : 1], n2own = 0.f;
-        if constexpr (kF32) {
-            qk_tile32<G>(ktile, qf, lane, sown32, n2own);
-#pragma unroll
-            for (int g = 0; g < G; ++g) sown[g] = (double)sown32[g];
-        } else {
-            qk_tile<G>(ktile, qd, lane, sown);
-        }
+        qk_tile<G>(ktile, qd, lane, sown);
         __syncwarp();
         if (lane == 0 && it + kKStages < my_n) { fence_async_smem(); issue_k(it + kKStages); }
 
@@ -468,13 +406,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             M[g] = Mn[g];
             psm[key_own * G + g] = (float)ex[g];
             if (valid) {
-                if constexpr (kF32) stash32[(size_t)g * p.C + j_own] = sown32[g];
-                else if (single) stash_sm[g * p.single_cap + j_own] = sv[g];
+                if (single) stash_sm[g * p.single_cap + j_own] = sv[g];
                 else p.stash[((size_t)u * G + g) * p.C + j_own] = sv[g];
             }
-        }
-        if constexpr (kF32) {
-            if (valid) { stash32[(size_t)G * p.C + j_own] = n2own; kmax2 = fmaxf(kmax2, n2own); }
         }
         if (moved) {                                                       // warp-uniform
 #pragma unroll
@@ -529,14 +463,8 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], 16);
     }
-    if constexpr (kF32) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) kmax2 = fmaxf(kmax2, __shfl_xor_sync(0xffffffffu, kmax2, o));
-        if (lane == 0) atomicMax(&s_kmax2_bits, __float_as_uint(kmax2));   // non-negative floats order like their bits
-    }
     __syncthreads();                       // every warp is done with its tiles: the tile area becomes scratch
     if (s_failed) return;                  // a bounded wait expired: reported through the status word, unit left as is
-    const float s_kmax2 = __uint_as_float(s_kmax2_bits);
     unsigned char* merge = smem + lay.tiles;                      // [NW][G] records {double M, double Z, float acc[128]}
     constexpr int kRec = 16 + 4 * 128;
 #pragma unroll
@@ -579,17 +507,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             else {
                 unsigned char* rec = p.partials + (((size_t)u * p.max_splits + split) * G + g) * pstride;
                 reinterpret_cast<double*>(rec)[0] = Mb; reinterpret_cast<double*>(rec)[1] = Zb;
-                if constexpr (kF32) {                          // what the verdict launch needs for the error bound
-                    double qn2 = 0.0;
-                    for (int c = 0; c < 128; ++c) qn2 = fma(qs[g * 128 + c], qs[g * 128 + c], qn2);
-                    float* tail = reinterpret_cast<float*>(rec + 16 + 4 * 128);
-                    tail[0] = s_kmax2;
-                    tail[1] = (float)(qn2 * (1.0 + 1e-6));      // rounded up
-                }
             }
         }
     }
-    if constexpr (!fast_f32_logits(G)) if (single) {
+    if (single) {
         __syncthreads();
         unsigned char* lists = merge + NW * G * kRec;
         int* holes = reinterpret_cast<int*>(lists + 2 * ((l + 31) / 32 + 2) * 4);
@@ -599,8 +520,6 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     // a unit of several splits: its partial records and logits are complete once this launch ends; the verdict
     // launch that follows takes Algorithm 1 from there
 }
-
-inline corm_status_t launch_redo(DecodeParams& p, int G, int n_splits, cudaStream_t st, int* n_launched);   // corm_redo.cuh
 
 // Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
 inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int tune_split_len, int sm_count,
@@ -669,12 +588,10 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: verdict launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;
     };
-    rc = G == 1 ? launch_v(decode_verdict_kernel<bf16_t, 128, 1, false>)
-       : G == 2 ? launch_v(decode_verdict_kernel<bf16_t, 128, 2, true>) : launch_v(decode_verdict_kernel<bf16_t, 128, 4, true>);
-    if (rc != CORM_OK) return rc;
-    *n_launched = 2;
-    if (!fast_f32_logits(G)) return CORM_OK;
-    return launch_redo(p, G, n_splits, st, n_launched);
+    rc = G == 1 ? launch_v(decode_verdict_kernel<bf16_t, 128, 1>) : G == 2 ? launch_v(decode_verdict_kernel<bf16_t, 128, 2>)
+                                                                           : launch_v(decode_verdict_kernel<bf16_t, 128, 4>);
+    if (rc == CORM_OK) *n_launched = 2;
+    return rc;
 }
 
 }  // namespace corm

@@ -28,17 +28,11 @@ __host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G) {
     return (size_t)G * n_splits * (8 + 8 + 4) + 16 + (size_t)2 * keepmask_words(C) * 4;
 }
 
-// kF32: the streaming kernel left raw fp32 dot products and squared key norms instead of fp64 logits. A logit is then
-// known to within e_j = kDotErr |q| |k_j| / sqrt(D), and lse (a 1-Lipschitz function of the logits in the sup norm) to
-// within max_j e_j, so [s_j >= thr] is certain whenever |s_j - thr| >= e_j + max_j e_j. A key is important as soon
-// as one head says so with certainty; it is undecided when no head does and some head is uncertain. Undecided keys
-// get a 0 verdict for now and flag the unit: its compaction is left to the exact fp64 redo launch that follows.
-template <typename T, int D, int G, bool kF32>
+template <typename T, int D, int G>
 __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
                                                                          const int n_splits) {
     extern __shared__ __align__(128) unsigned char smem[];
-    __shared__ double s_thr[G], s_Z[G], s_err[G];     // s_err[g] = scale * kDotErr * |q_g| / sqrt(D)
-    __shared__ float s_kmax;                          // largest key norm of the unit
+    __shared__ double s_thr[G], s_Z[G];
     __shared__ int s_scan[kVerdictThreads];
     __shared__ int s_last;
     constexpr int NT = kVerdictThreads, kListCap = 512;
@@ -69,22 +63,12 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     // everything this block needs from the streaming kernel is requested at once: status, split records, logits
     const int status = __ldcg(p.status);
     const double* stash_u = p.stash + (size_t)u * G * p.C;
-    const float* stash32 = reinterpret_cast<const float*>(stash_u);       // kF32: [G + 1][C] raw dots, squared key norms
     double sv[kVerdictPer][G];
-    float kn2[kVerdictPer];
-    constexpr double inv_root_d = inv_root_dim(D);
 #pragma unroll
     for (int k = 0; k < kVerdictPer; ++k) {
         const int j = base0 + k * NT + tid;
-        kn2[k] = 0.f;
-        if constexpr (kF32) {
 #pragma unroll
-            for (int g = 0; g < G; ++g) sv[k][g] = j < l ? (double)__ldcg(stash32 + (size_t)g * p.C + j) * inv_root_d : -INFINITY;
-            if (j < l) kn2[k] = __ldcg(stash32 + (size_t)G * p.C + j);
-        } else {
-#pragma unroll
-            for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
-        }
+        for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
     }
 
     double* sm_m = reinterpret_cast<double*>(smem);                        // [G][n_splits]
@@ -121,23 +105,10 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
             s_Z[g] = Z;
             s_thr[g] = m + log(Z) + p.log_alpha - log((double)t);         // Definition 3.1: s >= lse + ln(alpha) - ln(t)
         }
-        if constexpr (kF32) {
-            float km = 0.f;                                                // record tails: {kmax2, qn2}
-            for (int s = lane; s < n_act; s += 32)
-                km = fmaxf(km, __ldcg(reinterpret_cast<const float*>(rec_u + ((size_t)s * G + g) * pstride + 16 + 4 * D)));
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) km = fmaxf(km, __shfl_xor_sync(0xffffffffu, km, o));
-            if (lane == 0) {
-                const float qn2 = __ldcg(reinterpret_cast<const float*>(rec_u + (size_t)g * pstride + 16 + 4 * D) + 1);
-                s_err[g] = p.delta_scale * kDotErr * inv_root_d * sqrt((double)qn2) * (1.0 + 1e-6);
-                if (g == 0) s_kmax = (float)(sqrt((double)km) * (1.0 + 1e-6));
-            }
-        }
     }
     __syncthreads();
     // b. verdicts, register update, keep flags of this block's slots
     uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
-    bool undecided = false;
     {
 #pragma unroll
         for (int k = 0; k < kVerdictPer; ++k) {
@@ -146,20 +117,8 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
             bool keep = false;
             if (j < l) {
                 bool imp = false;
-                if constexpr (kF32) {
-                    const double kn = sqrt((double)kn2[k]) * (1.0 + 1e-6) + (double)s_kmax;
-                    bool unsure = false;
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        const double margin = sv[k][g] - s_thr[g], err = s_err[g] * kn;
-                        imp |= (margin >= err);
-                        unsure |= !(margin >= err) && !(margin < -err);
-                    }
-                    undecided |= (!imp && unsure);
-                } else {
-#pragma unroll
-                    for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
-                }
+                for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
                 const uint32_t wd = update_register(wv[k], imp, p.w, t);
                 wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
@@ -168,8 +127,6 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
             if (lane == 0 && base + warp * 32 < l) keep_g[(base >> 5) + warp] = ballot;
         }
     }
-
-    if (kF32 && undecided) p.redo_flag[u] = 1;                             // any thread: the redo launch takes the unit over
 
     // c. the last block of the unit to get here compacts it
     __threadfence();
@@ -201,7 +158,6 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
         }
     }
     if (!s_last) return;
-    if (kF32 && __ldcg(p.redo_flag + u) != 0) return;                      // every block's flag write precedes its arrival
     int new_len = l, n_moved = 0;
     if (evict_on) {
         const int nwords = (l + 31) / 32;
