@@ -394,29 +394,31 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             for (int g = 0; g < G; ++g) mt[g] = fmaxf(mt[g], __shfl_xor_sync(0xffffffffu, mt[g], o));
 #pragma unroll
         for (int g = 0; g < G; ++g) Mn[g] = fmax(M[g], (double)mt[g]);   // new reference: warp-uniform, >= every logit so far (up to fp32 rounding)
-#pragma unroll
-        for (int g = 0; g < G; ++g) sc[g] = exp_nonpos(M[g] - Mn[g]);    // exactly 1 when the reference did not move
-#pragma unroll
-        for (int g = 0; g < G; ++g) ex[g] = valid ? exp_nonpos(sv[g] - Mn[g]) : 0.0;
         bool moved = false;
 #pragma unroll
+        for (int g = 0; g < G; ++g) moved |= (Mn[g] != M[g]);
+        if (moved) {                                                       // warp-uniform; rare after the first tiles
+#pragma unroll
+            for (int g = 0; g < G; ++g) sc[g] = exp_nonpos(M[g] - Mn[g]);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                Zl[g] *= sc[g];
+                const float scf = (float)sc[g];
+                const unsigned long long sc2 = pack_f32x2(scf, scf);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) mul_f32x2(acc2[g][e], sc2);
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) ex[g] = valid ? exp_nonpos(sv[g] - Mn[g]) : 0.0;
+#pragma unroll
         for (int g = 0; g < G; ++g) {
-            moved |= (Mn[g] != M[g]);
-            Zl[g] = fma(Zl[g], sc[g], ex[g]);
+            Zl[g] += ex[g];
             M[g] = Mn[g];
             psm[key_own * G + g] = (float)ex[g];
             if (valid) {
                 if (single) stash_sm[g * p.single_cap + j_own] = sv[g];
                 else p.stash[((size_t)u * G + g) * p.C + j_own] = sv[g];
-            }
-        }
-        if (moved) {                                                       // warp-uniform
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float scf = (float)sc[g];
-                const unsigned long long sc2 = pack_f32x2(scf, scf);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) mul_f32x2(acc2[g][e], sc2);
             }
         }
         __syncwarp();
