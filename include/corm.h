@@ -156,8 +156,11 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
                                       const int32_t* pos_host, int32_t live_len, int32_t n_tokens, int32_t n_obs,
                                       void* stream);
 
-/* Tuning knobs (performance only; results do not depend on them): keys per split of the decode kernel
- * (multiple of 32, 0 = automatic) and whether the fast bf16/head_dim-128 kernel may be used. */
+/* Tuning knobs (performance only; live lists and registers do not depend on them, outputs only within rounding):
+ * keys per split of the decode kernel (multiple of 32, 0 = automatic) and which kernels may be used:
+ * allow_fast_path 0 = the generic kernels only; 1 = the bf16/head_dim-128 kernels (default), which finish a unit
+ * of several splits inside the decode launch when the launch has many units and by a second, verdict launch when
+ * it has few; 2 / 3 = those kernels with the first / the second way always. Errors: INVALID_ARG. */
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Number of kernels this library has launched on behalf of `cache` since create. */

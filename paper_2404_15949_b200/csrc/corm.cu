@@ -204,7 +204,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     corm_status_t rc;
     int n_launched = 1;
     if (fast) {
-        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st, &n_launched);
+        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
         const int n_splits = (upper + p.split_len - 1) / p.split_len;
@@ -626,7 +626,8 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
 corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
-    c->allow_fast = allow_fast_path ? 1 : 0;
+    if (allow_fast_path < 0 || allow_fast_path > 3) return CORM_ERR_INVALID_ARG;
+    c->allow_fast = allow_fast_path;
     return CORM_OK;
 }
 

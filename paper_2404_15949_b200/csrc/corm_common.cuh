@@ -61,6 +61,7 @@ struct DecodeParams {
     void* out;                // [B][Hq][D]
     int32_t U, Hkv, C, split_len, max_splits, step, w, r;
     int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
+    int32_t inline_finalize;  // fast kernel: the last-arriving split of a longer unit finishes it (else the verdict launch does)
     double log_alpha;         // ln(alpha), -inf for alpha = 0
 };
 

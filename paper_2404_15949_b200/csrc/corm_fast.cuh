@@ -256,6 +256,7 @@ template <int G>
 __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_failed;
+    __shared__ int s_last;
     __shared__ double s_thr1[G];
     constexpr int NT = kFastThreads, NW = kFastWarps;
     constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
@@ -519,13 +520,27 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l);
         return;
     }
-    // a unit of several splits: its partial records and logits are complete once this launch ends; the verdict
-    // launch that follows takes Algorithm 1 from there
+    // A unit of several splits: its partial records and logits are complete once every split is done. With many
+    // units in flight the split that arrives last finishes the unit right here (its serial walk over the unit hides
+    // behind the other units' streaming); with few units that walk would be the tail of the launch, and the verdict
+    // launch that follows spreads it over many blocks instead.
+    if (!p.inline_finalize) return;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned prev = atomicAdd(p.ticket + u, 1u);
+        s_last = (prev == (unsigned)(n_act - 1));
+        if (s_last) p.ticket[u] = 0u;
+        __threadfence();
+    }
+    __syncthreads();
+    if (!s_last) return;
+    finalize_unit<bf16_t, 128, G, NT>(p, u, b, l, n_act, t, smem);
 }
 
 // Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
 inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int tune_split_len, int sm_count,
-                                        cudaStream_t st, int* n_launched) {
+                                        cudaStream_t st, int* n_launched, int finish_mode) {
     *n_launched = 0;
     if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
     // longest unit that can finish inside one block: bounded by the verdict registers a thread carries and by the
@@ -554,6 +569,11 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     p.single_cap = split_len < cap ? split_len : cap;
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
     const size_t smem = (size_t)lay.total;
+    const bool all_single = n_splits == 1 && upper <= p.single_cap;      // every unit finishes inside its one block
+    // who finishes the longer units: see the end of decode_fast_kernel
+    const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // keep mask + prefix sums of finalize_unit
+    const bool many = finish_mode == 2 || (finish_mode != 3 && (long long)p.U * n_splits >= 4ll * sms * fast_blocks_per_sm(G));
+    p.inline_finalize = !all_single && many && fin <= smem;
     const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
                         (size_t)2 * p.single_cap * 4;
     if (fin1 > (size_t)kFastWarps * fast_warp_bytes(G)) return CORM_ERR_UNSUPPORTED;
@@ -569,7 +589,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     corm_status_t rc = G == 1 ? launch(decode_fast_kernel<1>) : G == 2 ? launch(decode_fast_kernel<2>) : launch(decode_fast_kernel<4>);
     if (rc != CORM_OK) return rc;
     *n_launched = 1;
-    if (n_splits == 1 && upper <= p.single_cap) return CORM_OK;          // every unit finishes inside the streaming kernel
+    if (all_single || p.inline_finalize) return CORM_OK;
     // verdict launch for the units that do not
     const size_t vsmem = verdict_smem(p.C, n_splits, G);
     auto launch_v = [&](auto kern) -> corm_status_t {

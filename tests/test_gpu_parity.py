@@ -45,8 +45,11 @@ def test_config1_other_seeds(seed):
 SMALL = [
     # dtype, head_dim, group, n_kv, batch, prompt range, steps, w, r, split_len, fast
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, True),
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, 2),      # units of several splits finished inside the decode launch
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, 3),      # ... by the verdict launch
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, False),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True),
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, 2),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, False),
     ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True),
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 64, True),
