@@ -305,6 +305,7 @@ def main():
         "retention": st2["retention"],
         "live_keys_per_unit": st2["live_keys"] / (L * cfg.batch * cfg.n_kv_heads),
         "evicted_keys_timed": st2["evicted_keys"] - st1["evicted_keys"], "moved_rows_timed": moved,
+        "important_key_fraction_timed": (st2["important_keys"] - st1["important_keys"]) / max(1, attended),
         "prompt_pass_ms": prompt_ms, "retention_after_prompt": st0["retention"],
         "paper_context": "paper reports KV memory only: up to 70% reduction (V100-32GB / A100-80GB), no throughput",
     }

@@ -67,6 +67,9 @@ typedef struct {
     int64_t moved_rows;                              /* rows copied by hole-filling compaction so far */
     int64_t attended_keys;                           /* sum over decode steps and units of the live length read */
     int32_t device_status;                           /* first device-side error (corm_status_t), CORM_OK if none */
+    int64_t important_keys;                          /* sum over decode steps and units of the keys judged important
+                                                        (Definition 3.1, OR over the group): important_keys /
+                                                        attended_keys is the sparsity figure of Section 3.1 */
 } corm_stats_t;
 
 /* Bytes of device memory a cache with this configuration needs (host, pure). 0 if the configuration is invalid. */

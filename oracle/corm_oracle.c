@@ -41,6 +41,7 @@ typedef struct {
     int     *t;      /* [L*B]                tokens seen                      */
     int     *n_obs;  /* [L*B]                verdict rows recorded            */
     long long appended, evicted, verdict_evals, near_threshold;
+    long long important, judged; /* decode steps only: keys judged important / keys judged (the sparsity of Section 3.1) */
     double  near_rel; /* half-width of the reported band around the threshold, relative */
 } corm_oracle;
 
@@ -164,8 +165,8 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
     for (int b = 0; b < B; ++b)
         for (int h = 0; h < Hkv; ++h)
             if (o->live[unit_index(o, layer, b, h)] + 1 > o->max_tokens) return ORACLE_CAPACITY;
-    long long evals_total = 0, near_total = 0, appended = 0, evicted = 0;
-#pragma omp parallel for collapse(2) schedule(dynamic) reduction(+ : evals_total, near_total, appended, evicted)
+    long long evals_total = 0, near_total = 0, appended = 0, evicted = 0, important_total = 0, judged_total = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic) reduction(+ : evals_total, near_total, appended, evicted, important_total, judged_total)
     for (int b = 0; b < B; ++b) {
         for (int h = 0; h < Hkv; ++h) {
             size_t u = unit_index(o, layer, b, h);
@@ -201,7 +202,9 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
             for (int j = 0; j < l; ++j) {                             /* newest verdict enters at bit 0 */
                 reg_shift_in(o->word + (u * C + j) * REG_WORDS, o->w, (uint32_t)imp[j]);
                 if (imp_out) imp_out[((size_t)b * Hkv + h) * C + j] = imp[j];
+                important_total += imp[j];
             }
+            judged_total += l;
             evals_total += evals; near_total += near;
             free(p); free(qv); free(imp);
             evicted += evict_unit(o, u, t, n_obs);                    /* Algorithm 1's eviction, effective next step */
@@ -216,7 +219,16 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
     o->appended += appended;
     o->verdict_evals += evals_total;
     o->near_threshold += near_total;
+    o->important += important_total;
+    o->judged += judged_total;
     return ORACLE_OK;
+}
+
+/* Section 3.1's sparsity over the decode steps so far: keys judged important (Definition 3.1, OR over the group)
+ * and keys judged. */
+void oracle_sparsity(const corm_oracle *o, long long *important, long long *judged) {
+    if (important) *important = o->important;
+    if (judged) *judged = o->judged;
 }
 
 /* Prompt-end pass for every unit of one layer.

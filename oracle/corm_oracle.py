@@ -50,6 +50,8 @@ def _load():
     lib.oracle_export_age.restype = c_int
     lib.oracle_export_age.argtypes = [vp, c_int, c_int, c_int, vp]
     lib.oracle_counters.argtypes = [vp, vp, vp, vp, vp]
+    lib.oracle_sparsity.argtypes = [vp, vp, vp]
+    lib.oracle_sparsity.restype = None
     lib.oracle_set_near_band.argtypes = [vp, c_dbl]
     _lib = lib
     return lib
@@ -147,6 +149,12 @@ class CormOracle:
         self.lib.oracle_counters(self.h, *[ctypes.byref(x) for x in vals])
         return dict(appended=vals[0].value, evicted=vals[1].value, verdict_evals=vals[2].value,
                     near_threshold=vals[3].value)
+
+    def sparsity(self):
+        """(keys judged important, keys judged) over the decode steps so far."""
+        a, b = ctypes.c_longlong(0), ctypes.c_longlong(0)
+        self.lib.oracle_sparsity(self.h, ctypes.byref(a), ctypes.byref(b))
+        return a.value, b.value
 
     def set_near_band(self, rel):
         self.lib.oracle_set_near_band(self.h, float(rel))

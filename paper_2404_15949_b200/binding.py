@@ -29,7 +29,8 @@ class CormConfig(ctypes.Structure):
 class CormStats(ctypes.Structure):
     _fields_ = [("live_keys", ctypes.c_int64), ("appended_keys", ctypes.c_int64), ("evicted_keys", ctypes.c_int64),
                 ("retention", ctypes.c_double), ("kv_bytes_live", ctypes.c_int64), ("aux_bytes_live", ctypes.c_int64),
-                ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32)]
+                ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32),
+                ("important_keys", ctypes.c_int64)]
 
 
 class CormError(RuntimeError):

@@ -556,6 +556,7 @@ corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* st
         s.evicted_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_EVICTED];
         s.moved_rows += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_MOVED];
         s.attended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_ATTENDED];
+        s.important_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_IMPORTANT];
     }
     s.retention = s.appended_keys ? (double)s.live_keys / (double)s.appended_keys : 1.0;
     s.kv_bytes_live = s.live_keys * 2 * c->cfg.head_dim * (int64_t)c->e;

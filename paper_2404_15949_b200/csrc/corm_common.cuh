@@ -37,7 +37,7 @@ inline cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
 }
 
 // Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
-enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_COUNT = 4 };
+enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_IMPORTANT = 4, CNT_COUNT = 5 };
 
 struct DecodeParams {
     void* K;                  // [U][C][D] this layer's key slabs
@@ -128,6 +128,13 @@ template <> __device__ __forceinline__ void load_slice<bf16_t, 4>(const bf16_t* 
 template <> __device__ __forceinline__ void load_slice<bf16_t, 2>(const bf16_t* p, float (&out)[2]) {
     uint32_t v = *reinterpret_cast<const uint32_t*>(p);
     out[0] = __uint_as_float(v << 16); out[1] = __uint_as_float(v & 0xffff0000u);
+}
+
+// Adds the warp's total of n to a 64-bit counter (one atomic per warp; all lanes must call).
+__device__ __forceinline__ void warp_count(unsigned long long* counter, int n) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+    if ((threadIdx.x & 31) == 0 && n) atomicAdd(counter, (unsigned long long)n);
 }
 
 __device__ __forceinline__ double warp_sum(double x) {
@@ -297,6 +304,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     const bool evict_on = n_obs >= p.w;
     const double* stash_u = p.stash + (size_t)u * G * p.C;
     constexpr int kBatch = (G >= 4 ? 4 : 8);                                      // slots per thread whose loads are issued together
+    int n_imp = 0;                                                                // keys this thread judged important
     for (int base0 = 0; base0 < l; base0 += kBatch * NT) {
         double sv[kBatch][G];
         uint32_t wv[kBatch];
@@ -326,11 +334,13 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 const uint32_t wd = update_register(wv[k], imp, p.w, t);
                 wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
+                n_imp += imp ? 1 : 0;
             }
             const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
             if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
         }
     }
+    warp_count(p.counters + CNT_IMPORTANT, n_imp);         // Section 3.1's sparsity: keys judged important this step
     __syncthreads();
     int new_len = l, n_moved = 0;
     if (evict_on) {

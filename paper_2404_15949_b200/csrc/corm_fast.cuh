@@ -207,6 +207,7 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     int32_t* posu = p.pos + (size_t)u * p.C;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
     const bool evict_on = n_obs >= p.w;
+    int n_imp = 0;                                                // keys this thread judged important
 #pragma unroll
     for (int k = 0; k < KPRE; ++k) {
         const int base = k * NT, j = base + tid;
@@ -217,12 +218,14 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
 #pragma unroll
             for (int g = 0; g < G; ++g) imp |= (stash_sm[g * stash_ld + j] >= thr[g]);
             const uint32_t wd = update_register(wv[k], imp, p.w, t);
+            n_imp += imp ? 1 : 0;
             wordu[j] = wd;
             keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
         }
         const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
         if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
     }
+    warp_count(p.counters + CNT_IMPORTANT, n_imp);                // Section 3.1's sparsity
     __syncthreads();
     int new_len = l, n_moved = 0;
     if (evict_on) {

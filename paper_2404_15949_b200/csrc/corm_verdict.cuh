@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     __syncthreads();
     // b. verdicts, register update, keep flags of this block's slots
     uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
+    int n_imp = 0;                                                         // keys this thread judged important
     {
 #pragma unroll
         for (int k = 0; k < kVerdictPer; ++k) {
@@ -122,11 +123,14 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
                 const uint32_t wd = update_register(wv[k], imp, p.w, t);
                 wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
+                n_imp += imp ? 1 : 0;
             }
             const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
             if (lane == 0 && base + warp * 32 < l) keep_g[(base >> 5) + warp] = ballot;
         }
     }
+
+    warp_count(p.counters + CNT_IMPORTANT, n_imp);                         // Section 3.1's sparsity
 
     // c. the last block of the unit to get here compacts it
     __threadfence();

@@ -81,4 +81,6 @@ def run_free(cfg, data, gpu, orc, layer=0, check_every=1, steps=None):
             assert_states_equal(gpu, orc, layer, nb, nh, f"after step {s}")
     st = gpu.corm_cache_stats()
     assert st["device_status"] == 0
+    if gpu.cfg.n_layers == 1:           # Section 3.1's sparsity counters: keys judged important / keys judged
+        assert (st["important_keys"], st["attended_keys"]) == orc.sparsity()
     return worst

@@ -358,3 +358,33 @@ def test_bad_arguments_and_capacity():
     o.decode_step(0, x, x, x)
     with pytest.raises(RuntimeError):
         o.decode_step(0, x, x, x)
+
+
+def test_sparsity_counters_match_the_verdict_rows():
+    """The proportion of important keys (Section 3.1) is counted over decode steps: the counters must equal what the
+    per-step verdict rows add up to, and with alpha = 0 every judged key is important."""
+    from oracle import CormOracle
+    rng = np.random.default_rng(5)
+    for alpha in (1.0, 0.0):
+        o = CormOracle(1, 2, 4, 2, 8, 64, 3, 2, alpha)
+        kp = rng.standard_normal((2, 2, 10, 8)).astype(np.float32)
+        vp = rng.standard_normal((2, 2, 10, 8)).astype(np.float32)
+        ql = rng.standard_normal((2, 4, 3, 8)).astype(np.float32)
+        o.compress_prompt(0, kp, vp, ql, np.array([10, 7], dtype=np.int32))
+        assert o.sparsity() == (0, 0)                      # the prompt pass is not counted
+        imp_sum = judged = 0
+        for s in range(12):
+            lens = o.live_lens(0)
+            q = rng.standard_normal((2, 4, 8)).astype(np.float32) * 2
+            kn = rng.standard_normal((2, 2, 8)).astype(np.float32)
+            vn = rng.standard_normal((2, 2, 8)).astype(np.float32)
+            _, imp = o.decode_step(0, q, kn, vn, want_verdicts=True)
+            for b in range(2):
+                for h in range(2):
+                    imp_sum += int(imp[b, h, :lens[b, h] + 1].sum())
+                    judged += int(lens[b, h]) + 1
+        assert o.sparsity() == (imp_sum, judged)
+        if alpha == 0.0:
+            assert imp_sum == judged
+        else:
+            assert 0 < imp_sum < judged
