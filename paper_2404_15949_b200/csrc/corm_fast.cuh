@@ -45,14 +45,13 @@ inline bool fast_path_available() { return true; }
 
 // ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
 struct FastSmem {
-    int tiles, qs, psm, stash, bars, total;
+    int tiles, psm, stash, bars, total;
 };
 __host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
     FastSmem s;
     int off = 0;
     auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
     s.tiles = take(kFastWarps * fast_warp_bytes(G));            // later reused: merge area, finalize lists
-    s.qs = take(G * 128 * 8);
     s.psm = take(kFastWarps * kTileKeys * G * 4);
     s.stash = take(single_cap * G * 8);
     s.bars = take(kFastWarps * fast_stages(G) * 8);
@@ -282,7 +281,6 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
     unsigned char* my_tiles = smem + lay.tiles + warp * fast_warp_bytes(G);
     const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kStagesPerWarp * 8;
-    double* qs = reinterpret_cast<double*>(smem + lay.qs);
     float* psm = reinterpret_cast<float*>(smem + lay.psm) + warp * kTileKeys * G;
     double* stash_sm = reinterpret_cast<double*>(smem + lay.stash);
     const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.K) + (size_t)u * p.C * kRowBytes;
@@ -335,19 +333,18 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             else if (j == l_old) { wv[k] = 0u; pv[k] = t; }          // the token appended by this step
         }
     }
-    {
-        const bf16_t* qg = reinterpret_cast<const bf16_t*>(p.q) + (size_t)u * G * 128;
-        for (int x = tid; x < G * 128; x += NT) qs[x] = (double)Elem<bf16_t>::load(qg + x);
-    }
-    __syncthreads();
-
     const int h = lane >> 4, ci = lane & 15;
     const int key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);     // tile key this lane owns after the fold
+    // the lane's 8 channels of every query head, widened to fp64: one 16-byte load per head, no staging
     double qd[G][8];
+    {
+        const uint4* qg = reinterpret_cast<const uint4*>(p.q) + (size_t)u * G * 16 + ci;
 #pragma unroll
-    for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) qd[g][e] = qs[g * 128 + ci * 8 + e];
+        for (int g = 0; g < G; ++g) {
+            const uint4 raw = __ldg(qg + g * 16);
+            unpack8_to_double(raw, qd[g]);
+        }
+    }
     double M[G], Zl[G];
     unsigned long long acc2[G][4];                                // P.V accumulators: channel pairs (2e, 2e+1) of this lane's 8
 #pragma unroll
