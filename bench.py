@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the decode kernel, from the ncu capture summarised in
 # profiles/decode_fast_kernel_batch32_bf16.md (323.9 MB moved for 313.1 MB algorithmic at the captured steps).
 # Set to None whenever the kernel changes until the counters are taken again.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.034}
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.013}
 
 
 def log(*a):
@@ -296,7 +296,7 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src,
                      "traffic": (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE.get(cfg.name) or 0) * abytes / (args.steps * L) or None,
-                     "kernel": "decode step kernel (one launch per layer per step)",
+                     "kernel": "decode_fast_kernel (one launch per layer per step; early steps with units longer than one block add a verdict launch, counted in the time)",
                      "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * ms / (args.steps * L)},
         "e2e": {"value": e2e_value, "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
