@@ -52,7 +52,8 @@ typedef enum { CORM_F32 = 0, CORM_BF16 = 1 } corm_dtype_t;
 typedef struct {
     int32_t n_layers, batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0, group size in {1,2,4,8} */
     int32_t head_dim;                                /* 64 or 128 */
-    int32_t max_tokens;                              /* slab capacity per unit: >= longest prompt + decode steps */
+    int32_t max_tokens;                              /* slab capacity per unit: >= longest prompt + decode steps;
+                                                        at most 524288 (UNSUPPORTED beyond) */
     int32_t window_w;                                /* 1..256 recent queries; see the register encodings below */
     int32_t recent_r;                                /* >= 1 (Algorithm 1's slice of the last r entries) */
     float   alpha;                                   /* >= 0; threshold alpha/t; 0 means nothing is ever evicted */
@@ -167,6 +168,15 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Number of kernels this library has launched on behalf of `cache` since create. */
+/* Opt-in monitor of the method's premise (Sections 3.2-3.3: the current query resembles recent ones, which is what
+ * lets recent verdicts stand in for future ones, and which the paper reports failing for some models): while
+ * enabled, every decode step also forms Eq. 3's cosine similarity between each query head's query and that head's
+ * query of the previous decode step of the same layer (one small extra launch per step; the first step after a
+ * prompt pass or after enabling has no partner; zero vectors are skipped). corm_cache_similarity returns the sum
+ * and the number of pairs since create/reset over all layers and synchronises `stream`. Off by default. */
+corm_status_t corm_cache_set_similarity_monitor(corm_cache_t* cache, int32_t enabled);
+corm_status_t corm_cache_similarity(corm_cache_t* cache, double* sum_host, int64_t* count_host, void* stream);
+
 int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
 
 const char* corm_status_string(corm_status_t status);

@@ -41,6 +41,9 @@ typedef struct {
     int     *t;      /* [L*B]                tokens seen                      */
     int     *n_obs;  /* [L*B]                verdict rows recorded            */
     long long appended, evicted, verdict_evals, near_threshold;
+    double *q_prev;      /* [n_layers][batch][n_q_heads][d]: the previous decode step's queries */
+    unsigned char *has_prev; /* [n_layers] */
+    double sim_sum; long long sim_count; /* Eq. 3 between each head's query and its previous one */
     long long important, judged; /* decode steps only: keys judged important / keys judged (the sparsity of Section 3.1) */
     double  near_rel; /* half-width of the reported band around the threshold, relative */
 } corm_oracle;
@@ -69,13 +72,15 @@ corm_oracle *oracle_create(int n_layers, int batch, int n_q_heads, int n_kv_head
     o->v = (double *)calloc(units * C * d, sizeof(double));
     o->t = (int *)calloc((size_t)n_layers * batch, sizeof(int));
     o->n_obs = (int *)calloc((size_t)n_layers * batch, sizeof(int));
-    if (!o->live || !o->pos || !o->word || !o->k || !o->v || !o->t || !o->n_obs) return NULL;
+    o->q_prev = (double *)calloc((size_t)n_layers * batch * n_q_heads * d, sizeof(double));
+    o->has_prev = (unsigned char *)calloc((size_t)n_layers, 1);
+    if (!o->live || !o->pos || !o->word || !o->k || !o->v || !o->t || !o->n_obs || !o->q_prev || !o->has_prev) return NULL;
     return o;
 }
 
 void oracle_destroy(corm_oracle *o) {
     if (!o) return;
-    free(o->live); free(o->pos); free(o->word); free(o->k); free(o->v); free(o->t); free(o->n_obs); free(o);
+    free(o->live); free(o->pos); free(o->word); free(o->k); free(o->v); free(o->t); free(o->n_obs); free(o->q_prev); free(o->has_prev); free(o);
 }
 
 /* register helpers: shift the newest verdict in at bit 0 and drop everything older than w verdicts */
@@ -165,6 +170,23 @@ int oracle_decode_step(corm_oracle *o, int layer, const float *q, const float *k
     for (int b = 0; b < B; ++b)
         for (int h = 0; h < Hkv; ++h)
             if (o->live[unit_index(o, layer, b, h)] + 1 > o->max_tokens) return ORACLE_CAPACITY;
+    /* Eq. 3: cosine similarity of every query head's query with the one of the previous decode step (Section 3.3
+     * observes that the current query is most similar to recent ones); heads with a zero vector are skipped */
+    {
+        double *prev = o->q_prev + (size_t)layer * B * Hq * d;
+        for (int x = 0; x < B * Hq; ++x) {
+            if (o->has_prev[layer]) {
+                double dot = 0.0, n1 = 0.0, n2 = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    double a = (double)q[(size_t)x * d + c], pb = prev[(size_t)x * d + c];
+                    dot += a * pb; n1 += a * a; n2 += pb * pb;
+                }
+                if (n1 > 0.0 && n2 > 0.0) { o->sim_sum += dot / (sqrt(n1) * sqrt(n2)); o->sim_count += 1; }
+            }
+            for (int c = 0; c < d; ++c) prev[(size_t)x * d + c] = (double)q[(size_t)x * d + c];
+        }
+        o->has_prev[layer] = 1;
+    }
     long long evals_total = 0, near_total = 0, appended = 0, evicted = 0, important_total = 0, judged_total = 0;
 #pragma omp parallel for collapse(2) schedule(dynamic) reduction(+ : evals_total, near_total, appended, evicted, important_total, judged_total)
     for (int b = 0; b < B; ++b) {
@@ -231,6 +253,12 @@ void oracle_sparsity(const corm_oracle *o, long long *important, long long *judg
     if (judged) *judged = o->judged;
 }
 
+/* Sum and number of the adjacent-query cosine similarities (Eq. 3) over the decode steps so far. */
+void oracle_similarity(const corm_oracle *o, double *sum, long long *count) {
+    if (sum) *sum = o->sim_sum;
+    if (count) *count = o->sim_count;
+}
+
 /* Prompt-end pass for every unit of one layer.
  * k_prompt/v_prompt [B,Hkv,p_max,d]; q_last [B,Hq,w,d] = queries of prompt positions P-w+1..P, oldest first (for
  * P < w the first w-P rows are ignored); prompt_lens [B]. All P keys enter the cache, then the causal attention
@@ -247,6 +275,7 @@ int oracle_compress_prompt(corm_oracle *o, int layer, const float *k_prompt, con
         if (prompt_lens[b] > o->max_tokens) return ORACLE_CAPACITY;
         if (prompt_lens[b] > 0 && (!k_prompt || !v_prompt || !q_last)) return ORACLE_BAD_ARG;
     }
+    o->has_prev[layer] = 0;                 /* a new prompt: the layer's previous decode query belongs to the old text */
     long long evals_total = 0, near_total = 0, appended = 0, evicted = 0;
 #pragma omp parallel for collapse(2) schedule(dynamic) reduction(+ : evals_total, near_total, appended, evicted)
     for (int b = 0; b < B; ++b) {

@@ -52,6 +52,8 @@ def _load():
     lib.oracle_counters.argtypes = [vp, vp, vp, vp, vp]
     lib.oracle_sparsity.argtypes = [vp, vp, vp]
     lib.oracle_sparsity.restype = None
+    lib.oracle_similarity.argtypes = [vp, vp, vp]
+    lib.oracle_similarity.restype = None
     lib.oracle_set_near_band.argtypes = [vp, c_dbl]
     _lib = lib
     return lib
@@ -154,6 +156,12 @@ class CormOracle:
         """(keys judged important, keys judged) over the decode steps so far."""
         a, b = ctypes.c_longlong(0), ctypes.c_longlong(0)
         self.lib.oracle_sparsity(self.h, ctypes.byref(a), ctypes.byref(b))
+        return a.value, b.value
+
+    def similarity(self):
+        """(sum, count) of Eq. 3 between each query head's query and its query of the previous decode step."""
+        a, b = ctypes.c_double(0.0), ctypes.c_longlong(0)
+        self.lib.oracle_similarity(self.h, ctypes.byref(a), ctypes.byref(b))
         return a.value, b.value
 
     def set_near_band(self, rel):

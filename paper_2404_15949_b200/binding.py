@@ -79,6 +79,10 @@ def load_library():
     lib.corm_cache_import_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp]
     lib.corm_cache_set_tuning.restype = i32
     lib.corm_cache_set_tuning.argtypes = [vp, i32, i32]
+    lib.corm_cache_set_similarity_monitor.restype = ctypes.c_int
+    lib.corm_cache_set_similarity_monitor.argtypes = [vp, ctypes.c_int32]
+    lib.corm_cache_similarity.restype = ctypes.c_int
+    lib.corm_cache_similarity.argtypes = [vp, vp, vp, vp]
     lib.corm_cache_kernel_launches.restype = i64
     lib.corm_cache_kernel_launches.argtypes = [vp]
     lib.corm_status_string.restype = ctypes.c_char_p
@@ -200,6 +204,16 @@ class CormCache:
         """allow_fast_path: False/0 generic kernels, True/1 fast kernels, 2 / 3 fast kernels that always finish units of
         several splits inside the decode launch / by the verdict launch."""
         _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
+
+    def corm_cache_set_similarity_monitor(self, enabled=True):
+        _check("corm_cache_set_similarity_monitor", self.lib.corm_cache_set_similarity_monitor(self.handle, int(enabled)))
+
+    def corm_cache_similarity(self, stream=None):
+        """(sum, count) of the adjacent-query cosine similarities (Eq. 3) recorded while the monitor was on."""
+        total, n = ctypes.c_double(0.0), ctypes.c_int64(0)
+        _check("corm_cache_similarity", self.lib.corm_cache_similarity(self.handle, ctypes.byref(total), ctypes.byref(n),
+                                                                     _stream_ptr(stream)))
+        return total.value, n.value
 
     def corm_cache_kernel_launches(self):
         return int(self.lib.corm_cache_kernel_launches(self.handle))

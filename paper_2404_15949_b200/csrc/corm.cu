@@ -27,7 +27,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, q_prev, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -46,7 +46,7 @@ bool config_ok(const corm_config_t* c, corm_status_t* why) {
     if (G != 1 && G != 2 && G != 4 && G != 8) return false;
     if (c->window_w > 256) return false;
     if ((long long)c->batch * c->n_kv_heads > 65535) return false;     // grid.y of the decode kernel
-    if (c->max_tokens > (1 << 22)) return false;
+    if (c->max_tokens > (1 << 19)) return false;                        // the keep mask of a unit must fit shared memory
     *why = CORM_OK;
     return true;
 }
@@ -71,7 +71,9 @@ Layout make_layout(const corm_config_t& c) {
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
+    L.sim_acc = take(16);
     L.bookkeeping_end = off;
+    L.q_prev = take(Ltot * (size_t)c.batch * c.n_q_heads * D * e);
     L.stash = take(U * G * C * 8);
     L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
     L.keepmask = take(U * (size_t)keepmask_words((int)C) * 4);
@@ -116,6 +118,8 @@ struct corm_cache {
     std::vector<cudaEvent_t> readback_ev;
     std::vector<int> readback_pending, last_readback_step;
     int tune_split_len = 0, allow_fast = 1;
+    int monitor_similarity = 0;
+    std::vector<int> have_q_prev;                 // the layer's previous decode queries are stored
     int sm_count = 148;
     long long launches = 0;
 };
@@ -225,6 +229,24 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
     if (c->steps[layer] - c->last_readback_step[layer] >= 8) schedule_live_readback(c, layer, st);
+    if (c->monitor_similarity) {
+        const int n_heads = cf.batch * cf.n_q_heads;
+        const size_t qb = (size_t)n_heads * D * c->e;
+        double* sum = reinterpret_cast<double*>(c->arena + c->lay.sim_acc);
+        unsigned long long* cnt = reinterpret_cast<unsigned long long*>(c->arena + c->lay.sim_acc + 8);
+        rc = dispatch(c, [&](auto* tp, auto dd, auto) -> corm_status_t {
+            using T = std::remove_pointer_t<decltype(tp)>;
+            constexpr int DD = decltype(dd)::value;
+            query_similarity_kernel<T, DD><<<(n_heads + 3) / 4, 128, 0, st>>>(
+                reinterpret_cast<const T*>(q), reinterpret_cast<T*>(layer_ptr(c, c->lay.q_prev, qb, layer)),
+                c->have_q_prev[layer], n_heads, sum, cnt);
+            CORM_CUDA(cudaGetLastError());
+            return CORM_OK;
+        });
+        if (rc != CORM_OK) return rc;
+        c->have_q_prev[layer] = 1;
+        c->launches += 1;
+    }
     return CORM_OK;
 }
 
@@ -260,6 +282,7 @@ corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, si
     c->steps.assign(cfg->n_layers, 0);
     c->ready.assign(cfg->n_layers, 0);
     c->live_upper.assign(cfg->n_layers, 0);
+    c->have_q_prev.assign(cfg->n_layers, 0);
     c->readback_pending.assign(cfg->n_layers, 0);
     c->last_readback_step.assign(cfg->n_layers, 0);
     c->readback_ev.assign(cfg->n_layers, nullptr);
@@ -307,7 +330,7 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
     CORM_CUDA(cudaMemsetAsync(c->arena + c->lay.bookkeeping_begin, 0, c->lay.bookkeeping_end - c->lay.bookkeeping_begin,
                               static_cast<cudaStream_t>(stream)));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-        c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0;
+        c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; c->have_q_prev[l] = 0;
         c->readback_pending[l] = 0; c->last_readback_step[l] = 0;
     }
     return CORM_OK;
@@ -383,6 +406,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     if (rc != CORM_OK) return rc;
     c->launches += n_launched;
     c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p;
+    c->have_q_prev[layer] = 0;                    // the previous decode query belonged to the old text
     c->last_readback_step[layer] = 0;
     schedule_live_readback(c, layer, st);
     return CORM_OK;
@@ -629,6 +653,28 @@ corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t 
     c->tune_split_len = split_len;
     if (allow_fast_path < 0 || allow_fast_path > 3) return CORM_ERR_INVALID_ARG;
     c->allow_fast = allow_fast_path;
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_set_similarity_monitor(corm_cache_t* c, int32_t enabled) {
+    if (!c) return CORM_ERR_INVALID_ARG;
+    c->monitor_similarity = enabled ? 1 : 0;
+    if (!enabled) std::fill(c->have_q_prev.begin(), c->have_q_prev.end(), 0);   // a gap breaks the chain of adjacent steps
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_similarity(corm_cache_t* c, double* sum_host, int64_t* count_host, void* stream) {
+    if (!c || !sum_host || !count_host) return CORM_ERR_INVALID_ARG;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char buf[16];
+    CORM_CUDA(cudaMemcpyAsync(buf, c->arena + c->lay.sim_acc, 16, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    std::memcpy(sum_host, buf, 8);
+    unsigned long long n;
+    std::memcpy(&n, buf + 8, 8);
+    *count_host = (int64_t)n;
     return CORM_OK;
 }
 

@@ -213,4 +213,29 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     }
 }
 
+// Opt-in monitor of the premise of Section 3.3 (the current query resembles recent ones): Eq. 3 between every query
+// head's query and its query of the previous decode step, summed into acc[0] (fp64) with the number of pairs in
+// acc[1] (as an integer in the same 8 bytes), then the queries are kept for the next step. One warp per head.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) query_similarity_kernel(const T* q, T* q_prev, int have_prev, int n_heads,
+                                                               double* sum, unsigned long long* count) {
+    const int lane = threadIdx.x & 31, head = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (head >= n_heads) return;
+    double dot = 0.0, n1 = 0.0, n2 = 0.0;
+    for (int c = lane; c < D; c += 32) {
+        const double a = (double)Elem<T>::load(q + (size_t)head * D + c);
+        if (have_prev) {
+            const double b = (double)Elem<T>::load(q_prev + (size_t)head * D + c);
+            dot = fma(a, b, dot); n1 = fma(a, a, n1); n2 = fma(b, b, n2);
+        }
+        Elem<T>::store(q_prev + (size_t)head * D + c, (float)a);
+    }
+    if (!have_prev) return;
+    dot = warp_sum(dot); n1 = warp_sum(n1); n2 = warp_sum(n2);
+    if (lane == 0 && n1 > 0.0 && n2 > 0.0) {
+        atomicAdd(sum, dot / (sqrt(n1) * sqrt(n2)));
+        atomicAdd(count, 1ull);
+    }
+}
+
 }  // namespace corm

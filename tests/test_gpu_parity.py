@@ -73,6 +73,21 @@ def test_small_shapes(case):
     assert orc.counters()["near_threshold"] == 0
 
 
+@pytest.mark.parametrize("dtype,d,G", [("bf16", 128, 1), ("bf16", 128, 4), ("f32", 64, 2)])
+def test_adjacent_query_similarity_monitor(dtype, d, G):
+    """Eq. 3 between consecutive decode queries, summed by the opt-in monitor, against the oracle's fp64 sum."""
+    cfg = CONFIGS[1].with_(name="sim", batch=2, n_q_heads=2 * G, n_kv_heads=2, head_dim=d, dtype=dtype, prompt_min=90,
+                           prompt_max=160, steps=20, gqa_rho=0.7 if G > 1 else 0.0, seed=321)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    gpu.corm_cache_set_similarity_monitor(True)
+    run_free(cfg, data, gpu, orc, check_every=10)
+    (sg, ng), (so, no) = gpu.corm_cache_similarity(), orc.similarity()
+    assert ng == no == 2 * 2 * G * (cfg.steps - 1)
+    assert abs(sg - so) <= 1e-9 * no
+    assert 0.0 < so / no < 1.0                                   # the generator's queries drift slowly (Section 3.3)
+
+
 def test_alpha_zero_never_evicts():
     cfg = CONFIGS[1].with_(prompt_min=100, prompt_max=100, steps=20, alpha=0.0, dtype="bf16")
     data = generate(cfg)

@@ -388,3 +388,32 @@ def test_sparsity_counters_match_the_verdict_rows():
             assert imp_sum == judged
         else:
             assert 0 < imp_sum < judged
+
+
+def test_adjacent_query_similarity_closed_forms():
+    """Eq. 3 between consecutive decode queries: a query repeated up to a positive factor gives 1, its negative -1, an
+    orthogonal one 0, and random ones what numpy's dot and norms give; the first step after a prompt has no partner."""
+    from oracle import CormOracle
+    rng = np.random.default_rng(11)
+    o = CormOracle(1, 1, 2, 2, 8, 64, 3, 2, 1.0)
+    z = np.zeros((1, 2, 4, 8), dtype=np.float32)
+    o.compress_prompt(0, rng.standard_normal((1, 2, 4, 8)).astype(np.float32), z.copy(), np.zeros((1, 2, 3, 8), dtype=np.float32),
+                      np.array([4], dtype=np.int32))
+    kn = rng.standard_normal((1, 2, 8)).astype(np.float32)
+    q0 = rng.standard_normal((1, 2, 8)).astype(np.float32)
+    e0 = np.zeros((1, 2, 8), dtype=np.float32); e0[..., 0] = 1
+    e1 = np.zeros((1, 2, 8), dtype=np.float32); e1[..., 1] = 3
+    qs = [q0, 2.5 * q0, -q0, e0, e1, q0, rng.standard_normal((1, 2, 8)).astype(np.float32)]
+    expect, total = [None, 1.0, -1.0, None, 0.0, None, None], 0.0
+    for i, q in enumerate(qs):
+        before = o.similarity()
+        o.decode_step(0, q, kn, kn)
+        after = o.similarity()
+        if i == 0:
+            assert after == (0.0, 0)
+            continue
+        a, b = qs[i].astype(np.float64), qs[i - 1].astype(np.float64)
+        ref = sum(float(a[0, h] @ b[0, h]) / (np.linalg.norm(a[0, h]) * np.linalg.norm(b[0, h])) for h in range(2))
+        assert after[1] == before[1] + 2 and abs((after[0] - before[0]) - ref) < 1e-12
+        if expect[i] is not None:
+            assert abs((after[0] - before[0]) - 2 * expect[i]) < 1e-12
