@@ -159,8 +159,18 @@ unsigned long long* maxlive_ptr(const corm_cache* c, int layer) {
 
 // If an earlier read-back has landed, tighten the bound on this layer's longest unit: a unit grows by at most one
 // key per step, so (length after step s) + (steps since s) bounds every unit now.
+// A host that enqueues steps much faster than the GPU runs them would otherwise size its launches from a bound that
+// is hundreds of steps stale (every step adds one key to it): once it is kMaxRunAhead steps past a read-back that
+// has not landed it waits for that one, which leaves the GPU that many steps of queued work and costs it nothing.
+constexpr int kMaxRunAhead = 24;
 void poll_live_bound(corm_cache* c, int layer) {
-    if (!c->readback_pending[layer] || cudaEventQuery(c->readback_ev[layer]) != cudaSuccess) return;
+    if (!c->readback_pending[layer]) return;
+    if (c->steps[layer] - c->last_readback_step[layer] >= kMaxRunAhead) {
+        if (cudaEventSynchronize(c->readback_ev[layer]) != cudaSuccess) return;
+    } else if (cudaEventQuery(c->readback_ev[layer]) != cudaSuccess) {
+        (void)cudaGetLastError();   // cudaErrorNotReady is not an error
+        return;
+    }
     c->readback_pending[layer] = 0;
     const unsigned long long v = c->maxlive_host[layer];
     const int steps_done = (int)(v >> 32), len = (int)(v & 0xffffffffu);
