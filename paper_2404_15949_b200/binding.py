@@ -122,6 +122,8 @@ class CormCache:
         code = {"bf16": CORM_BF16, "f32": CORM_F32}[kv_dtype]
         self.cfg = CormConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, window_w, recent_r,
                               float(alpha), code, device)
+        self._q_shape = (batch, n_q_heads, head_dim)
+        self._kv_shape = (batch, n_kv_heads, head_dim)
         self.kv_dtype, self.dtype, self.device = code, _torch_dtype(code), torch.device("cuda", device)
         nbytes = corm_cache_arena_bytes(self.cfg)
         if nbytes == 0:
@@ -156,15 +158,18 @@ class CormCache:
             _stream_ptr(stream)))
 
     def corm_decode_step(self, layer, q, k_new, v_new, out=None, stream=None):
-        c = self.cfg
-        assert tuple(q.shape) == (c.batch, c.n_q_heads, c.head_dim) and q.dtype == self.dtype and q.is_contiguous()
-        assert tuple(k_new.shape) == (c.batch, c.n_kv_heads, c.head_dim) and k_new.is_contiguous()
-        assert tuple(v_new.shape) == tuple(k_new.shape) and v_new.is_contiguous()
-        assert k_new.dtype == self.dtype and v_new.dtype == self.dtype and q.is_cuda and k_new.is_cuda and v_new.is_cuda
+        # argument checks kept cheap: this call is on the per-token path and a launch is only a few microseconds
+        if q.shape != self._q_shape or k_new.shape != self._kv_shape or v_new.shape != self._kv_shape:
+            raise ValueError("corm_decode_step: q / k_new / v_new have the wrong shape")
+        if not (q.dtype == k_new.dtype == v_new.dtype == self.dtype and q.is_cuda and k_new.is_cuda and v_new.is_cuda
+                and q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()):
+            raise ValueError("corm_decode_step: inputs must be contiguous device tensors of the cache dtype")
         if out is None:
             out = torch.empty_like(q)
-        _check("corm_decode_step", self.lib.corm_decode_step(self.handle, layer, q.data_ptr(), k_new.data_ptr(),
-                                                             v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream)))
+        rc = self.lib.corm_decode_step(self.handle, layer, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                                       out.data_ptr(), _stream_ptr(stream))
+        if rc != CORM_OK:
+            raise CormError("corm_decode_step", rc)
         return out
 
     def corm_decode_step_static(self, layer, q, k_new, v_new, out=None, stream=None):

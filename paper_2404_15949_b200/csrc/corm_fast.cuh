@@ -591,7 +591,9 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     const bool all_single = n_splits == 1 && upper <= p.single_cap;      // every unit finishes inside its one block
     // who finishes the longer units: see the end of decode_fast_kernel
     const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // keep mask + prefix sums of finalize_unit
-    const bool many = finish_mode == 2 || (finish_mode != 3 && (long long)p.U * n_splits >= 4ll * sms * fast_blocks_per_sm(G));
+    // ... or when units are so short that the serial walk (upper x G logits over 128 threads) is cheaper than a launch
+    const bool many = finish_mode == 2 || (finish_mode != 3 && ((long long)p.U * n_splits >= 4ll * sms * fast_blocks_per_sm(G) ||
+                                                                (long long)upper * G <= 2048));
     p.inline_finalize = !all_single && many && fin <= smem;
     const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
                         (size_t)2 * p.single_cap * 4;
