@@ -1,6 +1,7 @@
 // Shared device-side definitions of the CORM kernels: parameter blocks, element access, and the per-unit
 // "finalize" phase (split reduction, verdict, register update, keep decision, hole-filling compaction) that the
-// last-arriving thread block of a unit runs inside the decode kernel.
+// last-arriving thread block of a unit runs inside a decode kernel (the generic kernels always, the fast kernel when
+// it does not leave the unit to the verdict launch).
 #pragma once
 
 #include <cuda_runtime.h>

@@ -7,9 +7,10 @@
 // key; the 16 partial sums of 16 keys are folded with a transposing butterfly (15 exchanges for 16 keys, no
 // selects: each lane loads its keys in an order permuted by its lane bits so that every exchange step sends and
 // keeps fixed registers). After the fold each lane owns one key of the tile for softmax, verdict logit and
-// probability. P.V accumulates in fp32. A unit that fits one split keeps its logits, registers and positions in
-// shared memory and finishes entirely inside the block; longer units publish split partials and logits to global
-// scratch and the last-arriving block runs the shared finalize phase.
+// probability. P.V accumulates in fp32. A unit that fits one split keeps its logits in shared memory and its
+// registers and positions in thread registers and finishes entirely inside the block; longer units publish split
+// records and logits to global scratch, and either the last-arriving block runs the shared finalize phase (launches
+// with many blocks, or short units) or the verdict launch of corm_verdict.cuh takes over (few, long units).
 #pragma once
 
 #include <cmath>
@@ -584,7 +585,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     p.split_len = split_len;
     const int n_splits = (upper + split_len - 1) / split_len;
     if (n_splits > p.max_splits) return CORM_ERR_UNSUPPORTED;
-    // on-chip finish for units of one split, as long as two blocks still fit on an SM
+    // on-chip finish for units of one split, as far as shared memory for their logits allows
     p.single_cap = split_len < cap ? split_len : cap;
     const FastSmem lay = fast_smem_layout(G, p.single_cap);
     const size_t smem = (size_t)lay.total;
