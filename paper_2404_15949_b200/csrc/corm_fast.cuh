@@ -48,7 +48,7 @@ inline bool fast_path_available() { return true; }
 
 // ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
 struct FastSmem {
-    int tiles, psm, stash, bars, total;
+    int tiles, psm, stash, bars, newrow, total;
 };
 __host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
     FastSmem s;
@@ -58,6 +58,7 @@ __host__ __device__ inline FastSmem fast_smem_layout(int G, int single_cap) {
     s.psm = take(kFastWarps * kTileKeys * G * 4);
     s.stash = take(single_cap * G * 8);
     s.bars = take(kFastWarps * fast_stages(G) * 8);
+    s.newrow = take(2 * kRowBytes);                             // the appended K and V rows, fetched ahead
     s.total = off;
     return s;
 }
@@ -90,6 +91,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src_gme
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst_smem), "l"(src_gmem), "r"(bytes), "r"(bar) : "memory");
 }
+// 16-byte asynchronous copy global -> shared by the calling thread, and the wait for all of the thread's own
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src_gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
@@ -320,6 +326,15 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         for (int it = 0; it < min(my_n, kKStages); ++it) issue_k(it);
         for (int it = 0; it < min(my_n, kVStages); ++it) issue_v(it);
     }
+    // The appended token's rows are fetched now by the warp that will meet slot l_old (the unit's last tile), so that
+    // their latency (a PCIe round trip when the caller's buffers are pinned host memory) is off that tile's path.
+    unsigned char* newrow = smem + lay.newrow;
+    const bool new_is_mine = l_old >= begin && l_old < end && ((l_old - begin) / kTileKeys) % NW == warp;
+    if (new_is_mine) {
+        const unsigned char* src = lane < 16 ? reinterpret_cast<const unsigned char*>(p.k_new) + ((size_t)u * 16 + lane) * 16
+                                             : reinterpret_cast<const unsigned char*>(p.v_new) + ((size_t)u * 16 + lane - 16) * 16;
+        cp_async16(smem_addr(newrow + lane * 16), src);
+    }
 
     // queries widened to fp64 once per block; a single-split unit also fetches the registers and positions of the
     // slots this thread will judge in the finalize phase (slots tid, tid + NT, ...) and keeps them in registers
@@ -368,9 +383,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         unsigned char* vtile = my_tiles + (kKStages + vslot) * kTileBytes;
         if (!mbar_wait(my_bars + kslot * 8, (it / kKStages) & 1)) failed = true;
         if (has_new) {   // append: the new row goes to the slab and replaces whatever the copy fetched for that slot
-            const uint4* kn = reinterpret_cast<const uint4*>(p.k_new) + (size_t)u * 16;
+            cp_async_wait_all();
+            __syncwarp();
             if (lane < 16) {
-                const uint4 x = kn[lane];
+                const uint4 x = *reinterpret_cast<const uint4*>(newrow + lane * 16);
                 *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = x;
                 reinterpret_cast<uint4*>(const_cast<unsigned char*>(Ku) + (size_t)l_old * kRowBytes)[lane] = x;
             }
@@ -429,9 +445,8 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
         if (!mbar_wait(my_bars + (kKStages + vslot) * 8, (it / kVStages) & 1)) failed = true;
         if (has_new) {
-            const uint4* vn = reinterpret_cast<const uint4*>(p.v_new) + (size_t)u * 16;
             if (lane < 16) {
-                const uint4 x = vn[lane];
+                const uint4 x = *reinterpret_cast<const uint4*>(newrow + kRowBytes + lane * 16);
                 *reinterpret_cast<uint4*>(vtile + (l_old - k0) * kRowBytes + lane * 16) = x;
                 reinterpret_cast<uint4*>(const_cast<unsigned char*>(Vu) + (size_t)l_old * kRowBytes)[lane] = x;
             }
