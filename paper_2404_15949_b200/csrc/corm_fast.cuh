@@ -298,13 +298,6 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     int32_t* posu = p.pos + (size_t)u * p.C;
 
     if (tid == 0) s_failed = 0;
-    if (lane == 0) {
-#pragma unroll
-        for (int s = 0; s < kStagesPerWarp; ++s) mbar_init(my_bars + s * 8, 1);
-        fence_mbar_init();
-        fence_async_smem();
-    }
-    __syncthreads();
 
     // this warp's tiles: warp, warp + NW, ... (tile index inside the split)
     const int my_n = (n_tiles > warp) ? (n_tiles - warp + NW - 1) / NW : 0;
@@ -322,7 +315,12 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vu + (size_t)k0 * kRowBytes, bytes,
                   my_bars + (kKStages + slot) * 8);
     };
+    // a warp's barriers and stages are its own: its first copies leave before the block meets at its first barrier
     if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kStagesPerWarp; ++s) mbar_init(my_bars + s * 8, 1);
+        fence_mbar_init();
+        fence_async_smem();
         for (int it = 0; it < min(my_n, kKStages); ++it) issue_k(it);
         for (int it = 0; it < min(my_n, kVStages); ++it) issue_v(it);
     }
@@ -335,6 +333,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
                                              : reinterpret_cast<const unsigned char*>(p.v_new) + ((size_t)u * 16 + lane - 16) * 16;
         cp_async16(smem_addr(newrow + lane * 16), src);
     }
+    __syncthreads();                                              // s_failed is initialised for everybody
 
     // queries widened to fp64 once per block; a single-split unit also fetches the registers and positions of the
     // slots this thread will judge in the finalize phase (slots tid, tid + NT, ...) and keeps them in registers
