@@ -142,7 +142,7 @@ def run_reference(args, cfg):
 
 
 def workload_config(cfg, args):
-    return {"workload": f"{cfg.name} (BASELINE configs[{args.workload - 1}])", "batch": cfg.batch,
+    return {"workload": f"{cfg.name} (workload {args.workload} of 5, configs[{args.workload - 1}])", "batch": cfg.batch,
             "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
             "prompt_len": [cfg.prompt_min, cfg.prompt_max], "window_w": cfg.window_w, "recent_r": cfg.recent_r,
             "alpha": cfg.alpha, "layers_per_step": cfg.n_layers, "seed": cfg.seed,
