@@ -324,15 +324,6 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         for (int it = 0; it < min(my_n, kKStages); ++it) issue_k(it);
         for (int it = 0; it < min(my_n, kVStages); ++it) issue_v(it);
     }
-    // The appended token's rows are fetched now by the warp that will meet slot l_old (the unit's last tile), so that
-    // their latency (a PCIe round trip when the caller's buffers are pinned host memory) is off that tile's path.
-    unsigned char* newrow = smem + lay.newrow;
-    const bool new_is_mine = l_old >= begin && l_old < end && ((l_old - begin) / kTileKeys) % NW == warp;
-    if (new_is_mine) {
-        const unsigned char* src = lane < 16 ? reinterpret_cast<const unsigned char*>(p.k_new) + ((size_t)u * 16 + lane) * 16
-                                             : reinterpret_cast<const unsigned char*>(p.v_new) + ((size_t)u * 16 + lane - 16) * 16;
-        cp_async16(smem_addr(newrow + lane * 16), src);
-    }
     __syncthreads();                                              // s_failed is initialised for everybody
 
     // queries widened to fp64 once per block; a single-split unit also fetches the registers and positions of the
@@ -362,6 +353,18 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             unpack8_to_double(raw, qd[g]);
         }
     }
+    // The appended token's rows are fetched ahead by the warp that will meet slot l_old (the unit's last tile), so that
+    // their latency (a PCIe round trip when the caller's buffers are pinned host memory) is off that tile's path;
+    // requested once the warp's first tile is done, i.e. after the queries, which every warp needs first and which
+    // share that bus.
+    unsigned char* newrow = smem + lay.newrow;
+    const bool new_is_mine = l_old >= begin && l_old < end && ((l_old - begin) / kTileKeys) % NW == warp;
+    auto fetch_new_rows = [&]() {
+        const unsigned char* src = lane < 16 ? reinterpret_cast<const unsigned char*>(p.k_new) + ((size_t)u * 16 + lane) * 16
+                                             : reinterpret_cast<const unsigned char*>(p.v_new) + ((size_t)u * 16 + lane - 16) * 16;
+        cp_async16(smem_addr(newrow + lane * 16), src);
+    };
+    if (new_is_mine && my_n <= 1) fetch_new_rows();              // its only tile is the one with the new row
     double M[G], Zl[G];
     unsigned long long acc2[G][4];                                // P.V accumulators: channel pairs (2e, 2e+1) of this lane's 8
 #pragma unroll
@@ -396,6 +399,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         qk_tile<G>(ktile, qd, lane, sown);
         __syncwarp();
         if (lane == 0 && it + kKStages < my_n) { fence_async_smem(); issue_k(it + kKStages); }
+        if (new_is_mine && it == 0 && my_n > 1) fetch_new_rows();  // the queries are in: the bus is free for these
 
         const bool valid = key_own < n_valid;
         const int j_own = k0 + key_own;
