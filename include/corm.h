@@ -177,6 +177,13 @@ corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int3
 corm_status_t corm_cache_set_similarity_monitor(corm_cache_t* cache, int32_t enabled);
 corm_status_t corm_cache_similarity(corm_cache_t* cache, double* sum_host, int64_t* count_host, void* stream);
 
+/* The tiled prompt pass (bf16, head_dim 128) places each logit of its second launch on one side of its exact
+ * threshold with an fp32 dot product wherever a proven bound on the fp32 accumulation error allows, and forms the
+ * logit again in fp64 where it does not, so results never depend on this. `scale` >= 1 multiplies the bound
+ * (default 1): larger values send more logits through the exact path, which is how the tests exercise it.
+ * Errors: INVALID_ARG. */
+corm_status_t corm_cache_set_bound_scale(corm_cache_t* cache, double scale);
+
 int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
 
 const char* corm_status_string(corm_status_t status);

@@ -83,6 +83,8 @@ def load_library():
     lib.corm_cache_set_similarity_monitor.argtypes = [vp, ctypes.c_int32]
     lib.corm_cache_similarity.restype = ctypes.c_int
     lib.corm_cache_similarity.argtypes = [vp, vp, vp, vp]
+    lib.corm_cache_set_bound_scale.restype = ctypes.c_int
+    lib.corm_cache_set_bound_scale.argtypes = [vp, ctypes.c_double]
     lib.corm_cache_kernel_launches.restype = i64
     lib.corm_cache_kernel_launches.argtypes = [vp]
     lib.corm_status_string.restype = ctypes.c_char_p
@@ -219,6 +221,11 @@ class CormCache:
         _check("corm_cache_similarity", self.lib.corm_cache_similarity(self.handle, ctypes.byref(total), ctypes.byref(n),
                                                                      _stream_ptr(stream)))
         return total.value, n.value
+
+    def corm_cache_set_bound_scale(self, scale):
+        """Multiplies the proven fp32 error bound of the tiled prompt pass (>= 1; results never change, only how many
+        logits are formed again in fp64)."""
+        _check("corm_cache_set_bound_scale", self.lib.corm_cache_set_bound_scale(self.handle, float(scale)))
 
     def corm_cache_kernel_launches(self):
         return int(self.lib.corm_cache_kernel_launches(self.handle))

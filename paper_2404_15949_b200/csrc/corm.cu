@@ -119,6 +119,7 @@ struct corm_cache {
     std::vector<cudaEvent_t> readback_ev;
     std::vector<int> readback_pending, last_readback_step;
     int tune_split_len = 0, allow_fast = 1;
+    double bound_scale = 1.0;
     int monitor_similarity = 0;
     std::vector<int> have_q_prev;                 // the layer's previous decode queries are stored
     int sm_count = 148;
@@ -390,6 +391,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.p_max = p_max; p.w = cf.window_w; p.r = cf.recent_r;
     p.log_alpha = log_alpha_of(c);
+    p.bound_scale = c->bound_scale;
     corm_status_t rc = CORM_ERR_UNSUPPORTED;
     int n_launched = 1;
     if (cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->allow_fast) {     // two-launch tiled pass
@@ -686,6 +688,12 @@ corm_status_t corm_cache_similarity(corm_cache_t* c, double* sum_host, int64_t* 
     unsigned long long n;
     std::memcpy(&n, buf + 8, 8);
     *count_host = (int64_t)n;
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_set_bound_scale(corm_cache_t* c, double scale) {
+    if (!c || !(scale >= 1.0) || !std::isfinite(scale)) return CORM_ERR_INVALID_ARG;
+    c->bound_scale = scale;
     return CORM_OK;
 }
 

@@ -37,6 +37,14 @@ inline cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
     return e;
 }
 
+// |fp32 dot - exact dot| <= kDotErr * |q| * |k| for a 128-term dot product of bf16 values formed the way the fast
+// kernels fold it (bf16 x bf16 products are exact in fp32): 7 roundings in a lane's 8-term FMA chain and 5 in the
+// cross-lane fold make 12 * 2^-24 to first order; 16 * 2^-24 leaves a third of slack for the higher-order terms and
+// for the rounding of the fp32 key norm itself.
+constexpr double kDotErr = 16.0 / 16777216.0;
+// 1 / sqrt(head_dim), the scale of Eq. 2's exponent
+__host__ __device__ constexpr double inv_root_dim(int D) { return D == 128 ? 0.088388347648318440550 : 0.125; }
+
 // Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
 enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_IMPORTANT = 4, CNT_COUNT = 5 };
 
@@ -82,6 +90,7 @@ struct PromptParams {
     double* stash;            // scratch, reused for temporary registers
     int32_t U, Hkv, C, p_max, w, r;
     double log_alpha;
+    double bound_scale;       // multiplies the proven fp32 error bound of the tiled pass (1; tests raise it)
 };
 
 __host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D; }

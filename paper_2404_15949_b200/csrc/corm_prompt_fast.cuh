@@ -30,7 +30,7 @@ struct PromptFastParams {
 };
 
 __host__ __device__ inline size_t prompt_fast_smem(int rows, int C) {
-    size_t a = (size_t)rows * 256 + (size_t)kPromptFastWarps * rows * 16 + (size_t)rows * 8;   // q rows (bf16), per-warp (m, Z), thresholds
+    size_t a = (size_t)rows * 256 + (size_t)kPromptFastWarps * rows * 16 + (size_t)rows * 16;  // q rows (bf16), per-warp (m, Z), thresholds + error factors
     size_t b = (size_t)2 * ((C + 31) / 32 + 2) * 4;                                            // keep mask + prefix (last arriver)
     return a + b + 256;
 }
@@ -73,9 +73,74 @@ __device__ __forceinline__ void qk_tile_clamped(const unsigned char* ktile, int 
     for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
 }
 
+// fp32 form of qk_tile_clamped (bf16 x bf16 products are exact in fp32), with one more folded row: the squared norm
+// of the lane's key, which scales the proven bound kDotErr |q| |k| on the accumulation error of its logits.
+template <int G>
+__device__ __forceinline__ void qk_tile_clamped32(const unsigned char* ktile, int n_valid, const float (&qf)[G][8],
+                                                  int lane, float (&sown)[G], float& n2own) {
+    const int h = lane >> 4, i = lane & 15, m = i >> 1, b0 = i & 1;
+    float r[2][G + 1];
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        float a[G + 1][8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const int key = min(16 * h + 8 * (it ^ b0) + (s ^ m), n_valid - 1);
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(ktile + key * kRowBytes + i * 16));
+            float kf[8];
+            unpack8_to_float(raw, kf);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float acc = qf[g][0] * kf[0];
+#pragma unroll
+                for (int e = 1; e < 8; ++e) acc = fmaf(qf[g][e], kf[e], acc);
+                a[g][s] = acc;
+            }
+            float nn = kf[0] * kf[0];
+#pragma unroll
+            for (int e = 1; e < 8; ++e) nn = fmaf(kf[e], kf[e], nn);
+            a[G][s] = nn;
+        }
+#pragma unroll
+        for (int g = 0; g <= G; ++g) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 4], 8);
+#pragma unroll
+            for (int s = 0; s < 2; ++s) a[g][s] += __shfl_xor_sync(0xffffffffu, a[g][s + 2], 4);
+            a[g][0] += __shfl_xor_sync(0xffffffffu, a[g][1], 2);
+            r[it][g] = a[g][0];
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
+    n2own = r[0][G] + __shfl_xor_sync(0xffffffffu, r[1][G], 1);
+}
+
+// One logit exactly: query row q (128 bf16 in shared memory) against key row k (128 bf16 in global memory), fp64.
+__device__ __noinline__ double exact_logit(const uint16_t* q, const unsigned char* k) {
+    double acc = 0.0;
+    for (int c = 0; c < 16; ++c) {
+        const uint4 kr = __ldg(reinterpret_cast<const uint4*>(k) + c);
+        const uint4 qr = *reinterpret_cast<const uint4*>(q + c * 8);
+        double kd[8], qd[8];
+        unpack8_to_double(kr, kd);
+        unpack8_to_double(qr, qd);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fma(qd[e], kd[e], acc);
+    }
+    return acc;
+}
+
 // Rows of one launch are numbered r = (rho - slot0) * G + g (query slot rho of the window, head g); the query of
 // slot rho sits at prompt position P - (w - 1 - rho) and exists iff rho >= w - min(P, w). Windows whose rows do not
 // fit one launch (more than 64 rows) are recorded by several launch pairs, oldest slots first.
+__device__ __forceinline__ void load_row_group32(const uint16_t* q_sm, int group, int ci, float (&qf)[4][8]) {
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(q_sm + (size_t)(4 * group + x) * 128 + ci * 8);
+        unpack8_to_float(raw, qf[x]);
+    }
+}
 __device__ __forceinline__ void load_row_group(const uint16_t* q_sm, int group, int ci, double (&qd)[4][8]) {
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
@@ -211,11 +276,21 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     if (split >= n_act) return;
     uint16_t* q_sm = reinterpret_cast<uint16_t*>(smem);
     double* thr_sm = reinterpret_cast<double*>(smem + (size_t)rows_pad * 256 + (size_t)NW * rows_pad * 16);
-    uint32_t* keepmask = reinterpret_cast<uint32_t*>(thr_sm + rows_pad);
+    double* err_sm = thr_sm + rows_pad;                          // kDotErr |q_r| / sqrt(d): times |k_j| it bounds a logit's error
+    uint32_t* keepmask = reinterpret_cast<uint32_t*>(err_sm + rows_pad);
     int* prefix = reinterpret_cast<int*>(keepmask + (p.C + 31) / 32 + 2);
     stage_q_rows(p, u, G, slot0, rows, rows_pad, q_sm);
     const double* thr = reinterpret_cast<const double*>(fp.partials) + (size_t)p.U * fp.n_splits * rows_pad * 2 + (size_t)u * rows_pad;
     for (int r = tid; r < rows_pad; r += NT) thr_sm[r] = __ldcg(thr + r);
+    __syncthreads();
+    for (int r = tid; r < rows_pad; r += NT) {
+        double n2 = 0.0;
+        for (int c = 0; c < 128; ++c) {
+            const double x = (double)__uint_as_float((uint32_t)q_sm[(size_t)r * 128 + c] << 16);
+            n2 = fma(x, x, n2);
+        }
+        err_sm[r] = p.bound_scale * kDotErr * inv_root_dim(128) * sqrt(n2) * (1.0 + 1e-6);
+    }
     __syncthreads();
     const unsigned char* Kp = reinterpret_cast<const unsigned char*>(p.k_prompt) + (size_t)u * p.p_max * kRowBytes;
     const unsigned char* Vp = reinterpret_cast<const unsigned char*>(p.v_prompt) + (size_t)u * p.p_max * kRowBytes;
@@ -231,16 +306,27 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
         uint32_t reg = 0u;
         for (int gi = 0; gi < groups; ++gi) {
             if (slot0 + (4 * gi + 3) / G < w - wp) continue;                      // none of these queries exists
-            double qd[4][8], sown[4];
-            load_row_group(q_sm, gi, ci, qd);
-            qk_tile_clamped<4>(Kp + (size_t)k0 * kRowBytes, n_valid, qd, lane, sown);
+            // The thresholds are exact (fp64, from the first launch), so a logit only has to be placed on one side of
+            // its threshold: an fp32 dot product does that whenever it is farther from it than the proven bound on
+            // its own accumulation error; the rare logit inside the bound is formed again exactly.
+            float qf[4][8], s32[4], kn2;
+            load_row_group32(q_sm, gi, ci, qf);
+            qk_tile_clamped32<4>(Kp + (size_t)k0 * kRowBytes, n_valid, qf, lane, s32, kn2);
+            const double kn = sqrt((double)kn2) * (1.0 + 1e-6);
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 const int r = 4 * gi + x, rho = slot0 + r / G;
                 const bool exists = r < rows && rho >= w - wp;
                 const int qpos = P - (w - 1 - rho);
+                bool imp = false;
+                if (exists && pos_own <= qpos) {
+                    const double margin = (double)s32[x] * inv_root_d - thr_sm[r], err = err_sm[r] * kn;
+                    if (margin >= err) imp = true;
+                    else if (!(margin < -err))
+                        imp = exact_logit(q_sm + (size_t)r * 128, Kp + (size_t)(k0 + key_own) * kRowBytes) * inv_root_d >= thr_sm[r];
+                }
                 // Definition 3.1 in log form; keys newer than the query keep a 0 bit (Algorithm 1's zero padding)
-                if (exists && pos_own <= qpos && sown[x] * inv_root_d >= thr_sm[r]) {
+                if (imp) {
                     if (w <= 32) reg |= 1u << (w - 1 - rho);
                     else reg = max(reg, (uint32_t)qpos);
                 }

@@ -88,6 +88,20 @@ def test_adjacent_query_similarity_monitor(dtype, d, G):
     assert 0.0 < so / no < 1.0                                   # the generator's queries drift slowly (Section 3.3)
 
 
+@pytest.mark.parametrize("G,w,scale", [(1, 8, 1.0), (4, 8, 1e3), (1, 8, 1e12), (4, 40, 1e12)])
+def test_prompt_pass_fp32_placement_and_exact_path(G, w, scale):
+    """Second launch of the tiled prompt pass: fp32 logits against exact thresholds where a proven error bound allows,
+    fp64 again where it does not. Inflating the bound (at 1e12: every logit) must not change a single register."""
+    cfg = CONFIGS[1].with_(name="prompt32", batch=2, n_q_heads=2 * G, n_kv_heads=2, head_dim=128, dtype="bf16",
+                           prompt_min=500, prompt_max=900, steps=4, window_w=w, recent_r=16,
+                           gqa_rho=0.7 if G > 1 else 0.0, hh_min=2, hh_max=6, seed=578)
+    data = generate(cfg)
+    gpu, orc = _pair(cfg, data)
+    gpu.corm_cache_set_bound_scale(scale)
+    run_free(cfg, data, gpu, orc)
+    assert orc.counters()["near_threshold"] == 0 and orc.counters()["evicted"] > 0
+
+
 def test_alpha_zero_never_evicts():
     cfg = CONFIGS[1].with_(prompt_min=100, prompt_max=100, steps=20, alpha=0.0, dtype="bf16")
     data = generate(cfg)
