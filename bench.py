@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the decode kernel, from the ncu capture summarised in
 # profiles/decode_fast_kernel_batch32_bf16.md (323.9 MB moved for 313.1 MB algorithmic at the captured steps).
 # Set to None whenever the kernel changes until the counters are taken again.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.013}
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.014}
 
 
 def log(*a):
