@@ -273,9 +273,6 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
-    // the verdict launch that may follow is allowed to become resident from here on (it waits for this grid to
-    // complete before it reads anything written here)
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C) {
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
@@ -476,6 +473,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         if (lane == 0 && it + kVStages < my_n) { fence_async_smem(); issue_v(it + kVStages); }
     }
     if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
+    // The verdict launch that may follow is allowed to become resident once every block of this grid is past its
+    // tiles (it waits for this grid to complete before it reads anything written here). Allowing it from the top of
+    // the kernel costs 1.4 us per step on 128 units of 1600 keys: its waiting blocks take room next to streaming ones.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // fold the warp: lane-private sums of Z, the two halves of acc
     float acc[G][8];
