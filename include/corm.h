@@ -81,6 +81,27 @@ size_t corm_cache_arena_bytes(const corm_config_t* cfg);
  * Errors: INVALID_ARG (null/invalid fields), UNSUPPORTED (head_dim, group, w > 256), ARENA_TOO_SMALL, CUDA. */
 corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, size_t arena_bytes,
                                 corm_cache_t** out);
+
+/* Paged variant of the cache (the paper's result is KV memory saved, abstract and Section 5: with one slab of
+ * max_tokens rows per unit that saving is only a count; here evicted keys give their memory back). K and V of a
+ * layer live in one pool of `pool_pages` pages of 32 keys shared by all units of the layer; a unit holds
+ * live / 32 + 1 pages (the last one takes its next append) listed in its page table, claims a page when an append
+ * crosses a page boundary and returns pages as its live length shrinks. Registers and positions (8 bytes per key)
+ * stay in per-unit arrays of max_tokens entries, and max_tokens still bounds a unit's live length. Every other call
+ * works on a paged cache unchanged and gives the same results as on a slab cache; slot order and live lengths are
+ * identical too (the page table only changes where a slot's rows are stored).
+ *   pool_pages  pages per layer: a multiple of 32, >= batch * n_kv_heads (a unit always owns one page).
+ * A pool that runs out: the unit that could not get a page reports CORM_ERR_CAPACITY through the device status at
+ * its next decode step and is left untouched from then on, like a unit whose slab is full; a prompt pass whose
+ * survivors do not fit reports the same and leaves the unit empty. corm_compress_prompt on a layer returns all of
+ * that layer's pages to the pool first.
+ * Errors: as corm_cache_create; INVALID_ARG for a bad pool_pages (corm_cache_arena_bytes_paged returns 0). */
+size_t corm_cache_arena_bytes_paged(const corm_config_t* cfg, int32_t pool_pages);
+corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pages, void* arena_device,
+                                      size_t arena_bytes, corm_cache_t** out);
+/* Pages of one layer's pool in use and in total (0 and 0 for a slab cache). Synchronises `stream`. */
+corm_status_t corm_cache_pool_usage(corm_cache_t* cache, int32_t layer, int64_t* pages_in_use, int64_t* pages_total,
+                                    void* stream);
 corm_status_t corm_cache_destroy(corm_cache_t* cache);
 
 /* Empties every unit (asynchronous on `stream`); a prompt pass is needed again before decoding. */

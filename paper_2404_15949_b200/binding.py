@@ -57,6 +57,12 @@ def load_library():
     lib.corm_cache_arena_bytes.argtypes = [cfgp]
     lib.corm_cache_create.restype = i32
     lib.corm_cache_create.argtypes = [cfgp, vp, sz, ctypes.POINTER(vp)]
+    lib.corm_cache_arena_bytes_paged.restype = sz
+    lib.corm_cache_arena_bytes_paged.argtypes = [cfgp, i32]
+    lib.corm_cache_create_paged.restype = i32
+    lib.corm_cache_create_paged.argtypes = [cfgp, i32, vp, sz, ctypes.POINTER(vp)]
+    lib.corm_cache_pool_usage.restype = i32
+    lib.corm_cache_pool_usage.argtypes = [vp, i32, vp, vp, vp]
     lib.corm_cache_destroy.restype = i32
     lib.corm_cache_destroy.argtypes = [vp]
     lib.corm_cache_reset.restype = i32
@@ -119,7 +125,9 @@ class CormCache:
     """Owns the arena tensor (torch device memory) and the library's host object."""
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, window_w, recent_r, alpha,
-                 kv_dtype="bf16", device=0):
+                 kv_dtype="bf16", device=0, pool_pages=0):
+        """pool_pages = 0: one slab of max_tokens rows per unit; > 0: a paged cache with that many 32-key pages of K
+        and of V per layer (corm_cache_create_paged)."""
         self.lib = load_library()
         code = {"bf16": CORM_BF16, "f32": CORM_F32}[kv_dtype]
         self.cfg = CormConfig(n_layers, batch, n_q_heads, n_kv_heads, head_dim, max_tokens, window_w, recent_r,
@@ -127,13 +135,14 @@ class CormCache:
         self._q_shape = (batch, n_q_heads, head_dim)
         self._kv_shape = (batch, n_kv_heads, head_dim)
         self.kv_dtype, self.dtype, self.device = code, _torch_dtype(code), torch.device("cuda", device)
-        nbytes = corm_cache_arena_bytes(self.cfg)
+        self.pool_pages = int(pool_pages)
+        nbytes = int(self.lib.corm_cache_arena_bytes_paged(ctypes.byref(self.cfg), self.pool_pages))
         if nbytes == 0:
-            raise CormError("corm_cache_arena_bytes", 1)
+            raise CormError("corm_cache_arena_bytes_paged", 1)
         self.arena = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
         handle = ctypes.c_void_p()
-        _check("corm_cache_create", self.lib.corm_cache_create(ctypes.byref(self.cfg), self.arena.data_ptr(), nbytes,
-                                                               ctypes.byref(handle)))
+        _check("corm_cache_create_paged", self.lib.corm_cache_create_paged(
+            ctypes.byref(self.cfg), self.pool_pages, self.arena.data_ptr(), nbytes, ctypes.byref(handle)))
         self.handle = handle
 
     def close(self):
@@ -198,6 +207,13 @@ class CormCache:
         return {name: getattr(st, name) for name, _ in CormStats._fields_}
 
     # ---- helpers --------------------------------------------------------------------------------------------------
+    def corm_cache_pool_usage(self, layer=0, stream=None):
+        """(pages in use, pages in total) of one layer's pool; (0, 0) for a slab cache."""
+        used, total = ctypes.c_int64(0), ctypes.c_int64(0)
+        _check("corm_cache_pool_usage", self.lib.corm_cache_pool_usage(self.handle, layer, ctypes.byref(used),
+                                                                       ctypes.byref(total), _stream_ptr(stream)))
+        return int(used.value), int(total.value)
+
     def corm_cache_reset(self, stream=None):
         _check("corm_cache_reset", self.lib.corm_cache_reset(self.handle, _stream_ptr(stream)))
 

@@ -28,7 +28,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, q_prev, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, page_table, page_bits, q_prev, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -54,14 +54,24 @@ bool config_ok(const corm_config_t* c, corm_status_t* why) {
 
 int max_splits_of(const corm_config_t& c) { return (c.max_tokens + kMinSplit - 1) / kMinSplit; }
 
-Layout make_layout(const corm_config_t& c) {
+int pt_stride_of(const corm_config_t& c) { return (c.max_tokens + kPageKeys - 1) / kPageKeys; }
+
+// pool_pages = 0: one slab of max_tokens rows per unit; > 0: that many 32-key pages of K and of V per layer
+bool pool_ok(const corm_config_t& c, int pool_pages) {
+    if (pool_pages == 0) return true;
+    const long long U = (long long)c.batch * c.n_kv_heads;
+    return pool_pages > 0 && pool_pages % 32 == 0 && pool_pages >= U;     // every unit always owns at least one page
+}
+
+Layout make_layout(const corm_config_t& c, int pool_pages) {
     Layout L{};
     const size_t U = (size_t)c.batch * c.n_kv_heads, Ltot = c.n_layers, C = c.max_tokens, D = c.head_dim;
     const size_t e = c.kv_dtype == CORM_BF16 ? 2 : 4, G = c.n_q_heads / c.n_kv_heads;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
-    L.K = take(Ltot * U * C * D * e);
-    L.V = take(Ltot * U * C * D * e);
+    const size_t kv_rows = pool_pages ? (size_t)pool_pages * kPageKeys : U * C;   // rows of K (and of V) per layer
+    L.K = take(Ltot * kv_rows * D * e);
+    L.V = take(Ltot * kv_rows * D * e);
     L.word = take(Ltot * U * C * 4);
     L.pos = take(Ltot * U * C * 4);
     L.bookkeeping_begin = off;
@@ -73,6 +83,8 @@ Layout make_layout(const corm_config_t& c) {
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
     L.sim_acc = take(16);
+    L.page_table = take(pool_pages ? Ltot * U * pt_stride_of(c) * 4 : 0);
+    L.page_bits = take(pool_pages ? Ltot * (size_t)(pool_pages / 32) * 4 : 0);
     L.bookkeeping_end = off;
     L.q_prev = take(Ltot * (size_t)c.batch * c.n_q_heads * D * e);
     L.stash = take(U * G * C * 8);
@@ -124,6 +136,7 @@ struct corm_cache {
     std::vector<int> have_q_prev;                 // the layer's previous decode queries are stored
     int sm_count = 148;
     long long launches = 0;
+    int pool_pages = 0, pt_stride = 0;            // paged cache: pages per layer, page-table entries per unit
 };
 
 namespace {
@@ -145,6 +158,26 @@ template <typename F> corm_status_t dispatch(const corm_cache* c, F&& f) {
 
 unsigned char* layer_ptr(const corm_cache* c, size_t base, size_t per_layer_bytes, int layer) {
     return c->arena + base + per_layer_bytes * (size_t)layer;
+}
+
+// bytes of K (and of V) one layer holds: its units' slabs or its page pool
+size_t kv_layer_bytes(const corm_cache* c) {
+    const size_t rows = c->pool_pages ? (size_t)c->pool_pages * kPageKeys : (size_t)c->U * c->cfg.max_tokens;
+    return rows * c->cfg.head_dim * c->e;
+}
+
+int32_t* page_table_ptr(const corm_cache* c, int layer) {
+    return reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.page_table, (size_t)c->U * c->pt_stride * 4, layer));
+}
+uint32_t* page_bits_ptr(const corm_cache* c, int layer) {
+    return reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.page_bits, (size_t)(c->pool_pages / 32) * 4, layer));
+}
+
+template <typename P> void set_paging(const corm_cache* c, int layer, P& p) {
+    p.page_table = c->pool_pages ? page_table_ptr(c, layer) : nullptr;
+    p.page_bits = c->pool_pages ? page_bits_ptr(c, layer) : nullptr;
+    p.pool_pages = c->pool_pages;
+    p.pt_stride = c->pt_stride;
 }
 
 int32_t* live_buf(const corm_cache* c, int layer, int parity) {
@@ -195,8 +228,9 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     const corm_config_t& cf = c->cfg;
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
     DecodeParams p{};
-    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
-    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.K = layer_ptr(c, c->lay.K, kv_layer_bytes(c), layer);
+    p.V = layer_ptr(c, c->lay.V, kv_layer_bytes(c), layer);
+    set_paging(c, layer, p);
     p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
     p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
     p.live_in = live_buf(c, layer, c->parity[layer]);
@@ -266,19 +300,27 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
 
 extern "C" {
 
-size_t corm_cache_arena_bytes(const corm_config_t* cfg) {
+size_t corm_cache_arena_bytes(const corm_config_t* cfg) { return corm_cache_arena_bytes_paged(cfg, 0); }
+
+size_t corm_cache_arena_bytes_paged(const corm_config_t* cfg, int32_t pool_pages) {
     corm_status_t why;
-    if (!config_ok(cfg, &why)) return 0;
-    return make_layout(*cfg).total;
+    if (!config_ok(cfg, &why) || !pool_ok(*cfg, pool_pages)) return 0;
+    return make_layout(*cfg, pool_pages).total;
 }
 
 corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, size_t arena_bytes, corm_cache_t** out) {
+    return corm_cache_create_paged(cfg, 0, arena_device, arena_bytes, out);
+}
+
+corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pages, void* arena_device, size_t arena_bytes,
+                                      corm_cache_t** out) {
     corm_status_t why;
     if (!out) return CORM_ERR_INVALID_ARG;
     *out = nullptr;
     if (!config_ok(cfg, &why)) return why;
+    if (!pool_ok(*cfg, pool_pages)) return CORM_ERR_INVALID_ARG;
     if (!arena_device || (reinterpret_cast<uintptr_t>(arena_device) % kAlign)) return CORM_ERR_INVALID_ARG;
-    Layout lay = make_layout(*cfg);
+    Layout lay = make_layout(*cfg, pool_pages);
     if (arena_bytes < lay.total) return CORM_ERR_ARENA_TOO_SMALL;
     DeviceGuard guard(cfg->device);
     if (!guard.ok) return CORM_ERR_CUDA;
@@ -290,6 +332,8 @@ corm_status_t corm_cache_create(const corm_config_t* cfg, void* arena_device, si
     c->U = cfg->batch * cfg->n_kv_heads;
     c->G = cfg->n_q_heads / cfg->n_kv_heads;
     c->e = cfg->kv_dtype == CORM_BF16 ? 2 : 4;
+    c->pool_pages = pool_pages;
+    c->pt_stride = pool_pages ? pt_stride_of(*cfg) : 0;
     c->parity.assign(cfg->n_layers, 0);
     c->steps.assign(cfg->n_layers, 0);
     c->ready.assign(cfg->n_layers, 0);
@@ -380,8 +424,13 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     PromptParams p{};
     p.k_prompt = k_prompt; p.v_prompt = v_prompt; p.q_last = q_last;
     p.prompt_lens = base_tokens;
-    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
-    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.K = layer_ptr(c, c->lay.K, kv_layer_bytes(c), layer);
+    p.V = layer_ptr(c, c->lay.V, kv_layer_bytes(c), layer);
+    set_paging(c, layer, p);
+    if (c->pool_pages) {   // whatever the layer held is replaced: all its pages return to the pool
+        CORM_CUDA(cudaMemsetAsync(p.page_table, 0, U * c->pt_stride * 4, st));
+        CORM_CUDA(cudaMemsetAsync(p.page_bits, 0, (size_t)(c->pool_pages / 32) * 4, st));
+    }
     p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
     p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
     p.live_out = live_buf(c, layer, 0);
@@ -524,8 +573,9 @@ corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void
     if (rc != CORM_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams p{};
-    p.K = layer_ptr(c, c->lay.K, U * C * D * c->e, layer);
-    p.V = layer_ptr(c, c->lay.V, U * C * D * c->e, layer);
+    p.K = layer_ptr(c, c->lay.K, kv_layer_bytes(c), layer);
+    p.V = layer_ptr(c, c->lay.V, kv_layer_bytes(c), layer);
+    set_paging(c, layer, p);
     p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
     p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
     p.live_in = live_buf(c, layer, c->parity[layer]);
@@ -615,8 +665,22 @@ corm_status_t corm_cache_export_state(corm_cache_t* c, int32_t layer, int32_t se
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U, u = (size_t)seq * cf.n_kv_heads + kv_head;
     const size_t row_bytes = C * D * c->e;
     int32_t bt = 0, bo = 0, lv = 0;
-    if (k_host) CORM_CUDA(cudaMemcpyAsync(k_host, layer_ptr(c, c->lay.K, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
-    if (v_host) CORM_CUDA(cudaMemcpyAsync(v_host, layer_ptr(c, c->lay.V, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
+    if (c->pool_pages) {   // page by page, in slot order; slots of pages the unit does not own are left as they are
+        std::vector<int32_t> pt(c->pt_stride);
+        CORM_CUDA(cudaMemcpyAsync(pt.data(), page_table_ptr(c, layer) + u * c->pt_stride, pt.size() * 4, cudaMemcpyDeviceToHost, st));
+        CORM_CUDA(cudaStreamSynchronize(st));
+        const size_t page_bytes = (size_t)kPageKeys * D * c->e;
+        for (int i = 0; i < c->pt_stride; ++i) {
+            if (pt[i] <= 0 || pt[i] > c->pool_pages) continue;
+            const size_t n = std::min(page_bytes, row_bytes - (size_t)i * page_bytes);
+            const size_t at = (size_t)(pt[i] - 1) * page_bytes;
+            if (k_host) CORM_CUDA(cudaMemcpyAsync(static_cast<unsigned char*>(k_host) + (size_t)i * page_bytes, layer_ptr(c, c->lay.K, kv_layer_bytes(c), layer) + at, n, cudaMemcpyDeviceToHost, st));
+            if (v_host) CORM_CUDA(cudaMemcpyAsync(static_cast<unsigned char*>(v_host) + (size_t)i * page_bytes, layer_ptr(c, c->lay.V, kv_layer_bytes(c), layer) + at, n, cudaMemcpyDeviceToHost, st));
+        }
+    } else {
+        if (k_host) CORM_CUDA(cudaMemcpyAsync(k_host, layer_ptr(c, c->lay.K, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
+        if (v_host) CORM_CUDA(cudaMemcpyAsync(v_host, layer_ptr(c, c->lay.V, U * row_bytes, layer) + u * row_bytes, row_bytes, cudaMemcpyDeviceToHost, st));
+    }
     if (word_host) CORM_CUDA(cudaMemcpyAsync(word_host, layer_ptr(c, c->lay.word, U * C * 4, layer) + u * C * 4, C * 4, cudaMemcpyDeviceToHost, st));
     if (pos_host) CORM_CUDA(cudaMemcpyAsync(pos_host, layer_ptr(c, c->lay.pos, U * C * 4, layer) + u * C * 4, C * 4, cudaMemcpyDeviceToHost, st));
     CORM_CUDA(cudaMemcpyAsync(&lv, live_buf(c, layer, c->parity[layer]) + u, 4, cudaMemcpyDeviceToHost, st));
@@ -643,7 +707,41 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U, u = (size_t)seq * cf.n_kv_heads + kv_head;
     const size_t row_bytes = C * D * c->e, n = (size_t)live_len;
-    if (n) {
+    if (c->pool_pages) {
+        // The host edits the layer's page bitmap and this unit's page table itself (nothing else runs meanwhile: the
+        // stream is drained first): the unit's old pages are returned, live_len / 32 + 1 pages are claimed, rows are
+        // copied page by page.
+        CORM_CUDA(cudaStreamSynchronize(st));
+        std::vector<int32_t> pt(c->pt_stride);
+        std::vector<uint32_t> bits(c->pool_pages / 32);
+        int32_t* pt_dev = page_table_ptr(c, layer) + u * c->pt_stride;
+        CORM_CUDA(cudaMemcpy(pt.data(), pt_dev, pt.size() * 4, cudaMemcpyDeviceToHost));
+        CORM_CUDA(cudaMemcpy(bits.data(), page_bits_ptr(c, layer), bits.size() * 4, cudaMemcpyDeviceToHost));
+        for (int i = 0; i < c->pt_stride; ++i) {
+            if (pt[i] > 0 && pt[i] <= c->pool_pages) bits[(pt[i] - 1) >> 5] &= ~(1u << ((pt[i] - 1) & 31));
+            pt[i] = 0;
+        }
+        const int need = std::min(live_len / kPageKeys + 1, c->pt_stride);
+        int next = 0;
+        for (int i = 0; i < need; ++i) {
+            while (next < c->pool_pages && (bits[next >> 5] >> (next & 31) & 1u)) ++next;
+            if (next >= c->pool_pages) return CORM_ERR_CAPACITY;          // nothing has been written to the device yet
+            bits[next >> 5] |= 1u << (next & 31);
+            pt[i] = next + 1;
+        }
+        CORM_CUDA(cudaMemcpy(pt_dev, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice));
+        CORM_CUDA(cudaMemcpy(page_bits_ptr(c, layer), bits.data(), bits.size() * 4, cudaMemcpyHostToDevice));
+        const size_t page_bytes = (size_t)kPageKeys * D * c->e;
+        for (size_t i = 0; i * kPageKeys < n; ++i) {
+            const size_t bytes = std::min(page_bytes, n * D * c->e - i * page_bytes), at = (size_t)(pt[i] - 1) * page_bytes;
+            CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.K, kv_layer_bytes(c), layer) + at, static_cast<const unsigned char*>(k_host) + i * page_bytes, bytes, cudaMemcpyHostToDevice, st));
+            CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.V, kv_layer_bytes(c), layer) + at, static_cast<const unsigned char*>(v_host) + i * page_bytes, bytes, cudaMemcpyHostToDevice, st));
+        }
+        if (n) {
+            CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.word, U * C * 4, layer) + u * C * 4, word_host, n * 4, cudaMemcpyHostToDevice, st));
+            CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.pos, U * C * 4, layer) + u * C * 4, pos_host, n * 4, cudaMemcpyHostToDevice, st));
+        }
+    } else if (n) {
         CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.K, U * row_bytes, layer) + u * row_bytes, k_host, n * D * c->e, cudaMemcpyHostToDevice, st));
         CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.V, U * row_bytes, layer) + u * row_bytes, v_host, n * D * c->e, cudaMemcpyHostToDevice, st));
         CORM_CUDA(cudaMemcpyAsync(layer_ptr(c, c->lay.word, U * C * 4, layer) + u * C * 4, word_host, n * 4, cudaMemcpyHostToDevice, st));
@@ -658,6 +756,21 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     c->ready[layer] = 1;
     c->readback_pending[layer] = 0;   // a read-back enqueued before this import knows nothing of it
     c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
+    return CORM_OK;
+}
+
+corm_status_t corm_cache_pool_usage(corm_cache_t* c, int32_t layer, int64_t* pages_in_use, int64_t* pages_total, void* stream) {
+    if (!layer_ok(c, layer) || !pages_in_use || !pages_total) return CORM_ERR_INVALID_ARG;
+    *pages_in_use = 0;
+    *pages_total = c->pool_pages;
+    if (!c->pool_pages) return CORM_OK;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<uint32_t> bits(c->pool_pages / 32);
+    CORM_CUDA(cudaMemcpyAsync(bits.data(), page_bits_ptr(c, layer), bits.size() * 4, cudaMemcpyDeviceToHost, st));
+    CORM_CUDA(cudaStreamSynchronize(st));
+    for (uint32_t w : bits) *pages_in_use += __builtin_popcount(w);
     return CORM_OK;
 }
 

@@ -72,6 +72,10 @@ struct DecodeParams {
     int32_t single_cap;       // fast kernel: units up to this length finish inside one block (0 = never)
     int32_t inline_finalize;  // fast kernel: the last-arriving split of a longer unit finishes it (else the verdict launch does)
     double log_alpha;         // ln(alpha), -inf for alpha = 0
+    // paged caches only (page_table == nullptr: every unit owns a slab of C rows of K and V)
+    int32_t* page_table;      // [U][pt_stride] page number + 1 of each 32-key page of a unit, 0 = none
+    uint32_t* page_bits;      // [pool_pages / 32] bit set = page in use
+    int32_t pool_pages, pt_stride;
 };
 
 struct PromptParams {
@@ -91,6 +95,9 @@ struct PromptParams {
     int32_t U, Hkv, C, p_max, w, r;
     double log_alpha;
     double bound_scale;       // multiplies the proven fp32 error bound of the tiled pass (1; tests raise it)
+    int32_t* page_table;      // paged caches only, as in DecodeParams
+    uint32_t* page_bits;
+    int32_t pool_pages, pt_stride;
 };
 
 __host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D; }
@@ -172,6 +179,77 @@ __device__ __forceinline__ bool register_needed(uint32_t reg, int w, int t) {
     return w <= 32 ? reg != 0u : (reg != 0u && t - (int)reg < w);
 }
 
+// ---- paged caches --------------------------------------------------------------------------------------------
+// The paper's result is memory saved; with one slab of C rows per unit the saving is only logical. A paged cache
+// keeps K and V of a layer in one pool of 32-key pages (one tile of the streaming kernel) shared by all its units:
+// slot j of a unit lives in row (page_table[j / 32] - 1) * 32 + j % 32 of the pool. Registers and positions stay in
+// per-unit arrays of C entries (8 bytes per key against 2 * D * e). Invariant between steps: a unit of n live keys
+// owns the pages of slots 0 .. n, i.e. n / 32 + 1 pages, so the next append always has a row to go to; the block
+// that finishes a unit's step (or its prompt pass) claims or releases pages to restore it. A unit whose claim failed
+// because the pool is exhausted has no page for its next append: that step reports CORM_ERR_CAPACITY and leaves
+// the unit untouched, like a full slab.
+constexpr int kPageKeys = 32;
+
+// row of slot `slot` in the layer's K / V storage: through the unit's page table, or inside its slab
+__device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, int slot) {
+    return pt_u ? (size_t)(__ldcg(pt_u + (slot >> 5)) - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
+}
+
+// Claims one free page: scans the in-use bitmap from a start word spread by `seed`, sets a clear bit with atomicOr
+// and owns the page iff the bit was clear before. Bounded: every word is visited once and the inner loop ends after
+// at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1 when the pool is exhausted.
+__device__ inline int claim_page(uint32_t* bits, int pool_pages, unsigned seed) {
+    const int n_words = pool_pages >> 5;
+    int i = (int)((seed * 2654435761u) % (unsigned)n_words);
+    for (int tries = 0; tries < n_words; ++tries) {
+        uint32_t w = __ldcg(bits + i);
+        while (w != 0xffffffffu) {
+            const uint32_t bit = 1u << (__ffs((int)~w) - 1);
+            const uint32_t old = atomicOr(bits + i, bit);
+            if (!(old & bit)) return i * 32 + __ffs((int)bit) - 1;
+            w = old | bit;
+        }
+        i = (i + 1 == n_words) ? 0 : i + 1;
+    }
+    return -1;
+}
+
+// Restores the page invariant of unit u after a decode step that took it from l_old live keys (pages 0 .. l_old / 32
+// owned) to new_len. Called by every thread of the block that finished the unit, after its row moves: the barrier
+// below orders the block's reads of rows in released pages before another unit can claim them.
+template <int NT>
+__device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page_bits, int pool_pages, int pt_stride,
+                                             int u, int l_old, int new_len) {
+    if (!page_table) return;
+    __syncthreads();
+    int32_t* pt_u = page_table + (size_t)u * pt_stride;
+    const int have = l_old / kPageKeys + 1, need = new_len / kPageKeys + 1;
+    for (int i = need + (int)threadIdx.x; i < have; i += NT) {
+        const int pg = __ldcg(pt_u + i) - 1;
+        pt_u[i] = 0;
+        if (pg >= 0) atomicAnd(page_bits + (pg >> 5), ~(1u << (pg & 31)));
+    }
+    if (need > have && have < pt_stride && threadIdx.x == 0)      // the next append starts a new page
+        pt_u[have] = claim_page(page_bits, pool_pages, (unsigned)u * 977u + (unsigned)have) + 1;   // 0 if exhausted
+}
+
+// Prompt pass: unit u ends with `kept` live keys and owns no page yet (the pass starts from an empty pool). Claims
+// kept / 32 + 1 pages, one per thread. Returns false (to every thread) if the pool ran out.
+template <int NT>
+__device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* page_bits, int pool_pages, int pt_stride,
+                                                 int u, int kept) {
+    if (!page_table) return true;
+    int32_t* pt_u = page_table + (size_t)u * pt_stride;
+    const int need = min(kept / kPageKeys + 1, pt_stride);
+    int failed = 0;
+    for (int i = (int)threadIdx.x; i < need; i += NT) {
+        const int pg = claim_page(page_bits, pool_pages, (unsigned)u * 977u + (unsigned)i);
+        pt_u[i] = pg + 1;
+        failed |= (pg < 0);
+    }
+    return !__syncthreads_or(failed);      // also makes the table entries visible to the whole block
+}
+
 // Exclusive prefix sums of popc(mask[i]) into prefix[0..nwords], block-wide. scratch holds NT ints.
 // Each thread sums a contiguous run of words; warp 0 scans the NT run totals with shuffles.
 template <int NT>
@@ -214,12 +292,13 @@ __device__ __forceinline__ int kept_before(const uint32_t* mask, const int* pref
 // four rows at a time and issues all their loads before the first store (the copies are latency-, not
 // bandwidth-limited). Rows are D*sizeof(T) bytes = a multiple of 16.
 template <typename T, int D, int NT>
-__device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, int32_t* posu, const int* movers,
-                                                const int* holes, int n_moved) {
+__device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, const int32_t* pt_u, size_t slab_row0, uint32_t* wordu,
+                                                int32_t* posu, const int* movers, const int* holes, int n_moved) {
     constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = 4, NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i0 = warp * kRows; i0 < n_moved; i0 += NW * kRows) {
         int src[kRows], dst[kRows];
+        size_t srow[kRows], drow[kRows];                 // rows of the layer's K / V storage (Kl, Vl)
         uint4 buf[kRows][kIter];
         uint32_t wd = 0u;
         int32_t ps = 0;
@@ -228,6 +307,8 @@ __device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, i
             const bool on = i0 + r < n_moved;
             src[r] = on ? movers[i0 + r] : -1;
             dst[r] = on ? holes[i0 + r] : -1;
+            srow[r] = on ? kv_row(pt_u, slab_row0, src[r]) : 0;
+            drow[r] = on ? kv_row(pt_u, slab_row0, dst[r]) : 0;
         }
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
@@ -235,8 +316,8 @@ __device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, i
 #pragma unroll
             for (int x = 0; x < kIter; ++x) {
                 const int c = lane + 32 * x;
-                if (c < kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Ku + (size_t)src[r] * D) + c);
-                else if (c < 2 * kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Vu + (size_t)src[r] * D) + (c - kChunks));
+                if (c < kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Kl + srow[r] * D) + c);
+                else if (c < 2 * kChunks) buf[r][x] = __ldcg(reinterpret_cast<const uint4*>(Vl + srow[r] * D) + (c - kChunks));
             }
             if (lane == r) { wd = __ldcg(wordu + src[r]); ps = __ldcg(posu + src[r]); }
         }
@@ -246,8 +327,8 @@ __device__ __forceinline__ void block_move_rows(T* Ku, T* Vu, uint32_t* wordu, i
 #pragma unroll
             for (int x = 0; x < kIter; ++x) {
                 const int c = lane + 32 * x;
-                if (c < kChunks) reinterpret_cast<uint4*>(Ku + (size_t)dst[r] * D)[c] = buf[r][x];
-                else if (c < 2 * kChunks) reinterpret_cast<uint4*>(Vu + (size_t)dst[r] * D)[c - kChunks] = buf[r][x];
+                if (c < kChunks) reinterpret_cast<uint4*>(Kl + drow[r] * D)[c] = buf[r][x];
+                else if (c < 2 * kChunks) reinterpret_cast<uint4*>(Vl + drow[r] * D)[c - kChunks] = buf[r][x];
             }
             if (lane == r) { wordu[dst[r]] = wd; posu[dst[r]] = ps; }
         }
@@ -270,8 +351,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     const int cap_words = (p.C + 31) / 32 + 2;
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(smem);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
-    T* Ku = reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D;
-    T* Vu = reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D;
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     const size_t pstride = partial_stride(D);
@@ -370,9 +450,11 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            block_move_rows<T, D, NT>(Ku, Vu, wordu, posu, movers, holes, n_moved);
+            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V), pt_u, (size_t)u * p.C, wordu, posu,
+                                      movers, holes, n_moved);
         }
     }
+    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);

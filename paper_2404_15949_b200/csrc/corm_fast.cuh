@@ -209,8 +209,7 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     const int cap_words = (l + 31) / 32 + 2;
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(lists);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
-    bf16_t* Ku = reinterpret_cast<bf16_t*>(p.K) + (size_t)u * p.C * 128;
-    bf16_t* Vu = reinterpret_cast<bf16_t*>(p.V) + (size_t)u * p.C * 128;
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
@@ -250,9 +249,11 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            block_move_rows<bf16_t, 128, NT>(Ku, Vu, wordu, posu, movers, holes, n_moved);
+            block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), pt_u,
+                                             (size_t)u * p.C, wordu, posu, movers, holes, n_moved);
         }
     }
+    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);
@@ -274,7 +275,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
-    if (l > p.C) {
+    // paged caches: the unit's page table; a unit without a page for the appended row (pool exhausted) is full
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) {
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
@@ -289,8 +292,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kStagesPerWarp * 8;
     float* psm = reinterpret_cast<float*>(smem + lay.psm) + warp * kTileKeys * G;
     double* stash_sm = reinterpret_cast<double*>(smem + lay.stash);
-    const unsigned char* Ku = reinterpret_cast<const unsigned char*>(p.K) + (size_t)u * p.C * kRowBytes;
-    const unsigned char* Vu = reinterpret_cast<const unsigned char*>(p.V) + (size_t)u * p.C * kRowBytes;
+    static_assert(kTileKeys == kPageKeys, "a page is one tile of the streaming kernel");
+    unsigned char* Kl = reinterpret_cast<unsigned char*>(p.K);       // the layer's K / V storage: slabs or page pool
+    unsigned char* Vl = reinterpret_cast<unsigned char*>(p.V);
+    const size_t slab_row0 = (size_t)u * p.C;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
 
@@ -303,13 +308,13 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kKStages;
         const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
         mbar_expect_tx(my_bars + slot * 8, bytes);
-        bulk_load(smem_addr(my_tiles + slot * kTileBytes), Ku + (size_t)k0 * kRowBytes, bytes, my_bars + slot * 8);
+        bulk_load(smem_addr(my_tiles + slot * kTileBytes), Kl + kv_row(pt_u, slab_row0, k0) * kRowBytes, bytes, my_bars + slot * 8);
     };
     auto issue_v = [&](int it) {
         const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kVStages;
         const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
         mbar_expect_tx(my_bars + (kKStages + slot) * 8, bytes);
-        bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vu + (size_t)k0 * kRowBytes, bytes,
+        bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vl + kv_row(pt_u, slab_row0, k0) * kRowBytes, bytes,
                   my_bars + (kKStages + slot) * 8);
     };
     // a warp's barriers and stages are its own: its first copies leave before the block meets at its first barrier
@@ -387,7 +392,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             if (lane < 16) {
                 const uint4 x = *reinterpret_cast<const uint4*>(newrow + lane * 16);
                 *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = x;
-                reinterpret_cast<uint4*>(const_cast<unsigned char*>(Ku) + (size_t)l_old * kRowBytes)[lane] = x;
+                reinterpret_cast<uint4*>(Kl + kv_row(pt_u, slab_row0, l_old) * kRowBytes)[lane] = x;
             }
             if (lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
             __syncwarp();
@@ -448,7 +453,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             if (lane < 16) {
                 const uint4 x = *reinterpret_cast<const uint4*>(newrow + kRowBytes + lane * 16);
                 *reinterpret_cast<uint4*>(vtile + (l_old - k0) * kRowBytes + lane * 16) = x;
-                reinterpret_cast<uint4*>(const_cast<unsigned char*>(Vu) + (size_t)l_old * kRowBytes)[lane] = x;
+                reinterpret_cast<uint4*>(Vl + kv_row(pt_u, slab_row0, l_old) * kRowBytes)[lane] = x;
             }
         }
         if (n_valid < kTileKeys)     // rows the copy did not fetch: make them harmless for 0 * v

@@ -26,7 +26,8 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
-    if (l > p.C) {   // the slab is full: report, leave the unit untouched
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) {   // the slab is full (paged: no page for the new row): report, leave the unit untouched
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
@@ -34,14 +35,16 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     if (split >= n_act) return;
     const int t = __ldg(p.base_tokens + b) + p.step + 1;
     const int begin = split * p.split_len, end = min(l, begin + p.split_len);
-    T* Ku = reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D;
-    T* Vu = reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D;
+    T* Kl = reinterpret_cast<T*>(p.K);                 // the layer's K / V storage: slabs or page pool
+    T* Vl = reinterpret_cast<T*>(p.V);
+    const size_t slab_row0 = (size_t)u * p.C;
 
     // append the current token (Algorithm 1's keys include it; its register starts at zero)
     if (l_old >= begin && l_old < end) {
         const T* kn = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
         const T* vn = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
-        for (int c = tid; c < D; c += NT) { Ku[(size_t)l_old * D + c] = kn[c]; Vu[(size_t)l_old * D + c] = vn[c]; }
+        const size_t row = kv_row(pt_u, slab_row0, l_old);
+        for (int c = tid; c < D; c += NT) { Kl[row * D + c] = kn[c]; Vl[row * D + c] = vn[c]; }
         if (tid == 0) { p.word[(size_t)u * p.C + l_old] = 0u; p.pos[(size_t)u * p.C + l_old] = t; }
         __syncthreads();
     }
@@ -70,8 +73,9 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     const double root_d = sqrt((double)D);
     for (int j = begin + warp; j < end; j += NW) {
         float kf[NPL], vf[NPL];
-        load_slice<T, NPL>(Ku + (size_t)j * D + c0, kf);
-        load_slice<T, NPL>(Vu + (size_t)j * D + c0, vf);
+        const size_t row = kv_row(pt_u, slab_row0, j);
+        load_slice<T, NPL>(Kl + row * D + c0, kf);
+        load_slice<T, NPL>(Vl + row * D + c0, vf);
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             double part = 0.0;
@@ -160,7 +164,14 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
         if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
         return;
     }
-    if (P == 0) { if (tid == 0) p.live_out[u] = 0; return; }
+    if (P == 0) {
+        if (tid == 0) {
+            p.live_out[u] = 0;
+            if (p.page_table)    // an empty unit still owns the page its first append goes to
+                p.page_table[(size_t)u * p.pt_stride] = claim_page(p.page_bits, p.pool_pages, (unsigned)u * 977u) + 1;
+        }
+        return;
+    }
     const int w = p.w, wp = min(P, w);
     const int cs = prompt_chunk_slots(G, w), rows = G * cs;           // window slots per pass, rows per pass
     double* sm_mz = reinterpret_cast<double*>(smem);                   // [NW][rows][2], row = g * cs + (slot - slot0)
@@ -251,16 +262,22 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     const int nwords = (P + 31) / 32;
     block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
     const int kept_total = prefix[nwords];
-    T* Ku = reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D;
-    T* Vu = reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D;
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, kept_total)) {
+        if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }   // the pool is too small
+        return;
+    }
+    T* Kl = reinterpret_cast<T*>(p.K);
+    T* Vl = reinterpret_cast<T*>(p.V);
     constexpr int kChunks = D * Elem<T>::kBytes / 16;
     for (int j = warp; j < P; j += NW) {
         if (!((keepmask[j >> 5] >> (j & 31)) & 1u)) continue;
         const int dst = kept_before(keepmask, prefix, j);
         const uint4* ks = reinterpret_cast<const uint4*>(Kp + (size_t)j * D);
         const uint4* vs = reinterpret_cast<const uint4*>(Vp + (size_t)j * D);
-        uint4* kd = reinterpret_cast<uint4*>(Ku + (size_t)dst * D);
-        uint4* vd = reinterpret_cast<uint4*>(Vu + (size_t)dst * D);
+        const size_t drow = kv_row(pt_u, (size_t)u * p.C, dst);
+        uint4* kd = reinterpret_cast<uint4*>(Kl + drow * D);
+        uint4* vd = reinterpret_cast<uint4*>(Vl + drow * D);
         for (int c = lane; c < 2 * kChunks; c += 32) {
             if (c < kChunks) kd[c] = ks[c];
             else vd[c - kChunks] = vs[c - kChunks];

@@ -269,7 +269,14 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
         if (last_launch && split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
         return;
     }
-    if (P == 0) { if (last_launch && split == 0 && tid == 0) { p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); } return; }
+    if (P == 0) {
+        if (last_launch && split == 0 && tid == 0) {
+            p.live_out[u] = 0; publish_live(p.maxlive, 0, 0);
+            if (p.page_table)    // an empty unit still owns the page its first append goes to
+                p.page_table[(size_t)u * p.pt_stride] = claim_page(p.page_bits, p.pool_pages, (unsigned)u * 977u) + 1;
+        }
+        return;
+    }
     const int rows = fp.rows, rows_pad = (rows + 3) / 4 * 4, groups = rows_pad / 4, slot0 = fp.slot0;
     const int begin = split * fp.split_len, end = min(P, begin + fp.split_len);
     const int n_act = (P + fp.split_len - 1) / fp.split_len;
@@ -363,25 +370,32 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     const int nwords = (P + 31) / 32;
     block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
     const int kept_total = prefix[nwords];
-    unsigned char* Ku = reinterpret_cast<unsigned char*>(p.K) + (size_t)u * p.C * kRowBytes;
-    unsigned char* Vu = reinterpret_cast<unsigned char*>(p.V) + (size_t)u * p.C * kRowBytes;
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, kept_total)) {
+        if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); }
+        return;                                                                       // the pool is too small
+    }
+    unsigned char* Kl = reinterpret_cast<unsigned char*>(p.K);
+    unsigned char* Vl = reinterpret_cast<unsigned char*>(p.V);
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     // a warp takes 8 consecutive prompt rows at a time; lanes 0-15 copy the K row, 16-31 the V row; loads first
     for (int j0 = warp * 8; j0 < P; j0 += NW * 8) {
         uint4 buf[8];
         int dst[8];
+        size_t drow[8];
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
             const int j = j0 + x;
             const bool kept = j < P && ((keepmask[j >> 5] >> (j & 31)) & 1u);
             dst[x] = kept ? kept_before(keepmask, prefix, j) : -1;
+            drow[x] = kept ? kv_row(pt_u, (size_t)u * p.C, dst[x]) : 0;
             if (kept) buf[x] = __ldg(reinterpret_cast<const uint4*>((lane < 16 ? Kp : Vp) + (size_t)j * kRowBytes) + (lane & 15));
         }
 #pragma unroll
         for (int x = 0; x < 8; ++x) {
             if (dst[x] < 0) continue;
-            reinterpret_cast<uint4*>((lane < 16 ? Ku : Vu) + (size_t)dst[x] * kRowBytes)[lane & 15] = buf[x];
+            reinterpret_cast<uint4*>((lane < 16 ? Kl : Vl) + drow[x] * kRowBytes)[lane & 15] = buf[x];
             if (lane == 0) { wordu[dst[x]] = __ldcg(tmp_word + j0 + x); posu[dst[x]] = j0 + x + 1; }
         }
     }

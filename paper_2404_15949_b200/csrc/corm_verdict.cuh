@@ -40,7 +40,8 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     const int u = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
-    if (l > p.C) return;                                                   // reported by the streaming kernel
+    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) return;     // reported by the streaming kernel
     const int n_act = (l + p.split_len - 1) / p.split_len;
     if (n_act == 1 && l <= p.single_cap) return;                           // finished inside the streaming kernel
     const int n_chunks = (l + kVerdictChunk - 1) / kVerdictChunk;
@@ -199,10 +200,11 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
                 }
             }
             __syncthreads();
-            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K) + (size_t)u * p.C * D,
-                                      reinterpret_cast<T*>(p.V) + (size_t)u * p.C * D, wordu, posu, movers, holes, n_moved);
+            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V), pt_u, (size_t)u * p.C, wordu, posu,
+                                      movers, holes, n_moved);
         }
     }
+    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l_old, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);

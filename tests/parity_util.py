@@ -13,10 +13,10 @@ def to_dev(a, dtype):
     return t.to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
 
 
-def make_gpu_cache(cfg, nb, nh, max_tokens=None, n_layers=1):
+def make_gpu_cache(cfg, nb, nh, max_tokens=None, n_layers=1, pool_pages=0):
     from paper_2404_15949_b200.binding import CormCache
     return CormCache(n_layers, nb, nh * cfg.group, nh, cfg.head_dim, max_tokens or cfg.max_tokens, cfg.window_w,
-                     cfg.recent_r, cfg.alpha, cfg.dtype, 0)
+                     cfg.recent_r, cfg.alpha, cfg.dtype, 0, pool_pages=pool_pages)
 
 
 def make_oracle(cfg, nb, nh, max_tokens=None, n_layers=1):
