@@ -167,6 +167,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--window", type=int, default=None, help="override the verdict window w (1..256)")
     ap.add_argument("--recent", type=int, default=None, help="override the protected recent tokens r")
+    ap.add_argument("--pool-pages", type=int, default=0,
+                    help="paged cache with this many 32-key pages per layer (multiple of 32); 0 = one slab per unit")
     args = ap.parse_args()
     cfg = CONFIGS[args.workload]
     if args.alpha is not None:
@@ -200,7 +202,7 @@ def main():
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
-                      cfg.recent_r, cfg.alpha, cfg.dtype, local)
+                      cfg.recent_r, cfg.alpha, cfg.dtype, local, pool_pages=args.pool_pages)
     cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3}[args.finish])
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
@@ -311,6 +313,10 @@ def main():
         "prompt_pass_ms": prompt_ms, "retention_after_prompt": st0["retention"],
         "paper_context": "paper reports KV memory only: up to 70% reduction (V100-32GB / A100-80GB), no throughput",
     }
+    line["arena_bytes"] = int(cache.arena.numel())
+    if args.pool_pages:
+        line["config"]["pool_pages"] = args.pool_pages
+        line["pool_pages_in_use"] = sum(cache.corm_cache_pool_usage(l)[0] for l in range(L))
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"], _ = oracle_baseline(cfg, args.ref_seqs, args.ref_steps)
     print(json.dumps(line), flush=True)

@@ -28,7 +28,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, page_table, page_bits, q_prev, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -85,6 +85,7 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.sim_acc = take(16);
     L.page_table = take(pool_pages ? Ltot * U * pt_stride_of(c) * 4 : 0);
     L.page_bits = take(pool_pages ? Ltot * (size_t)(pool_pages / 32) * 4 : 0);
+    L.page_room = take(pool_pages ? Ltot * U * 4 : 0);
     L.bookkeeping_end = off;
     L.q_prev = take(Ltot * (size_t)c.batch * c.n_q_heads * D * e);
     L.stash = take(U * G * C * 8);
@@ -173,7 +174,12 @@ uint32_t* page_bits_ptr(const corm_cache* c, int layer) {
     return reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.page_bits, (size_t)(c->pool_pages / 32) * 4, layer));
 }
 
+int32_t* page_room_ptr(const corm_cache* c, int layer) {
+    return reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.page_room, (size_t)c->U * 4, layer));
+}
+
 template <typename P> void set_paging(const corm_cache* c, int layer, P& p) {
+    p.page_room = c->pool_pages ? page_room_ptr(c, layer) : nullptr;
     p.page_table = c->pool_pages ? page_table_ptr(c, layer) : nullptr;
     p.page_bits = c->pool_pages ? page_bits_ptr(c, layer) : nullptr;
     p.pool_pages = c->pool_pages;
@@ -430,6 +436,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     if (c->pool_pages) {   // whatever the layer held is replaced: all its pages return to the pool
         CORM_CUDA(cudaMemsetAsync(p.page_table, 0, U * c->pt_stride * 4, st));
         CORM_CUDA(cudaMemsetAsync(p.page_bits, 0, (size_t)(c->pool_pages / 32) * 4, st));
+        CORM_CUDA(cudaMemsetAsync(p.page_room, 0, U * 4, st));
     }
     p.word = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.word, U * C * 4, layer));
     p.pos = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.pos, U * C * 4, layer));
@@ -731,6 +738,8 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
         }
         CORM_CUDA(cudaMemcpy(pt_dev, pt.data(), pt.size() * 4, cudaMemcpyHostToDevice));
         CORM_CUDA(cudaMemcpy(page_bits_ptr(c, layer), bits.data(), bits.size() * 4, cudaMemcpyHostToDevice));
+        const int32_t has_room = 1;
+        CORM_CUDA(cudaMemcpy(page_room_ptr(c, layer) + u, &has_room, 4, cudaMemcpyHostToDevice));
         const size_t page_bytes = (size_t)kPageKeys * D * c->e;
         for (size_t i = 0; i * kPageKeys < n; ++i) {
             const size_t bytes = std::min(page_bytes, n * D * c->e - i * page_bytes), at = (size_t)(pt[i] - 1) * page_bytes;

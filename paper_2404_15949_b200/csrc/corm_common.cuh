@@ -75,6 +75,7 @@ struct DecodeParams {
     // paged caches only (page_table == nullptr: every unit owns a slab of C rows of K and V)
     int32_t* page_table;      // [U][pt_stride] page number + 1 of each 32-key page of a unit, 0 = none
     uint32_t* page_bits;      // [pool_pages / 32] bit set = page in use
+    int32_t* page_room;       // [U] 1 iff the unit owns the page its next append goes to (0: pool exhausted)
     int32_t pool_pages, pt_stride;
 };
 
@@ -97,6 +98,7 @@ struct PromptParams {
     double bound_scale;       // multiplies the proven fp32 error bound of the tiled pass (1; tests raise it)
     int32_t* page_table;      // paged caches only, as in DecodeParams
     uint32_t* page_bits;
+    int32_t* page_room;
     int32_t pool_pages, pt_stride;
 };
 
@@ -186,8 +188,9 @@ __device__ __forceinline__ bool register_needed(uint32_t reg, int w, int t) {
 // per-unit arrays of C entries (8 bytes per key against 2 * D * e). Invariant between steps: a unit of n live keys
 // owns the pages of slots 0 .. n, i.e. n / 32 + 1 pages, so the next append always has a row to go to; the block
 // that finishes a unit's step (or its prompt pass) claims or releases pages to restore it. A unit whose claim failed
-// because the pool is exhausted has no page for its next append: that step reports CORM_ERR_CAPACITY and leaves
-// the unit untouched, like a full slab.
+// because the pool is exhausted has no page for its next append: its page_room flag is cleared, and the next step
+// (which reads the flag next to the live length, not behind it) reports CORM_ERR_CAPACITY and leaves the unit
+// untouched, like a full slab.
 constexpr int kPageKeys = 32;
 
 // row of slot `slot` in the layer's K / V storage: through the unit's page table, or inside its slab
@@ -195,12 +198,14 @@ __device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, 
     return pt_u ? (size_t)(__ldcg(pt_u + (slot >> 5)) - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
 }
 
-// Claims one free page: scans the in-use bitmap from a start word spread by `seed`, sets a clear bit with atomicOr
-// and owns the page iff the bit was clear before. Bounded: every word is visited once and the inner loop ends after
-// at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1 when the pool is exhausted.
-__device__ inline int claim_page(uint32_t* bits, int pool_pages, unsigned seed) {
+// Claims one free page for page-table entry `index` of unit u: scans the in-use bitmap from a start word that is
+// spread over the pool by the unit and advances with index / 32 (so a unit's pages tend to be neighbours), sets a
+// clear bit with atomicOr and owns the page iff the bit was clear before. Bounded: every word is visited once and
+// the inner loop ends after at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1
+// when the pool is exhausted.
+__device__ inline int claim_page(uint32_t* bits, int pool_pages, int u, int index) {
     const int n_words = pool_pages >> 5;
-    int i = (int)((seed * 2654435761u) % (unsigned)n_words);
+    int i = (int)(((unsigned)u * 2654435761u + (unsigned)(index >> 5)) % (unsigned)n_words);
     for (int tries = 0; tries < n_words; ++tries) {
         uint32_t w = __ldcg(bits + i);
         while (w != 0xffffffffu) {
@@ -218,8 +223,8 @@ __device__ inline int claim_page(uint32_t* bits, int pool_pages, unsigned seed) 
 // owned) to new_len. Called by every thread of the block that finished the unit, after its row moves: the barrier
 // below orders the block's reads of rows in released pages before another unit can claim them.
 template <int NT>
-__device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page_bits, int pool_pages, int pt_stride,
-                                             int u, int l_old, int new_len) {
+__device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
+                                             int pt_stride, int u, int l_old, int new_len) {
     if (!page_table) return;
     __syncthreads();
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
@@ -229,25 +234,30 @@ __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page
         pt_u[i] = 0;
         if (pg >= 0) atomicAnd(page_bits + (pg >> 5), ~(1u << (pg & 31)));
     }
-    if (need > have && have < pt_stride && threadIdx.x == 0)      // the next append starts a new page
-        pt_u[have] = claim_page(page_bits, pool_pages, (unsigned)u * 977u + (unsigned)have) + 1;   // 0 if exhausted
+    if (need > have && have < pt_stride && threadIdx.x == 0) {    // the next append starts a new page
+        const int pg = claim_page(page_bits, pool_pages, u, have);
+        pt_u[have] = pg + 1;
+        if (pg < 0) page_room[u] = 0;                             // exhausted: the unit's next step reports it
+    }
 }
 
 // Prompt pass: unit u ends with `kept` live keys and owns no page yet (the pass starts from an empty pool). Claims
 // kept / 32 + 1 pages, one per thread. Returns false (to every thread) if the pool ran out.
 template <int NT>
-__device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* page_bits, int pool_pages, int pt_stride,
-                                                 int u, int kept) {
+__device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
+                                                 int pt_stride, int u, int kept) {
     if (!page_table) return true;
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
     const int need = min(kept / kPageKeys + 1, pt_stride);
     int failed = 0;
     for (int i = (int)threadIdx.x; i < need; i += NT) {
-        const int pg = claim_page(page_bits, pool_pages, (unsigned)u * 977u + (unsigned)i);
+        const int pg = claim_page(page_bits, pool_pages, u, i);
         pt_u[i] = pg + 1;
         failed |= (pg < 0);
     }
-    return !__syncthreads_or(failed);      // also makes the table entries visible to the whole block
+    const bool ok = !__syncthreads_or(failed);      // also makes the table entries visible to the whole block
+    if (threadIdx.x == 0) page_room[u] = ok ? 1 : 0;
+    return ok;
 }
 
 // Exclusive prefix sums of popc(mask[i]) into prefix[0..nwords], block-wide. scratch holds NT ints.
@@ -291,9 +301,10 @@ __device__ __forceinline__ int kept_before(const uint32_t* mask, const int* pref
 // block. Sources lie at or above the new length, destinations below it, so copies never overlap. Each warp takes
 // four rows at a time and issues all their loads before the first store (the copies are latency-, not
 // bandwidth-limited). Rows are D*sizeof(T) bytes = a multiple of 16.
-template <typename T, int D, int NT>
-__device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, const int32_t* pt_u, size_t slab_row0, uint32_t* wordu,
-                                                int32_t* posu, const int* movers, const int* holes, int n_moved) {
+// row_of(slot) gives the slot's row in the layer's K / V storage (Kl, Vl).
+template <typename T, int D, int NT, typename RowOf>
+__device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, RowOf row_of, uint32_t* wordu, int32_t* posu,
+                                                const int* movers, const int* holes, int n_moved) {
     constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = 4, NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i0 = warp * kRows; i0 < n_moved; i0 += NW * kRows) {
@@ -307,8 +318,8 @@ __device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, const int32_t* pt_
             const bool on = i0 + r < n_moved;
             src[r] = on ? movers[i0 + r] : -1;
             dst[r] = on ? holes[i0 + r] : -1;
-            srow[r] = on ? kv_row(pt_u, slab_row0, src[r]) : 0;
-            drow[r] = on ? kv_row(pt_u, slab_row0, dst[r]) : 0;
+            srow[r] = on ? row_of(src[r]) : 0;
+            drow[r] = on ? row_of(dst[r]) : 0;
         }
 #pragma unroll
         for (int r = 0; r < kRows; ++r) {
@@ -450,11 +461,12 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V), pt_u, (size_t)u * p.C, wordu, posu,
-                                      movers, holes, n_moved);
+            const size_t slab_row0 = (size_t)u * p.C;
+            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
+                                      [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l - 1, new_len);
+    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);

@@ -38,8 +38,8 @@ __host__ __device__ constexpr int fast_k_stages(int G) { return G == 1 ? 1 : 2; 
 __host__ __device__ constexpr int fast_stages(int G) { return fast_k_stages(G) + kVStages; }
 __host__ __device__ constexpr int fast_warp_bytes(int G) { return fast_stages(G) * kTileBytes; }
 __host__ __device__ constexpr int fast_blocks_per_sm(int G) { return G == 1 ? CORM_FAST_BLOCKS_G1 : 2; }
-// 228 KB per SM, minus 1 KB the system reserves per block and ~1.2 KB of static shared memory
-__host__ __device__ constexpr int fast_smem_budget(int G) { return (228 * 1024) / fast_blocks_per_sm(G) - 2304; }
+// 228 KB per SM, minus 1 KB the system reserves per block and ~1.7 KB of static shared memory
+__host__ __device__ constexpr int fast_smem_budget(int G) { return (228 * 1024) / fast_blocks_per_sm(G) - 2816; }
 constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits (about 2 s)
 // longest unit that may finish inside one block (bounded by the registers that carry its verdict words)
 __host__ __device__ constexpr int fast_max_single_cap(int G) { return (G == 1 ? 8 : 2) * kFastThreads; }
@@ -200,16 +200,18 @@ __device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double
 // Single-split finalize: logits, registers and positions of the whole unit are in shared memory.
 // lists: scratch for the keep mask, its prefix sums and the hole / mover lists (ints).
 // wv / pv: registers and positions of slots tid, tid + NT, ... (loaded by the caller at block start).
+// tile_pages: paged caches, page + 1 of tile T of the unit at [T % kFastWarps][T / kFastWarps] (shared memory).
 template <int G, int NT, int KPRE>
 __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int t, const double* thr,
                                 const double* stash_sm, int stash_ld, const uint32_t (&wv)[KPRE],
-                                const int32_t (&pv)[KPRE], unsigned char* lists, int* holes, int* movers) {
+                                const int32_t (&pv)[KPRE], unsigned char* lists, int* holes, int* movers,
+                                const int32_t (*tile_pages)[32]) {
     __shared__ int s_scan1[NT];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cap_words = (l + 31) / 32 + 2;
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(lists);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
-    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    const bool paged = p.page_table != nullptr;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
@@ -249,11 +251,18 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
                 if (j >= new_len && kept) movers[kb - kept_below] = j;
             }
             __syncthreads();
-            block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), pt_u,
-                                             (size_t)u * p.C, wordu, posu, movers, holes, n_moved);
+            const size_t slab_row0 = (size_t)u * p.C;
+            block_move_rows<bf16_t, 128, NT>(
+                reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
+                [&](int slot) -> size_t {      // the unit is one split: its pages are the ones the warps fetched for their tiles
+                    const int tile = slot >> 5;
+                    return paged ? (size_t)(tile_pages[tile % kFastWarps][tile / kFastWarps] - 1) * kPageKeys + (slot & 31)
+                                 : slab_row0 + (size_t)slot;
+                },
+                wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l - 1, new_len);
+    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);
@@ -274,10 +283,19 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     constexpr int kKStages = fast_k_stages(G), kStagesPerWarp = fast_stages(G);
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
-    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
-    // paged caches: the unit's page table; a unit without a page for the appended row (pool exhausted) is full
+    // Paged caches: the pages of this warp's tiles (tile it of warp w is tile w + it * NW of the split, lane it fetches
+    // its entry) and the unit's room flag are requested together with the live length, none behind another; a unit
+    // without a page for the appended row (pool exhausted) is treated like a full slab.
+    __shared__ int32_t s_pt[kFastWarps][32];
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) {
+    int32_t my_page = 0, room = 1;
+    if (pt_u) {
+        const int idx = split * (p.split_len >> 5) + warp + lane * kFastWarps;
+        if (idx < p.pt_stride) my_page = __ldcg(pt_u + idx);
+        room = __ldcg(p.page_room + u);
+    }
+    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    if (l > p.C || !room) {
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
@@ -303,18 +321,25 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
     // this warp's tiles: warp, warp + NW, ... (tile index inside the split)
     const int my_n = (n_tiles > warp) ? (n_tiles - warp + NW - 1) / NW : 0;
+    if (pt_u) { s_pt[warp][lane] = my_page; __syncwarp(); }
+    // first row of the warp's tile `it` in the layer's K / V storage
+    auto tile_row0 = [&](int it) -> size_t {
+        if (!pt_u) return slab_row0 + (size_t)(begin + (warp + it * NW) * kTileKeys);
+        const int pg = it < 32 ? s_pt[warp][it] : __ldcg(pt_u + (begin >> 5) + warp + it * NW);
+        return (size_t)(pg - 1) * kPageKeys;
+    };
     auto tile_keys = [&](int it) { return min(kTileKeys, end - (begin + (warp + it * NW) * kTileKeys)); };
     auto issue_k = [&](int it) {
         const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kKStages;
         const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
         mbar_expect_tx(my_bars + slot * 8, bytes);
-        bulk_load(smem_addr(my_tiles + slot * kTileBytes), Kl + kv_row(pt_u, slab_row0, k0) * kRowBytes, bytes, my_bars + slot * 8);
+        bulk_load(smem_addr(my_tiles + slot * kTileBytes), Kl + tile_row0(it) * kRowBytes, bytes, my_bars + slot * 8);
     };
     auto issue_v = [&](int it) {
         const int k0 = begin + (warp + it * NW) * kTileKeys, slot = it % kVStages;
         const uint32_t bytes = (uint32_t)tile_keys(it) * kRowBytes;
         mbar_expect_tx(my_bars + (kKStages + slot) * 8, bytes);
-        bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vl + kv_row(pt_u, slab_row0, k0) * kRowBytes, bytes,
+        bulk_load(smem_addr(my_tiles + (kKStages + slot) * kTileBytes), Vl + tile_row0(it) * kRowBytes, bytes,
                   my_bars + (kKStages + slot) * 8);
     };
     // a warp's barriers and stages are its own: its first copies leave before the block meets at its first barrier
@@ -392,7 +417,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             if (lane < 16) {
                 const uint4 x = *reinterpret_cast<const uint4*>(newrow + lane * 16);
                 *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = x;
-                reinterpret_cast<uint4*>(Kl + kv_row(pt_u, slab_row0, l_old) * kRowBytes)[lane] = x;
+                reinterpret_cast<uint4*>(Kl + (tile_row0(it) + (size_t)(l_old - k0)) * kRowBytes)[lane] = x;
             }
             if (lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
             __syncwarp();
@@ -453,7 +478,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             if (lane < 16) {
                 const uint4 x = *reinterpret_cast<const uint4*>(newrow + kRowBytes + lane * 16);
                 *reinterpret_cast<uint4*>(vtile + (l_old - k0) * kRowBytes + lane * 16) = x;
-                reinterpret_cast<uint4*>(Vl + kv_row(pt_u, slab_row0, l_old) * kRowBytes)[lane] = x;
+                reinterpret_cast<uint4*>(Vl + (tile_row0(it) + (size_t)(l_old - k0)) * kRowBytes)[lane] = x;
             }
         }
         if (n_valid < kTileKeys)     // rows the copy did not fetch: make them harmless for 0 * v
@@ -544,7 +569,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         __syncthreads();
         unsigned char* lists = merge + NW * G * kRec;
         int* holes = reinterpret_cast<int*>(lists + 2 * ((l + 31) / 32 + 2) * 4);
-        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l);
+        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l, s_pt);
         return;
     }
     // A unit of several splits: its partial records and logits are complete once every split is done. With many

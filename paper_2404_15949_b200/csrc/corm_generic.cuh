@@ -25,9 +25,10 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     constexpr int NT = kGenericThreads, NW = NT / 32, NPL = D / 32;
     const int u = blockIdx.y, split = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
-    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) {   // the slab is full (paged: no page for the new row): report, leave the unit untouched
+    const int room = pt_u ? __ldcg(p.page_room + u) : 1;
+    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    if (l > p.C || !room) {   // the slab is full (paged: no page for the new row): report, leave the unit untouched
         if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
@@ -167,8 +168,11 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     if (P == 0) {
         if (tid == 0) {
             p.live_out[u] = 0;
-            if (p.page_table)    // an empty unit still owns the page its first append goes to
-                p.page_table[(size_t)u * p.pt_stride] = claim_page(p.page_bits, p.pool_pages, (unsigned)u * 977u) + 1;
+            if (p.page_table) {  // an empty unit still owns the page its first append goes to
+                const int pg = claim_page(p.page_bits, p.pool_pages, u, 0);
+                p.page_table[(size_t)u * p.pt_stride] = pg + 1;
+                p.page_room[u] = pg >= 0;
+            }
         }
         return;
     }
@@ -263,7 +267,7 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
     const int kept_total = prefix[nwords];
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, kept_total)) {
+    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, kept_total)) {
         if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }   // the pool is too small
         return;
     }

@@ -39,9 +39,10 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     __shared__ int s_lists[2 * kListCap];
     const int u = blockIdx.y, chunk = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = u / p.Hkv;
-    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (l > p.C || (pt_u && __ldcg(pt_u + (l_old >> 5)) <= 0)) return;     // reported by the streaming kernel
+    const int room = pt_u ? __ldcg(p.page_room + u) : 1;                   // paged caches: a page for the appended row
+    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    if (l > p.C || !room) return;                                          // reported by the streaming kernel
     const int n_act = (l + p.split_len - 1) / p.split_len;
     if (n_act == 1 && l <= p.single_cap) return;                           // finished inside the streaming kernel
     const int n_chunks = (l + kVerdictChunk - 1) / kVerdictChunk;
@@ -200,11 +201,12 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
                 }
             }
             __syncthreads();
-            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V), pt_u, (size_t)u * p.C, wordu, posu,
-                                      movers, holes, n_moved);
+            const size_t slab_row0 = (size_t)u * p.C;
+            block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
+                                      [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.pool_pages, p.pt_stride, u, l_old, new_len);
+    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, l_old, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);
