@@ -198,14 +198,22 @@ __device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, 
     return pt_u ? (size_t)(__ldcg(pt_u + (slot >> 5)) - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
 }
 
-// Claims one free page for page-table entry `index` of unit u: scans the in-use bitmap from a start word that is
-// spread over the pool by the unit and advances with index / 32 (so a unit's pages tend to be neighbours), sets a
-// clear bit with atomicOr and owns the page iff the bit was clear before. Bounded: every word is visited once and
-// the inner loop ends after at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1
-// when the pool is exhausted.
-__device__ inline int claim_page(uint32_t* bits, int pool_pages, int u, int index) {
+// Claims one free page for page-table entry `index` of unit u (of n_units). Every unit has a home region of the
+// pool, pool_pages / n_units pages starting at its share of the bitmap, and entry `index` first tries the page
+// `index` places into that region: while units stay inside their regions their pages are contiguous and in slot
+// order, so the streaming kernel reads them like a slab (neighbouring tiles share DRAM rows). If that page is taken
+// the bitmap is scanned from there on, wrapping around. A page is claimed by setting its bit with atomicOr and
+// belongs to the caller iff the bit was clear before. Bounded: every word is visited once and the inner loop ends
+// after at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1 when the pool is
+// exhausted.
+__device__ inline int claim_page(uint32_t* bits, int pool_pages, int n_units, int u, int index) {
     const int n_words = pool_pages >> 5;
-    int i = (int)(((unsigned)u * 2654435761u + (unsigned)(index >> 5)) % (unsigned)n_words);
+    const long long home = (long long)u * pool_pages / n_units + index;      // preferred page
+    int i = (int)((home >> 5) % n_words);
+    {
+        const uint32_t bit = 1u << (home & 31);
+        if (!(atomicOr(bits + i, bit) & bit)) return i * 32 + (int)(home & 31);
+    }
     for (int tries = 0; tries < n_words; ++tries) {
         uint32_t w = __ldcg(bits + i);
         while (w != 0xffffffffu) {
@@ -224,7 +232,7 @@ __device__ inline int claim_page(uint32_t* bits, int pool_pages, int u, int inde
 // below orders the block's reads of rows in released pages before another unit can claim them.
 template <int NT>
 __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
-                                             int pt_stride, int u, int l_old, int new_len) {
+                                             int pt_stride, int n_units, int u, int l_old, int new_len) {
     if (!page_table) return;
     __syncthreads();
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
@@ -235,7 +243,7 @@ __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page
         if (pg >= 0) atomicAnd(page_bits + (pg >> 5), ~(1u << (pg & 31)));
     }
     if (need > have && have < pt_stride && threadIdx.x == 0) {    // the next append starts a new page
-        const int pg = claim_page(page_bits, pool_pages, u, have);
+        const int pg = claim_page(page_bits, pool_pages, n_units, u, have);
         pt_u[have] = pg + 1;
         if (pg < 0) page_room[u] = 0;                             // exhausted: the unit's next step reports it
     }
@@ -245,13 +253,13 @@ __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page
 // kept / 32 + 1 pages, one per thread. Returns false (to every thread) if the pool ran out.
 template <int NT>
 __device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
-                                                 int pt_stride, int u, int kept) {
+                                                 int pt_stride, int n_units, int u, int kept) {
     if (!page_table) return true;
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
     const int need = min(kept / kPageKeys + 1, pt_stride);
     int failed = 0;
     for (int i = (int)threadIdx.x; i < need; i += NT) {
-        const int pg = claim_page(page_bits, pool_pages, u, i);
+        const int pg = claim_page(page_bits, pool_pages, n_units, u, i);
         pt_u[i] = pg + 1;
         failed |= (pg < 0);
     }
@@ -466,7 +474,7 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
                                       [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, l - 1, new_len);
+    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);

@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
         if (last_launch && split == 0 && tid == 0) {
             p.live_out[u] = 0; publish_live(p.maxlive, 0, 0);
             if (p.page_table) {  // an empty unit still owns the page its first append goes to
-                const int pg = claim_page(p.page_bits, p.pool_pages, u, 0);
+                const int pg = claim_page(p.page_bits, p.pool_pages, p.U, u, 0);
                 p.page_table[(size_t)u * p.pt_stride] = pg + 1;
                 p.page_room[u] = pg >= 0;
             }
@@ -374,7 +374,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
     const int kept_total = prefix[nwords];
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, kept_total)) {
+    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, kept_total)) {
         if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); }
         return;                                                                       // the pool is too small
     }

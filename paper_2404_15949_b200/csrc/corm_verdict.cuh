@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
                                       [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, u, l_old, new_len);
+    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l_old, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);

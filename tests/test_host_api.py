@@ -66,6 +66,26 @@ def test_create_rejects_before_any_cuda_call(lib):
     assert lib.corm_cache_destroy(None) == 1 and lib.corm_cache_kernel_launches(None) == 0
 
 
+def test_paged_arena_holds_the_pool_not_the_slabs(lib):
+    # The paper's headline is up to 70 % of the KV cache saved: a pool sized for 30 % of the slabs' rows must need
+    # about 30 % of the memory (page tables, bitmap, registers, positions and scratch on top).
+    cfg = _cfg(n_layers=4, batch=8, n_q_heads=32, n_kv_heads=32, max_tokens=4096)
+    slab = binding.corm_cache_arena_bytes(cfg)
+    units, pages_per_slab = 8 * 32, 4096 // 32
+    pool = units * pages_per_slab * 3 // 10 // 32 * 32
+    paged = lib.corm_cache_arena_bytes_paged(ctypes.byref(cfg), pool)
+    kv_pool = 4 * pool * 32 * 128 * 2 * 2
+    assert kv_pool < paged < kv_pool + 0.07 * slab and paged < 0.37 * slab
+    assert lib.corm_cache_arena_bytes_paged(ctypes.byref(cfg), 0) == slab            # 0 pages = slabs
+    for bad in (units - 32, units + 1, -32):                                         # too few pages / not a multiple of 32
+        assert lib.corm_cache_arena_bytes_paged(ctypes.byref(cfg), bad) == 0
+    handle = ctypes.c_void_p()
+    fake = ctypes.c_void_p(0x10000)
+    assert lib.corm_cache_create_paged(ctypes.byref(cfg), units + 1, fake, 1 << 40, ctypes.byref(handle)) == 1
+    assert lib.corm_cache_create_paged(ctypes.byref(cfg), pool, fake, paged - 1, ctypes.byref(handle)) == 3
+    assert handle.value is None
+
+
 def test_binding_fails_loudly_without_library(monkeypatch):
     monkeypatch.setattr(binding, "_lib", None)
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libcorm.so")
