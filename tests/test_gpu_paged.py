@@ -110,6 +110,65 @@ def test_paged_lockstep_from_imported_state():
         assert_states_equal(gpu, orc, 0, 1, 2, f"step {s}")
 
 
+@pytest.mark.parametrize("case", [
+    ("bf16", 128, 4, 2, 2, (400, 900), 40, 48, 32, 128, True, 2.0, 4242, 128),   # stamps, three prompt launch pairs
+    ("f32", 64, 2, 2, 2, (150, 260), 40, 100, 10, 64, False, 1.5, 4242, 64),     # generic kernels, chunked prompt rows
+], ids=lambda c: "-".join(str(x) for x in c))
+def test_paged_cache_with_windows_beyond_32_queries(case):
+    from parity_util import run_free
+    dtype, d, G, nkv, B, (pmin, pmax), steps, w, r, split_len, fast, alpha, seed, pool = case
+    cfg = CONFIGS[1].with_(name="wide", batch=B, n_q_heads=nkv * G, n_kv_heads=nkv, head_dim=d, dtype=dtype,
+                           prompt_min=pmin, prompt_max=pmax, steps=steps, window_w=w, recent_r=r, alpha=alpha,
+                           gqa_rho=0.7 if G > 1 else 0.0, hh_min=2, hh_max=6, seed=seed)
+    data = generate(cfg)
+    nb, nh = len(data.seqs), len(data.kv_heads)
+    gpu, orc = make_gpu_cache(cfg, nb, nh, pool_pages=pool), make_oracle(cfg, nb, nh)
+    gpu.corm_cache_set_tuning(split_len, fast)
+    run_free(cfg, data, gpu, orc, check_every=5)
+    assert orc.counters()["near_threshold"] == 0 and gpu.corm_cache_stats()["evicted_keys"] > 0
+    assert gpu.corm_cache_pool_usage(0)[0] == _pages_expected(orc.live_lens(0))
+
+
+def test_paged_cache_through_the_host_buffer_and_static_scratch_entry_points():
+    """The other two decode entry points on a paged cache: pinned host buffers read in place, and the step whose
+    scratch lives inside the library. Each must leave the state the plain call leaves on a slab cache."""
+    import torch
+    cfg = CONFIGS[4].with_(batch=2, n_q_heads=8, n_kv_heads=2, prompt_min=500, prompt_max=700, steps=10,
+                           recent_r=64, seed=4242)
+    data = generate(cfg)
+    nb, nh = len(data.seqs), len(data.kv_heads)
+    dt = cfg.dtype
+    ref = make_gpu_cache(cfg, nb, nh)
+    hst, sta = make_gpu_cache(cfg, nb, nh, pool_pages=128), make_gpu_cache(cfg, nb, nh, pool_pages=128)
+    for g in (ref, hst, sta):
+        g.corm_compress_prompt(0, to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt),
+                               data.prompt_lens)
+    pin = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).pin_memory()
+    for s in range(cfg.steps):
+        q, k, v = to_dev(data.q[s], dt), to_dev(data.k_new[s], dt), to_dev(data.v_new[s], dt)
+        a = ref.corm_decode_step(0, q, k, v)
+        out_h = pin(np.zeros(tuple(a.shape), dtype=np.float32))
+        hst.corm_decode_step_host(0, pin(data.q[s]), pin(data.k_new[s]), pin(data.v_new[s]), out_h)
+        out_s = torch.empty_like(q)
+        sta.corm_decode_step_static(0, q, k, v, out_s)
+        torch.cuda.synchronize()
+        assert torch.equal(a.cpu(), out_h)
+        assert float((a.float() - out_s.float()).abs().max()) <= OUT_TOL[dt]
+    for b in range(nb):
+        for h in range(nh):
+            x = ref.corm_cache_export_state(0, b, h)
+            n = x["live_len"]
+            y = hst.corm_cache_export_state(0, b, h)
+            assert y["live_len"] == n and all(np.array_equal(x[key][:n], y[key][:n]) for key in ("k", "v", "word", "pos"))
+            z = sta.corm_cache_export_state(0, b, h)      # the generic kernel may order slots differently: compare by position
+            assert z["live_len"] == n
+            ox, oz = np.argsort(x["pos"][:n]), np.argsort(z["pos"][:n])
+            assert all(np.array_equal(x[key][:n][ox], z[key][:n][oz]) for key in ("k", "v", "word", "pos"))
+    for g in (hst, sta):
+        assert g.corm_cache_stats()["device_status"] == 0
+        assert g.corm_cache_pool_usage(0)[0] == _pages_expected(g.corm_cache_live_lens(0))
+
+
 def test_exhausted_pool_is_reported_not_fatal():
     """alpha = 0 evicts nothing. Sixteen units of 60 keys hold two pages each, which is the whole 32-page pool. Slots
     60..63 still fit the second page; the append to slot 64 needs a third page, finds none, the status word says so
