@@ -250,10 +250,11 @@ __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page
 }
 
 // Prompt pass: unit u ends with `kept` live keys and owns no page yet (the pass starts from an empty pool). Claims
-// kept / 32 + 1 pages, one per thread. Returns false (to every thread) if the pool ran out.
+// kept / 32 + 1 pages, one per thread. Returns false (to every thread) if the pool ran out. pt_copy, if given, is
+// a shared-memory copy of the unit's new table entries for the gather that follows.
 template <int NT>
 __device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
-                                                 int pt_stride, int n_units, int u, int kept) {
+                                                 int pt_stride, int n_units, int u, int kept, int32_t* pt_copy = nullptr) {
     if (!page_table) return true;
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
     const int need = min(kept / kPageKeys + 1, pt_stride);
@@ -261,6 +262,7 @@ __device__ __forceinline__ bool claim_unit_pages(int32_t* page_table, uint32_t* 
     for (int i = (int)threadIdx.x; i < need; i += NT) {
         const int pg = claim_page(page_bits, pool_pages, n_units, u, i);
         pt_u[i] = pg + 1;
+        if (pt_copy) pt_copy[i] = pg + 1;
         failed |= (pg < 0);
     }
     const bool ok = !__syncthreads_or(failed);      // also makes the table entries visible to the whole block

@@ -662,7 +662,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     *n_launched = 1;
     if (all_single || p.inline_finalize) return CORM_OK;
     // verdict launch for the units that do not
-    const size_t vsmem = verdict_smem(p.C, n_splits, G);
+    const size_t vsmem = verdict_smem(p.C, n_splits, G, p.page_table != nullptr);
     auto launch_v = [&](auto kern) -> corm_status_t {
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), vsmem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }

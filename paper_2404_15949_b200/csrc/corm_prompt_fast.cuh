@@ -29,9 +29,9 @@ struct PromptFastParams {
     int32_t rows;                 // (slot1 - slot0) * G
 };
 
-__host__ __device__ inline size_t prompt_fast_smem(int rows, int C) {
+__host__ __device__ inline size_t prompt_fast_smem(int rows, int C, bool paged) {
     size_t a = (size_t)rows * 256 + (size_t)kPromptFastWarps * rows * 16 + (size_t)rows * 16;  // q rows (bf16), per-warp (m, Z), thresholds + error factors
-    size_t b = (size_t)2 * ((C + 31) / 32 + 2) * 4;                                            // keep mask + prefix (last arriver)
+    size_t b = (size_t)(paged ? 3 : 2) * ((C + 31) / 32 + 2) * 4;                              // keep mask + prefix (+ page entries) of the last arriver
     return a + b + 256;
 }
 
@@ -289,6 +289,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     double* err_sm = thr_sm + rows_pad;                          // kDotErr |q_r| / sqrt(d): times |k_j| it bounds a logit's error
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(err_sm + rows_pad);
     int* prefix = reinterpret_cast<int*>(keepmask + (p.C + 31) / 32 + 2);
+    int32_t* pt_sm = prefix + (p.C + 31) / 32 + 2;               // paged caches: the unit's page entries for the gather
     stage_q_rows(p, u, G, slot0, rows, rows_pad, q_sm);
     const double* thr = reinterpret_cast<const double*>(fp.partials) + (size_t)p.U * fp.n_splits * rows_pad * 2 + (size_t)u * rows_pad;
     for (int r = tid; r < rows_pad; r += NT) thr_sm[r] = __ldcg(thr + r);
@@ -373,8 +374,8 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     const int nwords = (P + 31) / 32;
     block_popc_scan<NT>(keepmask, prefix, nwords, s_scan);
     const int kept_total = prefix[nwords];
-    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, kept_total)) {
+    const bool paged = p.page_table != nullptr;
+    if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, kept_total, pt_sm)) {
         if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); }
         return;                                                                       // the pool is too small
     }
@@ -392,7 +393,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
             const int j = j0 + x;
             const bool kept = j < P && ((keepmask[j >> 5] >> (j & 31)) & 1u);
             dst[x] = kept ? kept_before(keepmask, prefix, j) : -1;
-            drow[x] = kept ? kv_row(pt_u, (size_t)u * p.C, dst[x]) : 0;
+            drow[x] = !kept ? 0 : paged ? (size_t)(pt_sm[dst[x] >> 5] - 1) * kPageKeys + (dst[x] & 31) : (size_t)u * p.C + dst[x];
             if (kept) buf[x] = __ldg(reinterpret_cast<const uint4*>((lane < 16 ? Kp : Vp) + (size_t)j * kRowBytes) + (lane & 15));
         }
 #pragma unroll
@@ -425,7 +426,7 @@ inline corm_status_t launch_prompt_fast(PromptFastParams& fp, int G, int max_p, 
     fp.split_len = split_len;
     fp.n_splits = max_p > 0 ? (max_p + split_len - 1) / split_len : 1;
     const size_t need = ((size_t)p.U * fp.n_splits * rows_pad * 2 + (size_t)p.U * rows_pad) * 8;
-    const size_t smem = prompt_fast_smem(rows_pad, p.C);
+    const size_t smem = prompt_fast_smem(rows_pad, p.C, p.page_table != nullptr);
     if (need > partial_capacity || smem > 200 * 1024 || p.U > 65535) return CORM_ERR_UNSUPPORTED;
     auto run = [&](auto k1, auto k2) -> corm_status_t {
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(k1), smem);

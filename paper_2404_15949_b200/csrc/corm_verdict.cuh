@@ -24,8 +24,8 @@ constexpr int kVerdictPer = kVerdictChunk / kVerdictThreads;
 
 __host__ __device__ inline int keepmask_words(int C) { return (C + 31) / 32 + 2; }
 
-__host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G) {
-    return (size_t)G * n_splits * (8 + 8 + 4) + 16 + (size_t)2 * keepmask_words(C) * 4;
+__host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G, bool paged) {
+    return (size_t)G * n_splits * (8 + 8 + 4) + 16 + (size_t)(paged ? 3 : 2) * keepmask_words(C) * 4;   // + keep mask, prefix sums (, page entries)
 }
 
 template <typename T, int D, int G>
@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     float* sm_sc = reinterpret_cast<float*>(sm_Z + (size_t)G * n_splits);
     uint32_t* keep_sm = reinterpret_cast<uint32_t*>(smem + (((size_t)G * n_splits * 20 + 15) & ~(size_t)15));
     int* prefix = reinterpret_cast<int*>(keep_sm + keepmask_words(p.C));
+    int32_t* pt_sm = prefix + keepmask_words(p.C);                         // paged caches: the unit's page entries (last block)
     const size_t pstride = partial_stride(D);
     const unsigned char* rec_u = p.partials + (size_t)u * p.max_splits * G * pstride;
 
@@ -167,7 +168,10 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     int new_len = l, n_moved = 0;
     if (evict_on) {
         const int nwords = (l + 31) / 32;
-        for (int i = tid; i < nwords; i += NT) keep_sm[i] = __ldcg(keep_g + i);
+        for (int i = tid; i < nwords; i += NT) {
+            keep_sm[i] = __ldcg(keep_g + i);
+            if (pt_u) pt_sm[i] = __ldcg(pt_u + i);                         // one entry per 32 slots, like the mask
+        }
         __syncthreads();
         block_popc_scan<NT>(keep_sm, prefix, nwords, s_scan);
         new_len = prefix[nwords];
@@ -203,7 +207,9 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
             __syncthreads();
             const size_t slab_row0 = (size_t)u * p.C;
             block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
-                                      [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
+                                      [&](int slot) -> size_t {
+                                          return pt_u ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
+                                      }, wordu, posu, movers, holes, n_moved);
         }
     }
     settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l_old, new_len);
