@@ -267,7 +267,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
         rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
             using T = std::remove_pointer_t<decltype(tp)>;
             constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
-            const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
+            const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens, c->pool_pages != 0);
             auto kern = decode_generic_kernel<T, DD, GG>;
             CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
             kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
@@ -604,7 +604,7 @@ corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void
     rc = dispatch(c, [&](auto* tp, auto dd, auto gg) -> corm_status_t {
         using T = std::remove_pointer_t<decltype(tp)>;
         constexpr int DD = decltype(dd)::value, GG = decltype(gg)::value;
-        const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens);
+        const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens, c->pool_pages != 0);
         auto kern = decode_generic_kernel<T, DD, GG>;
         CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
         kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);

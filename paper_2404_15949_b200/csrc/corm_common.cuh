@@ -234,9 +234,10 @@ template <int NT>
 __device__ __forceinline__ void settle_pages(int32_t* page_table, uint32_t* page_bits, int32_t* page_room, int pool_pages,
                                              int pt_stride, int n_units, int u, int l_old, int new_len) {
     if (!page_table) return;
+    const int have = l_old / kPageKeys + 1, need = new_len / kPageKeys + 1;
+    if (need == have) return;                                     // the usual step: nothing to claim or release (uniform)
     __syncthreads();
     int32_t* pt_u = page_table + (size_t)u * pt_stride;
-    const int have = l_old / kPageKeys + 1, need = new_len / kPageKeys + 1;
     for (int i = need + (int)threadIdx.x; i < have; i += NT) {
         const int pg = __ldcg(pt_u + i) - 1;
         pt_u[i] = 0;
@@ -363,7 +364,8 @@ __device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, RowOf row_of, uint
 //      form; GQA rule), shifted into the key's register
 //   3. once w rows exist: keep iff register != 0 or position > t - r; holes below the new length are filled with
 //      kept rows from above it (as many row copies as there are holes; sources and destinations are disjoint)
-// smem: 2*(ceil(C/32)+2) 32-bit words of dynamic shared memory.
+// smem: 2*(ceil(C/32)+2) 32-bit words of dynamic shared memory, 3*(ceil(C/32)+2) for a paged cache (the unit's page
+// entries are staged there for the row moves).
 template <typename T, int D, int G, int NT>
 __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_act, int t, unsigned char* smem) {
     __shared__ double s_thr[G];
@@ -373,6 +375,9 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(smem);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    int32_t* pt_sm = prefix + cap_words;
+    if (pt_u)
+        for (int i = tid; i < (l + 31) / 32; i += NT) pt_sm[i] = __ldcg(pt_u + i);   // visible after the barriers below
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     const size_t pstride = partial_stride(D);
@@ -473,7 +478,9 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
             __syncthreads();
             const size_t slab_row0 = (size_t)u * p.C;
             block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
-                                      [&](int slot) { return kv_row(pt_u, slab_row0, slot); }, wordu, posu, movers, holes, n_moved);
+                                      [&](int slot) -> size_t {
+                                          return pt_u ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
+                                      }, wordu, posu, movers, holes, n_moved);
         }
     }
     settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);

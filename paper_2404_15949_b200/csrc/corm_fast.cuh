@@ -201,7 +201,7 @@ __device__ __forceinline__ void qk_tile(const unsigned char* ktile, const double
 // lists: scratch for the keep mask, its prefix sums and the hole / mover lists (ints).
 // wv / pv: registers and positions of slots tid, tid + NT, ... (loaded by the caller at block start).
 // tile_pages: paged caches, page + 1 of tile T of the unit at [T % kFastWarps][T / kFastWarps] (shared memory).
-template <int G, int NT, int KPRE>
+template <int G, int NT, int KPRE, bool PAGED>
 __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int t, const double* thr,
                                 const double* stash_sm, int stash_ld, const uint32_t (&wv)[KPRE],
                                 const int32_t (&pv)[KPRE], unsigned char* lists, int* holes, int* movers,
@@ -211,7 +211,6 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     const int cap_words = (l + 31) / 32 + 2;
     uint32_t* keepmask = reinterpret_cast<uint32_t*>(lists);
     int* prefix = reinterpret_cast<int*>(keepmask + cap_words);
-    const bool paged = p.page_table != nullptr;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
@@ -256,13 +255,13 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
                 reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
                 [&](int slot) -> size_t {      // the unit is one split: its pages are the ones the warps fetched for their tiles
                     const int tile = slot >> 5;
-                    return paged ? (size_t)(tile_pages[tile % kFastWarps][tile / kFastWarps] - 1) * kPageKeys + (slot & 31)
+                    return PAGED ? (size_t)(tile_pages[tile % kFastWarps][tile / kFastWarps] - 1) * kPageKeys + (slot & 31)
                                  : slab_row0 + (size_t)slot;
                 },
                 wordu, posu, movers, holes, n_moved);
         }
     }
-    settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+    if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
     if (tid == 0) {
         p.live_out[u] = new_len;
         publish_live(p.maxlive, p.step + 1, new_len);
@@ -273,7 +272,9 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
     }
 }
 
-template <int G>
+// PAGED selects the cache layout at compile time (the launcher picks the instance from p.page_table), so that the
+// slab instance carries none of the paging code.
+template <int G, bool PAGED>
 __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fast_kernel(const __grid_constant__ DecodeParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ int s_failed;
@@ -287,9 +288,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     // its entry) and the unit's room flag are requested together with the live length, none behind another; a unit
     // without a page for the appended row (pool exhausted) is treated like a full slab.
     __shared__ int32_t s_pt[kFastWarps][32];
-    const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
     int32_t my_page = 0, room = 1;
-    if (pt_u) {
+    if (PAGED) {
         const int idx = split * (p.split_len >> 5) + warp + lane * kFastWarps;
         if (idx < p.pt_stride) my_page = __ldcg(pt_u + idx);
         room = __ldcg(p.page_room + u);
@@ -321,10 +322,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
     // this warp's tiles: warp, warp + NW, ... (tile index inside the split)
     const int my_n = (n_tiles > warp) ? (n_tiles - warp + NW - 1) / NW : 0;
-    if (pt_u) { s_pt[warp][lane] = my_page; __syncwarp(); }
+    if (PAGED) { s_pt[warp][lane] = my_page; __syncwarp(); }
     // first row of the warp's tile `it` in the layer's K / V storage
     auto tile_row0 = [&](int it) -> size_t {
-        if (!pt_u) return slab_row0 + (size_t)(begin + (warp + it * NW) * kTileKeys);
+        if (!PAGED) return slab_row0 + (size_t)(begin + (warp + it * NW) * kTileKeys);
         const int pg = it < 32 ? s_pt[warp][it] : __ldcg(pt_u + (begin >> 5) + warp + it * NW);
         return (size_t)(pg - 1) * kPageKeys;
     };
@@ -569,7 +570,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         __syncthreads();
         unsigned char* lists = merge + NW * G * kRec;
         int* holes = reinterpret_cast<int*>(lists + 2 * ((l + 31) / 32 + 2) * 4);
-        finalize_single<G, NT, kPre>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l, s_pt);
+        finalize_single<G, NT, kPre, PAGED>(p, u, b, l, t, s_thr1, stash_sm, p.single_cap, wv, pv, lists, holes, holes + l, s_pt);
         return;
     }
     // A unit of several splits: its partial records and logits are complete once every split is done. With many
@@ -640,7 +641,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     const size_t smem = (size_t)lay.total;
     const bool all_single = n_splits == 1 && upper <= p.single_cap;      // every unit finishes inside its one block
     // who finishes the longer units: see the end of decode_fast_kernel
-    const size_t fin = (size_t)2 * ((p.C + 31) / 32 + 2) * 4;            // keep mask + prefix sums of finalize_unit
+    const size_t fin = (size_t)(p.page_table ? 3 : 2) * ((p.C + 31) / 32 + 2) * 4;   // keep mask + prefix sums (+ page entries) of finalize_unit
     // ... or when units are so short that the serial walk (upper x G logits over 128 threads) is cheaper than a launch
     const bool many = finish_mode == 2 || (finish_mode != 3 && ((long long)p.U * n_splits >= 4ll * sms * fast_blocks_per_sm(G) ||
                                                                 (long long)upper * G <= 2048));
@@ -657,7 +658,9 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;
     };
-    corm_status_t rc = G == 1 ? launch(decode_fast_kernel<1>) : G == 2 ? launch(decode_fast_kernel<2>) : launch(decode_fast_kernel<4>);
+    corm_status_t rc;
+    if (p.page_table) rc = G == 1 ? launch(decode_fast_kernel<1, true>) : G == 2 ? launch(decode_fast_kernel<2, true>) : launch(decode_fast_kernel<4, true>);
+    else rc = G == 1 ? launch(decode_fast_kernel<1, false>) : G == 2 ? launch(decode_fast_kernel<2, false>) : launch(decode_fast_kernel<4, false>);
     if (rc != CORM_OK) return rc;
     *n_launched = 1;
     if (all_single || p.inline_finalize) return CORM_OK;

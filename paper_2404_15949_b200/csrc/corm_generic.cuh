@@ -10,10 +10,10 @@ namespace corm {
 constexpr int kGenericThreads = 128;
 constexpr int kPromptThreads = 256;
 
-__host__ __device__ inline size_t generic_decode_smem(int D, int G, int C) {
+__host__ __device__ inline size_t generic_decode_smem(int D, int G, int C, bool paged) {
     const size_t warps = kGenericThreads / 32;
     size_t a = (size_t)G * D * 8 + warps * G * 16 + warps * G * D * 4;
-    size_t b = (size_t)2 * ((C + 31) / 32 + 2) * 4;
+    size_t b = (size_t)(paged ? 3 : 2) * ((C + 31) / 32 + 2) * 4;
     return a > b ? a : b;
 }
 
