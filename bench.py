@@ -31,9 +31,9 @@ METRIC = "corm_decode_step_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the decode kernel, from the ncu capture summarised in
-# profiles/decode_fast_kernel_batch32_bf16.md (241.6 and 240.1 MB moved for 237.4 MB algorithmic at the two captured
+# profiles/decode_fast_kernel_batch32_bf16.md (243.0 and 240.3 MB moved for 237.4 MB algorithmic at the two captured
 # steps). Set to None whenever the kernel changes until the counters are taken again.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.015}
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.018}
 
 
 def log(*a):
