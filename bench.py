@@ -317,6 +317,11 @@ def main():
     if args.pool_pages:
         line["config"]["pool_pages"] = args.pool_pages
         line["pool_pages_in_use"] = sum(cache.corm_cache_pool_usage(l)[0] for l in range(L))
+        # the paper's own metric, made physical: K+V bytes of the pages held against K+V bytes of every token seen
+        row = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4)
+        line["kv_bytes_held"] = line["pool_pages_in_use"] * 32 * row
+        line["kv_bytes_full_cache"] = st3["appended_keys"] * row
+        line["kv_memory_reduction"] = 1.0 - line["kv_bytes_held"] / max(1, line["kv_bytes_full_cache"])
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"], _ = oracle_baseline(cfg, args.ref_seqs, args.ref_steps)
     print(json.dumps(line), flush=True)
