@@ -169,6 +169,37 @@ def test_paged_cache_through_the_host_buffer_and_static_scratch_entry_points():
         assert g.corm_cache_pool_usage(0)[0] == _pages_expected(g.corm_cache_live_lens(0))
 
 
+def test_paged_layers_have_pools_of_their_own():
+    """Three layers, each with its own pool, page tables and bitmap: stepping them in mixed order matches the oracle
+    layer by layer, and a prompt pass on one layer returns that layer's pages only."""
+    cfg = CONFIGS[2].with_(n_layers=3, n_q_heads=4, n_kv_heads=4, prompt_min=300, prompt_max=300, steps=40,
+                           recent_r=32, dense_layers=1)
+    gpu = make_gpu_cache(cfg, 1, 4, n_layers=3, pool_pages=64)
+    orc = make_oracle(cfg, 1, 4, n_layers=3)
+    datas = [generate(cfg, layer=l) for l in range(3)]
+    dt = cfg.dtype
+    for l in (2, 0, 1):
+        d = datas[l]
+        gpu.corm_compress_prompt(l, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+        orc.compress_prompt(l, d.k_prompt, d.v_prompt, d.q_last, d.prompt_lens)
+    for s in range(cfg.steps):
+        for l in (1, 2, 0):
+            d = datas[l]
+            a = gpu.corm_decode_step(l, to_dev(d.q[s], dt), to_dev(d.k_new[s], dt), to_dev(d.v_new[s], dt))
+            o = orc.decode_step(l, d.q[s], d.k_new[s], d.v_new[s])
+            assert np.abs(a.float().cpu().numpy() - o).max() <= OUT_TOL[dt]
+    for l in range(3):
+        assert_states_equal(gpu, orc, l, 1, 4, f"layer {l}")
+        assert gpu.corm_cache_pool_usage(l) == (_pages_expected(orc.live_lens(l)), 64)
+    before = [gpu.corm_cache_pool_usage(l)[0] for l in range(3)]
+    d = datas[1]
+    gpu.corm_compress_prompt(1, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+    after = [gpu.corm_cache_pool_usage(l)[0] for l in range(3)]
+    assert after[0] == before[0] and after[2] == before[2]
+    assert after[1] == _pages_expected(gpu.corm_cache_live_lens(1))
+    assert gpu.corm_cache_stats()["device_status"] == 0
+
+
 def test_exhausted_pool_is_reported_not_fatal():
     """alpha = 0 evicts nothing. Sixteen units of 60 keys hold two pages each, which is the whole 32-page pool. Slots
     60..63 still fit the second page; the append to slot 64 needs a third page, finds none, the status word says so
