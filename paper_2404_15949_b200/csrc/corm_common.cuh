@@ -201,8 +201,8 @@ __device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, 
 // Claims one free page for page-table entry `index` of unit u (of n_units). Every unit has a home region of the
 // pool, pool_pages / n_units pages starting at its share of the bitmap, and entry `index` first tries the page
 // `index` places into that region: while units stay inside their regions their pages are contiguous and in slot
-// order, so the streaming kernel reads them like a slab (neighbouring tiles share DRAM rows). If that page is taken
-// the bitmap is scanned from there on, wrapping around. A page is claimed by setting its bit with atomicOr and
+// order, as in a slab, and units do not contend for the same bitmap words. If that page is taken the bitmap is
+// scanned from there on, wrapping around. A page is claimed by setting its bit with atomicOr and
 // belongs to the caller iff the bit was clear before. Bounded: every word is visited once and the inner loop ends
 // after at most 32 rounds (each failed round adds a bit to w). Returns the page number or -1 when the pool is
 // exhausted.
