@@ -34,6 +34,8 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/decode_fast_kernel_batch32_bf16.md (243.0 and 240.3 MB moved for 237.4 MB algorithmic at the two captured
 # steps). Set to None whenever the kernel changes until the counters are taken again.
 DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.018}
+# the same for the kernel's paged instance (--pool-pages; 241.5 and 241.0 MB moved for 237.4 MB, same file)
+DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE_PAGED = {"batch32_bf16": 1.016}
 
 
 def log(*a):
@@ -299,7 +301,8 @@ def main():
         "config": workload_config(cfg, args),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src,
-                     "traffic": (DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE.get(cfg.name) or 0) * abytes / (args.steps * L) or None,
+                     "traffic": ((DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE_PAGED if args.pool_pages else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE)
+                                 .get(cfg.name) or 0) * abytes / (args.steps * L) or None,
                      "kernel": "decode_fast_kernel (one launch per layer per step; early steps with units longer than one block add a verdict launch, counted in the time)",
                      "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * ms / (args.steps * L)},
         "e2e": {"value": e2e_value, "unit": UNIT,
