@@ -9,7 +9,9 @@
  * it (Section 5, "Integrate into grouped-query attention").
  *
  * A "unit" is one (layer, sequence, kv head). Each unit owns a slab of max_tokens slots holding K rows, V rows,
- * one 32-bit verdict register per key and the key's absolute 1-based token position. Register encodings: for
+ * one 32-bit verdict register per key and the key's absolute 1-based token position (in a paged cache,
+ * corm_cache_create_paged, the K and V rows of a slot live in 32-key pages drawn from a pool the layer's units share;
+ * slots, their order and everything below are the same). Register encodings: for
  * window_w <= 32 a shift register (bit b = verdict of the query b steps ago); for 33..256 (the paper's experiments
  * use up to 256) the absolute step of the latest query that found the key important, 0 if none has, which decides
  * Algorithm 1's any() over the last w rows as step_now - register < w. Live entries occupy slots [0, live_len); their slot ORDER IS NOT the token order once decode
