@@ -89,6 +89,41 @@ def test_paged_cache_equals_slab_cache_bit_for_bit():
     assert paged.corm_cache_stats()["device_status"] == 0
 
 
+def test_tight_pool_under_churn_equals_slab_cache():
+    """256 units claim and release pages concurrently in a pool only a little larger than what they hold at the peak,
+    so home regions overflow into their neighbours' and claims fall back to scanning the bitmap. Outputs must still
+    equal the slab cache's bit for bit at every step, no page may be lost or held twice (pages in use = what the live
+    lengths require, every 8 steps), and the final states must be identical."""
+    cfg = CONFIGS[1].with_(name="churn", batch=8, n_q_heads=32, n_kv_heads=32, head_dim=128, dtype="bf16",
+                           prompt_min=200, prompt_max=700, steps=160, window_w=4, recent_r=16, hh_min=2, hh_max=6,
+                           seed=99)
+    data = generate(cfg)
+    nb, nh = len(data.seqs), len(data.kv_heads)
+    dt = cfg.dtype
+    slab = make_gpu_cache(cfg, nb, nh)
+    args = (to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt), data.prompt_lens)
+    slab.corm_compress_prompt(0, *args)
+    need = _pages_expected(slab.corm_cache_live_lens(0))            # the peak: lengths only shrink towards r + a few
+    pool = (need + 256 + 31) // 32 * 32                             # one spare page per unit
+    paged = make_gpu_cache(cfg, nb, nh, pool_pages=pool)
+    paged.corm_compress_prompt(0, *args)
+    assert paged.corm_cache_pool_usage(0) == (need, pool)
+    q, k, v = to_dev(data.q, dt), to_dev(data.k_new, dt), to_dev(data.v_new, dt)
+    for s in range(cfg.steps):
+        a, b = slab.corm_decode_step(0, q[s], k[s], v[s]), paged.corm_decode_step(0, q[s], k[s], v[s])
+        assert (a == b).all(), f"step {s}"
+        if s % 8 == 7:
+            live = paged.corm_cache_live_lens(0)
+            assert (live == slab.corm_cache_live_lens(0)).all()
+            assert paged.corm_cache_pool_usage(0)[0] == _pages_expected(live), f"step {s}"
+    assert paged.corm_cache_stats()["device_status"] == 0 and paged.corm_cache_stats()["evicted_keys"] > 0
+    for b in range(0, nb, 3):
+        for h in range(0, nh, 5):
+            x, y = slab.corm_cache_export_state(0, b, h), paged.corm_cache_export_state(0, b, h)
+            assert x["live_len"] == y["live_len"]
+            assert all(np.array_equal(x[key], y[key]) for key in ("k", "v", "word", "pos")), (b, h)
+
+
 def test_paged_lockstep_from_imported_state():
     """Import hook on a paged cache: the host hands the unit its pages; every step restarts from the oracle's state."""
     cfg = CONFIGS[1].with_(prompt_min=200, prompt_max=200, steps=12, dtype="bf16", n_q_heads=8, n_kv_heads=2,
