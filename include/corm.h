@@ -131,8 +131,8 @@ corm_status_t corm_compress_prompt(corm_cache_t* cache, int32_t layer, const voi
  *   q      device [batch, n_q_heads, head_dim]
  *   k_new  device [batch, n_kv_heads, head_dim], v_new likewise
  *   out    device [batch, n_q_heads, head_dim]
- * The call enqueues one or two launches and returns; it sizes them from the longest live length the kernels last
- * reported, which it reads back asynchronously every 8 steps. A host that has run 24 steps past a read-back that
+ * The call enqueues one or two launches and returns; it sizes them from the longest and the mean live length the
+ * kernels last reported, which it reads back asynchronously every 8 steps (batch * n_kv_heads integers). A host that has run 24 steps past a read-back that
  * has not landed waits for it here (the GPU still has those steps queued), so the call can block briefly, and a
  * layer's decode steps cannot be recorded into a CUDA graph.
  * Errors: STATE if the layer has had no corm_compress_prompt since create/reset; INVALID_ARG. */

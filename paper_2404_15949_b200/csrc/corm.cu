@@ -128,7 +128,9 @@ struct corm_cache {
     size_t e;
     std::vector<int> parity, steps, ready, live_upper;
     // sizing feedback: the kernels publish the longest live length, the host reads it back without ever waiting
-    unsigned long long* maxlive_host = nullptr;   // pinned, [n_layers]
+    unsigned long long* maxlive_host = nullptr;   // pinned, [n_layers] words followed by [n_layers][U] live lengths
+    int32_t* live_host = nullptr;                 // the second part of that buffer
+    std::vector<int> live_mean;                   // mean live length at the last read-back that landed (0 = unknown)
     std::vector<cudaEvent_t> readback_ev;
     std::vector<int> readback_pending, last_readback_step;
     int tune_split_len = 0, allow_fast = 1;
@@ -218,11 +220,16 @@ void poll_live_bound(corm_cache* c, int layer) {
     if (steps_done > c->steps[layer]) return;   // stale word from before a reset / new prompt
     const int bound = len + (c->steps[layer] - steps_done);
     if (bound < c->live_upper[layer]) c->live_upper[layer] = bound;
+    long long sum = 0;                            // the lengths themselves came with the same read-back
+    for (int u = 0; u < c->U; ++u) sum += c->live_host[(size_t)layer * c->U + u];
+    c->live_mean[layer] = (int)(sum / c->U);
 }
 
 void schedule_live_readback(corm_cache* c, int layer, cudaStream_t st) {
     if (c->readback_pending[layer] || !c->maxlive_host) return;
     if (cudaMemcpyAsync(c->maxlive_host + layer, maxlive_ptr(c, layer), 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return;
+    if (cudaMemcpyAsync(c->live_host + (size_t)layer * c->U, live_buf(c, layer, c->parity[layer]), (size_t)c->U * 4,
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess) return;
     if (cudaEventRecord(c->readback_ev[layer], st) != cudaSuccess) return;
     c->readback_pending[layer] = 1;
     c->last_readback_step[layer] = c->steps[layer];
@@ -260,7 +267,9 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     corm_status_t rc;
     int n_launched = 1;
     if (fast) {
-        rc = launch_decode_fast(p, c->G, upper, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
+        // the mean grows by at most one key per step, like the bound
+        const int typical = c->live_mean[layer] ? std::min(upper, c->live_mean[layer] + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
+        rc = launch_decode_fast(p, c->G, upper, typical, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
         const int n_splits = (upper + p.split_len - 1) / p.split_len;
@@ -344,12 +353,18 @@ corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pag
     c->steps.assign(cfg->n_layers, 0);
     c->ready.assign(cfg->n_layers, 0);
     c->live_upper.assign(cfg->n_layers, 0);
+    c->live_mean.assign(cfg->n_layers, 0);
     c->have_q_prev.assign(cfg->n_layers, 0);
     c->readback_pending.assign(cfg->n_layers, 0);
     c->last_readback_step.assign(cfg->n_layers, 0);
     c->readback_ev.assign(cfg->n_layers, nullptr);
-    bool host_ok = cudaHostAlloc(reinterpret_cast<void**>(&c->maxlive_host), sizeof(unsigned long long) * cfg->n_layers,
+    bool host_ok = cudaHostAlloc(reinterpret_cast<void**>(&c->maxlive_host),
+                                 sizeof(unsigned long long) * cfg->n_layers + sizeof(int32_t) * (size_t)cfg->n_layers * c->U,
                                  cudaHostAllocDefault) == cudaSuccess;   // pinned HOST memory; device memory stays the caller's
+    if (host_ok) {
+        c->live_host = reinterpret_cast<int32_t*>(c->maxlive_host + cfg->n_layers);
+        std::memset(c->maxlive_host, 0, sizeof(unsigned long long) * cfg->n_layers + sizeof(int32_t) * (size_t)cfg->n_layers * c->U);
+    }
     for (int l = 0; host_ok && l < cfg->n_layers; ++l)
         host_ok = cudaEventCreateWithFlags(&c->readback_ev[l], cudaEventDisableTiming) == cudaSuccess;
     if (!host_ok) {
@@ -392,7 +407,7 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
     CORM_CUDA(cudaMemsetAsync(c->arena + c->lay.bookkeeping_begin, 0, c->lay.bookkeeping_end - c->lay.bookkeeping_begin,
                               static_cast<cudaStream_t>(stream)));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
-        c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; c->have_q_prev[l] = 0;
+        c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; c->live_mean[l] = 0; c->have_q_prev[l] = 0;
         c->readback_pending[l] = 0; c->last_readback_step[l] = 0;
     }
     return CORM_OK;
@@ -474,7 +489,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     }
     if (rc != CORM_OK) return rc;
     c->launches += n_launched;
-    c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p;
+    c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p; c->live_mean[layer] = 0;
     c->have_q_prev[layer] = 0;                    // the previous decode query belonged to the old text
     c->last_readback_step[layer] = 0;
     schedule_live_readback(c, layer, st);
@@ -765,6 +780,7 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     c->ready[layer] = 1;
     c->readback_pending[layer] = 0;   // a read-back enqueued before this import knows nothing of it
     c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
+    c->live_mean[layer] = 0;                      // unknown until the next read-back
     return CORM_OK;
 }
 
