@@ -163,7 +163,7 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=512)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict"],
+    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced"],
                     help="who finishes units of several splits: the decode launch itself or the verdict launch")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -205,7 +205,7 @@ def main():
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
                       cfg.recent_r, cfg.alpha, cfg.dtype, local, pool_pages=args.pool_pages)
-    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3}[args.finish])
+    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4}[args.finish])
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
     prompt_ms = 0.0

@@ -46,7 +46,9 @@ typedef enum {
     CORM_ERR_STATE = 4,
     CORM_ERR_CUDA = 5,
     CORM_ERR_CAPACITY = 6,
-    CORM_ERR_TIMEOUT = 7
+    CORM_ERR_TIMEOUT = 7,
+    CORM_ERR_INTERNAL = 8    /* a kernel met an index outside its range (a broken page table, a misplaced buffer):
+                                the access was skipped; the cache must be reset */
 } corm_status_t;
 
 typedef enum { CORM_F32 = 0, CORM_BF16 = 1 } corm_dtype_t;

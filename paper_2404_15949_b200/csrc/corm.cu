@@ -15,6 +15,7 @@
 #include "../../include/corm.h"
 #include "corm_common.cuh"
 #include "corm_fast.cuh"
+#include "corm_balanced.cuh"
 #include "corm_generic.cuh"
 #include "corm_prompt_fast.cuh"
 
@@ -28,7 +29,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -53,6 +54,14 @@ bool config_ok(const corm_config_t* c, corm_status_t* why) {
 }
 
 int max_splits_of(const corm_config_t& c) { return (c.max_tokens + kMinSplit - 1) / kMinSplit; }
+
+// Split partial records the arena holds: one per (unit, split) of the block-per-split kernels, and enough for the
+// balanced kernel's one record per (block, unit) pair of its tile list at up to kMaxBalancedBlocks blocks.
+constexpr int kMaxBalancedBlocks = 1024;
+size_t partial_records_of(const corm_config_t& c) {
+    const size_t U = (size_t)c.batch * c.n_kv_heads;
+    return std::max(U * (size_t)max_splits_of(c), bal_record_count(kMaxBalancedBlocks, (int)U));
+}
 
 int pt_stride_of(const corm_config_t& c) { return (c.max_tokens + kPageKeys - 1) / kPageKeys; }
 
@@ -79,6 +88,7 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.base_tokens = take(Ltot * c.batch * 4);
     L.base_obs = take(Ltot * c.batch * 4);
     L.ticket = take(Ltot * U * 4);
+    L.ticket2 = take(Ltot * U * 4);
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
@@ -89,7 +99,7 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.bookkeeping_end = off;
     L.q_prev = take(Ltot * (size_t)c.batch * c.n_q_heads * D * e);
     L.stash = take(U * G * C * 8);
-    L.partials = take(U * (size_t)max_splits_of(c) * G * partial_stride((int)D));
+    L.partials = take(partial_records_of(c) * G * partial_stride((int)D));
     L.keepmask = take(U * (size_t)keepmask_words((int)C) * 4);
     L.stage_q = take((size_t)c.batch * c.n_q_heads * D * e);
     L.stage_k = take(U * D * e);
@@ -140,6 +150,7 @@ struct corm_cache {
     int sm_count = 148;
     long long launches = 0;
     int pool_pages = 0, pt_stride = 0;            // paged cache: pages per layer, page-table entries per unit
+    std::vector<CUtensorMap> vmaps;               // per layer: the V storage as a tiled tensor (balanced kernel); empty = unavailable
 };
 
 namespace {
@@ -251,6 +262,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.base_tokens = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_tokens, (size_t)cf.batch * 4, layer));
     p.base_obs = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer));
     p.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
+    p.ticket2 = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket2, U * 4, layer));
     p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
     p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
     p.maxlive = maxlive_ptr(c, layer);
@@ -266,7 +278,15 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
     int n_launched = 1;
-    if (fast) {
+    // Group sizes above one take the balanced kernel while no unit can be longer than kBalancedAutoLimit keys (its
+    // compaction is one block per unit, which long units with many evictions per step outgrow); tuning value 4
+    // forces it for every group size and length the kernel covers.
+    constexpr int kBalancedAutoLimit = 6144;
+    const bool balanced = fast && !c->vmaps.empty() &&
+                          (c->allow_fast == 4 || (c->allow_fast == 1 && c->G >= 2 && upper <= kBalancedAutoLimit));
+    if (balanced) {
+        rc = launch_decode_balanced(p, c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf), st, &n_launched);
+    } else if (fast) {
         // the mean grows by at most one key per step, like the bound
         const int typical = c->live_mean[layer] ? std::min(upper, c->live_mean[layer] + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
         rc = launch_decode_fast(p, c->G, upper, typical, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
@@ -376,6 +396,16 @@ corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pag
     }
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0) c->sm_count = sms;
+    if (cfg->kv_dtype == CORM_BF16 && cfg->head_dim == 128 && c->G <= 4 && cfg->max_tokens <= kBalMaxTokens) {
+        const unsigned long long rows = pool_pages ? (unsigned long long)pool_pages * kPageKeys
+                                                   : (unsigned long long)c->U * cfg->max_tokens;
+        c->vmaps.resize(cfg->n_layers);
+        for (int l = 0; l < cfg->n_layers; ++l)
+            if (make_v_tensor_map(&c->vmaps[l], layer_ptr(c, lay.V, kv_layer_bytes(c), l), rows) != CORM_OK) {
+                c->vmaps.clear();                 // the block-per-split kernels serve the cache instead
+                break;
+            }
+    }
     cudaError_t e = cudaMemset(c->arena + lay.bookkeeping_begin, 0, lay.bookkeeping_end - lay.bookkeeping_begin);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -439,6 +469,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     CORM_CUDA(cudaMemcpyAsync(base_tokens, prompt_lens_host, (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemcpyAsync(base_obs, obs.data(), (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket, U * 4, layer), 0, U * 4, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket2, U * 4, layer), 0, U * 4, st));
     CORM_CUDA(cudaMemsetAsync(maxlive_ptr(c, layer), 0, 8, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer), 0, CNT_COUNT * 8, st));   // a new prompt restarts the layer's statistics
     c->readback_pending[layer] = 0;   // an older read-back no longer describes this layer
@@ -802,7 +833,7 @@ corm_status_t corm_cache_pool_usage(corm_cache_t* c, int32_t layer, int64_t* pag
 corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
-    if (allow_fast_path < 0 || allow_fast_path > 3) return CORM_ERR_INVALID_ARG;
+    if (allow_fast_path < 0 || allow_fast_path > 4) return CORM_ERR_INVALID_ARG;
     c->allow_fast = allow_fast_path;
     return CORM_OK;
 }
@@ -847,6 +878,7 @@ const char* corm_status_string(corm_status_t s) {
         case CORM_ERR_CUDA: return "CUDA runtime error";
         case CORM_ERR_CAPACITY: return "slab capacity exceeded";
         case CORM_ERR_TIMEOUT: return "bounded wait expired";
+        case CORM_ERR_INTERNAL: return "internal invariant broken (index outside its range)";
     }
     return "unknown status";
 }

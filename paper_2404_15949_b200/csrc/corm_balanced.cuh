@@ -1,0 +1,880 @@
+// Decode kernel for bf16 caches with head_dim 128 and grouped query heads (group size 1, 2 or 4): one launch per
+// step, every block the same share of the work.
+//
+// The step's work is the list of 32-key tiles of all units (a unit of l live keys has ceil(l / 32)). Every block
+// computes that list's prefix sums from the live lengths itself and takes the tiles [T b / n, T (b + 1) / n) of it, so
+// blocks differ by at most one tile whatever the units' lengths are; a block's range is cut into segments at unit
+// boundaries. The four warps of a block stream the tiles of a segment in turn, each through its own ring of
+// shared-memory stages: K tiles by bulk copies (a tile is one contiguous run of 256-byte rows), V tiles by 2-D
+// tensor-map copies with the 128-byte swizzle, both completing on mbarriers with bounded waits.
+//   Q.K   fp64 on the CUDA cores, as in corm_fast.cuh (qk_tile): verdicts are compared with an fp64 oracle.
+//   P.V   on the tensor cores: mma.m16n8k16 with A = V^T (ldmatrix.trans from the swizzled tile) and B = the
+//         tile's probabilities, each split into two bf16 (p = hi + lo to ~2^-17 relative), the 2 G columns of B
+//         being (head, hi / lo); fp32 accumulation. A group of four heads fills the 8 columns of one instruction.
+//   softmax  per head against a fixed reference (the maximum of the warp's first tile of the segment) that moves only
+//         when a logit exceeds it by more than 16; Z in fp64.
+// Per segment every warp stores one record {m, Z, acc[128]} per head and the scaled logits of its tiles and bumps the
+// unit's arrival counter; warps never meet inside the streaming loop. After its streaming a block applies
+// Algorithm 1 to the slots it streamed, once the unit's records are all in (thresholds of Definition 3.1 from the
+// records, verdicts, register update, keep bits), and the unit's last block compacts it (bal_finish_block).
+// Launched with programmatic stream serialization: a step's blocks set up their barriers while the previous
+// step drains and wait for it before they read anything.
+#pragma once
+
+#include <cuda.h>
+
+#include "corm_common.cuh"
+#include "corm_fast.cuh"
+
+namespace corm {
+
+constexpr int kBalWarps = 4;
+constexpr int kBalThreads = kBalWarps * 32;
+constexpr int kBalKStages = 2;
+constexpr int kBalStages = 3;                                   // 2 K + 1 V per warp
+constexpr int kBalWarpBytes = kBalStages * kTileBytes;         // 24 KiB
+constexpr int kBalRingBytes = kBalWarps * kBalWarpBytes;       // 96 KiB, reused by the finish phase
+constexpr int kBalBlocksPerSm = 2;
+constexpr int kBalSegCap = 32;                                  // segments listed per window of a block's range
+constexpr int kBalRec = 16 + 4 * 128;                           // {double m, double Z, float acc[128]}
+constexpr int kBalCacheUnits = 16384;                            // units whose lengths the prologue parks in shared memory
+constexpr int kBalMaxTokens = 1 << 17;                          // the finish phase keeps 3 bits-per-32 arrays on chip
+
+struct BalSeg {
+    int32_t u;          // unit
+    int32_t l;          // its live length including the token appended by this step
+    int32_t tile0;      // first tile of the segment, counted inside the unit
+    int32_t n_tiles;    // tiles of the segment
+    int32_t gtile0;     // index of the unit's first tile in the step's tile list
+    int32_t t;          // tokens the unit's sequence has seen, this one included
+    int32_t n_unit;     // tiles of the whole unit
+    int32_t pad;
+};
+
+// Small block-wide variables. The kernel declares no static shared memory at all: its dynamic shared memory then
+// starts at the block's first usable byte, which is 1024-byte aligned, as the swizzled V tiles need (checked at entry).
+struct BalMisc {
+    double thr[4], Zg[4];            // finish phase: thresholds and normalisers per head
+    int scan[kBalThreads];           // finish phase: scratch of the block-wide prefix sums
+    int wsum[kBalWarps];
+    int first_u, first_P, nseg, more, next_u, next_P, last, failed;
+};
+
+// shared-memory carve-up behind the 1024-byte aligned ring
+struct BalSmem {
+    int psm, segq, segnew, bars, segs, misc, total, n_pre;
+};
+__host__ __device__ inline BalSmem bal_smem_layout(int G) {
+    BalSmem s;
+    int off = kBalRingBytes;
+    auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
+    s.psm = take(kBalWarps * kTileKeys * 16);
+    s.bars = take(kBalWarps * kBalStages * 8);
+    s.segs = take(kBalSegCap * (int)sizeof(BalSeg));
+    s.misc = take((int)sizeof(BalMisc));
+    // queries and appended rows of the first n_pre segments are fetched ahead; whatever shared memory is left
+    const int budget = (228 * 1024) / kBalBlocksPerSm - 1024 /* system */;
+    const int per = G * kRowBytes + 2 * kRowBytes;
+    int n_pre = (budget - off) / per;
+    if (n_pre > 8) n_pre = 8;
+    if (n_pre < 1) n_pre = 1;
+    s.n_pre = n_pre;
+    s.segq = take(n_pre * G * kRowBytes);
+    s.segnew = take(n_pre * 2 * kRowBytes);
+    s.total = off;
+    return s;
+}
+
+// ---- PTX wrappers of this kernel ----
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst_smem), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_m16n8k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// two floats -> one word of two bf16 (round to nearest even): `hi` in the upper half, `lo` in the lower
+__device__ __forceinline__ uint32_t pack_bf16x2(float hi, float lo) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// byte offset of 16-byte chunk c (0..15) of row r inside a V tile as the swizzled tensor copies lay it out: two
+// halves of 64 channels, rows of 128 bytes, chunk index XOR (row mod 8)
+__device__ __forceinline__ int vtile_offset(int r, int c) {
+    return (c >> 3) * (kTileBytes / 2) + r * 128 + ((((c & 7) ^ r) & 7) << 4);
+}
+
+// block of the balanced partition that owns tile x of the step's list (T tiles, n blocks)
+__device__ __forceinline__ int bal_block_of(long long x, long long T, int n) { return (int)(((x + 1) * n - 1) / T); }
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Per-segment bookkeeping of the finish phase (shared memory).
+struct BalFin {
+    int32_t rec0, n_blocks, tile_prefix, evict_on, last, sc_off, first;
+    int32_t pad;
+};
+
+// Finish phase of a block, by all its NT threads, after its streaming: Algorithm 1 for the slots of ALL the block's
+// segments in one pass, so that a block with several segments pays the chain of dependent memory round trips once.
+//   A. registers, positions and logits of the block's slots (its own stores and older data) are requested; then the
+//      block waits (bounded) until the arrival counter of each of its units says all records are stored. Every block
+//      of the launch is resident or becomes resident without anybody's help (the grid is no larger than the resident
+//      slots, and a launch only starts once every block of the previous one has started), and every warp stores all
+//      its records before the block waits for anything, so the waits end.
+//   B. thresholds of Definition 3.1 per (segment, head) from the unit's records: one warp per pair, a record per
+//      lane, fixed reduction trees, so every block of a unit gets the same bits.
+//   C. verdicts of the slots (OR over the group), register update, keep bits to the unit's global bit mask
+//      (segments are whole tiles, so no two blocks share a mask word).
+//   D. the unit's first block reduces the accumulators to the output of Eq. 1; after a second arrival counter the
+//      unit's last block scans the mask, fills the holes and publishes the new length.
+// scratch: the block's ring area, free by now.
+template <int G, bool PAGED, int NT>
+__device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
+                                 unsigned char* scratch, BalMisc* misc) {
+    constexpr int NW = kBalWarps;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    BalFin* fin = reinterpret_cast<BalFin*>(scratch);                         // [kBalSegCap]
+    double* thr = reinterpret_cast<double*>(scratch + kBalSegCap * sizeof(BalFin));   // [kBalSegCap][4]
+    double* Zg = thr + kBalSegCap * 4;                                         // [kBalSegCap][4]
+    float* sc_sm = reinterpret_cast<float*>(Zg + kBalSegCap * 4);              // scale factors of the records this block reduces
+    unsigned char* comp = scratch + 32 * 1024;                                 // compaction arrays (behind at most 21 KB of factors)
+    const size_t pstride = partial_stride(128);
+    if (tid == 0) {
+        int tp = 0, off = 0;
+        for (int si = 0; si < nseg; ++si) {
+            const BalSeg& sg = segs[si];
+            const long long P0 = sg.gtile0;
+            const int fb = bal_block_of(P0, T, nblk);
+            BalFin f;
+            f.n_blocks = bal_block_of(P0 + sg.n_unit - 1, T, nblk) - fb + 1;
+            f.rec0 = (fb + sg.u) * NW;
+            f.tile_prefix = tp;
+            f.evict_on = min(p.w, __ldcg(p.base_obs + sg.u / p.Hkv) + p.step + 1) >= p.w;
+            f.last = 0;
+            f.first = fb == blk;
+            f.sc_off = off;
+            f.pad = 0;
+            if (f.first) off += G * f.n_blocks * NW;
+            tp += sg.n_tiles;
+            fin[si] = f;
+        }
+        misc->last = tp;                                                       // tiles of the block in this window
+    }
+    __syncthreads();
+    const int n_slots = misc->last * kTileKeys;
+
+    // ---- A. the block's slots, batch by batch (one batch unless units are long) ----
+    constexpr int kB = (G == 4 ? 6 : 8);                                       // slots per thread and batch
+    double sv[kB][G];
+    uint32_t wv[kB];
+    int32_t pv[kB], jv[kB], siv[kB];
+    auto load_batch = [&](int base0) {
+#pragma unroll
+        for (int k = 0; k < kB; ++k) {
+            const int x = base0 + k * NT + tid;
+            wv[k] = 0u; pv[k] = 0; jv[k] = -1; siv[k] = 0;
+#pragma unroll
+            for (int g = 0; g < G; ++g) sv[k][g] = -INFINITY;
+            if (x < n_slots) {
+                const int tile = x >> 5;
+                int si = 0;
+                while (si + 1 < nseg && fin[si + 1].tile_prefix <= tile) ++si;
+                const BalSeg& sg = segs[si];
+                const int j = (sg.tile0 + tile - fin[si].tile_prefix) * kTileKeys + (x & 31);
+                siv[k] = si;
+                if (j < sg.l) {
+                    jv[k] = j;
+                    const double* st = p.stash + ((size_t)sg.u * p.C + j) * G;
+                    if (G == 4) {
+                        const double2 a = __ldcg(reinterpret_cast<const double2*>(st));
+                        const double2 c = __ldcg(reinterpret_cast<const double2*>(st + 2));
+                        sv[k][0] = a.x; sv[k][1] = a.y; sv[k][2 % G] = c.x; sv[k][3 % G] = c.y;
+                    } else if (G == 2) {
+                        const double2 a = __ldcg(reinterpret_cast<const double2*>(st));
+                        sv[k][0] = a.x; sv[k][1 % G] = a.y;
+                    } else {
+                        sv[k][0] = __ldcg(st);
+                    }
+                    wv[k] = __ldcg(p.word + (size_t)sg.u * p.C + j);
+                    pv[k] = __ldcg(p.pos + (size_t)sg.u * p.C + j);
+                }
+            }
+        }
+    };
+    load_batch(0);
+    if (tid == 0) {
+        const long long start = clock64();
+        for (int si = 0; si < nseg && !misc->failed; ++si) {
+            if (fin[si].n_blocks == 1) continue;                               // a block's own warps arrived before its last barrier
+            const uint32_t want = (uint32_t)(fin[si].n_blocks * NW);
+            while (ld_acquire_u32(p.ticket + segs[si].u) < want) {
+                if (clock64() - start > kWaitLimitCycles) { misc->failed = 1; break; }
+                __nanosleep(64);
+            }
+        }
+    }
+    __syncthreads();
+    if (misc->failed) { if (tid == 0) atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); return; }
+
+    // ---- B. thresholds: warp w takes the (segment, head) pairs w, w + NW, ... ----
+    for (int task = warp; task < nseg * G; task += NW) {
+        const int si = task / G, g = task - si * G;
+        const BalFin f = fin[si];
+        const int n_rec = f.n_blocks * NW;
+        const unsigned char* rec_u = p.partials + ((size_t)f.rec0 * G + g) * pstride;
+        double m = -INFINITY;
+        for (int s0 = 0; s0 < n_rec; s0 += 128) {                              // four records per lane in flight
+            double mm[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int s_ = s0 + k * 32 + lane;
+                mm[k] = s_ < n_rec ? __ldcg(reinterpret_cast<const double*>(rec_u + (size_t)s_ * G * pstride)) : -INFINITY;
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) m = fmax(m, mm[k]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+        double Z = 0.0;
+        for (int s0 = 0; s0 < n_rec; s0 += 128) {
+            double2 mz[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int s_ = s0 + k * 32 + lane;
+                mz[k] = s_ < n_rec ? __ldcg(reinterpret_cast<const double2*>(rec_u + (size_t)s_ * G * pstride)) : make_double2(-INFINITY, 0.0);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int s_ = s0 + k * 32 + lane;
+                const double sc = exp_nonpos(mz[k].x - m);
+                Z += mz[k].y * sc;
+                if (f.first && s_ < n_rec) sc_sm[f.sc_off + g * n_rec + s_] = (float)sc;
+            }
+        }
+        Z = warp_sum(Z);
+        if (lane == 0) {
+            Zg[si * 4 + g] = Z;
+            thr[si * 4 + g] = m + log(Z) + p.log_alpha - log((double)segs[si].t);   // Definition 3.1: s >= lse + ln(alpha) - ln(t)
+        }
+    }
+    __syncthreads();
+
+    // ---- C. verdicts, register update, keep flags ----
+    int n_imp = 0;
+    for (int base0 = 0; base0 < n_slots; base0 += kB * NT) {
+        if (base0) load_batch(base0);
+#pragma unroll
+        for (int k = 0; k < kB; ++k) {
+            const int base = base0 + k * NT;
+            if (base >= n_slots) break;                                         // uniform
+            const int si = siv[k], j = jv[k];
+            const BalSeg& sg = segs[si];
+            bool keep = false;
+            if (j >= 0) {
+                bool imp = false;
+#pragma unroll
+                for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= thr[si * 4 + g]);
+                const uint32_t wd = update_register(wv[k], imp, p.w, sg.t);
+                p.word[(size_t)sg.u * p.C + j] = wd;
+                keep = !fin[si].evict_on || register_needed(wd, p.w, sg.t) || pv[k] > sg.t - p.r;
+                n_imp += imp ? 1 : 0;
+            }
+            const uint32_t ballot = __ballot_sync(0xffffffffu, keep);           // a warp's 32 slots are one tile of one segment
+            const int x0 = base + warp * 32;
+            if (lane == 0 && x0 < n_slots) {
+                const int tile = x0 >> 5;
+                int s2 = 0;
+                while (s2 + 1 < nseg && fin[s2 + 1].tile_prefix <= tile) ++s2;
+                p.keepmask[(size_t)segs[s2].u * keepmask_words(p.C) + segs[s2].tile0 + tile - fin[s2].tile_prefix] = ballot;
+            }
+        }
+    }
+    warp_count(p.counters + CNT_IMPORTANT, n_imp);                             // Section 3.1's sparsity
+    __threadfence();
+    __syncthreads();
+    if (tid < nseg) {
+        const int si = tid, u = segs[si].u;
+        const unsigned prev = atomicAdd(p.ticket2 + u, 1u);
+        if (prev == (unsigned)(fin[si].n_blocks - 1)) {
+            fin[si].last = 1;
+            p.ticket2[u] = 0u; p.ticket[u] = 0u;                                // every block of the unit is past its wait
+        }
+        __threadfence();
+    }
+    // ---- D. Eq. 1 for the units that start in this block (thread = channel), while the arrivals above are in flight ----
+    for (int si = 0; si < nseg; ++si) {
+        const BalFin f = fin[si];
+        if (!f.first) continue;                                                 // uniform: written before the barriers above
+        const int n_rec = f.n_blocks * NW, u = segs[si].u;
+        const unsigned char* rec_u = p.partials + (size_t)f.rec0 * G * pstride;
+        float acc[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) acc[g] = 0.f;
+        for (int s0 = 0; s0 < n_rec; s0 += 8) {                                 // 8 G values in flight
+            float a[8][G];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    a[k][g] = s0 + k < n_rec ? __ldcg(reinterpret_cast<const float*>(rec_u + ((size_t)(s0 + k) * G + g) * pstride + 16) + tid) : 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (s0 + k < n_rec) acc[g] += a[k][g] * sc_sm[f.sc_off + g * n_rec + s0 + k];
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+            Elem<bf16_t>::store(reinterpret_cast<bf16_t*>(p.out) + ((size_t)u * G + g) * 128 + tid, (float)((double)acc[g] / Zg[si * 4 + g]));
+    }
+    __syncthreads();
+
+    // ---- the units this block is the last of: compaction ----
+    for (int si = 0; si < nseg; ++si) {
+        if (!fin[si].last) continue;                                            // uniform
+        const BalSeg& sg = segs[si];
+        const int u = sg.u, l = sg.l, t = sg.t, words = (l + 31) / 32 + 2, nwords = (l + 31) / 32;
+        uint32_t* keep_sm = reinterpret_cast<uint32_t*>(comp);
+        int* prefix = reinterpret_cast<int*>(keep_sm + words);
+        int32_t* pt_sm = prefix + words;
+        const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+        const uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
+        uint32_t* wordu = p.word + (size_t)u * p.C;
+        int32_t* posu = p.pos + (size_t)u * p.C;
+        for (int i = tid; i < nwords; i += NT) {
+            keep_sm[i] = __ldcg(keep_g + i);
+            if (PAGED) pt_sm[i] = __ldcg(pt_u + i);
+        }
+        __syncthreads();
+        int new_len = l, n_moved = 0;
+        if (fin[si].evict_on) {
+            block_popc_scan<NT>(keep_sm, prefix, nwords, misc->scan);
+            new_len = prefix[nwords];
+            if (new_len < l) {
+                const int kept_below = kept_before(keep_sm, prefix, new_len);
+                n_moved = new_len - kept_below;
+                int* holes = reinterpret_cast<int*>(p.stash + (size_t)u * G * p.C);   // every block is done with the logits
+                int* movers = holes + p.C;
+                for (int i = tid; i < nwords; i += NT) {
+                    const uint32_t m = keep_sm[i];
+                    const int w0 = i * 32;
+                    const uint32_t valid = l - w0 >= 32 ? 0xffffffffu : (1u << (l - w0)) - 1u;
+                    const uint32_t below = new_len - w0 >= 32 ? 0xffffffffu : (new_len > w0 ? (1u << (new_len - w0)) - 1u : 0u);
+                    uint32_t hm = ~m & valid & below;                       // evicted slots below the new length
+                    while (hm) {
+                        const int bit = __ffs(hm) - 1;
+                        hm &= hm - 1u;
+                        holes[w0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = w0 + bit;
+                    }
+                    uint32_t km = m & valid & ~below;                       // kept slots at or above it
+                    while (km) {
+                        const int bit = __ffs(km) - 1;
+                        km &= km - 1u;
+                        movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = w0 + bit;
+                    }
+                }
+                __syncthreads();
+                const size_t slab_row0 = (size_t)u * p.C;
+                block_move_rows<bf16_t, 128, NT>(
+                    reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
+                    [&](int slot) -> size_t {
+                        return PAGED ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
+                    },
+                    wordu, posu, movers, holes, n_moved);
+            }
+        }
+        if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+        if (tid == 0) {
+            p.live_out[u] = new_len;
+            publish_live(p.maxlive, p.step + 1, new_len);
+            atomicAdd(p.counters + CNT_APPENDED, 1ull);
+            atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+            if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+            if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
+        }
+        __syncthreads();                                                     // the arrays are reused by the next unit
+        (void)t;
+    }
+}
+
+template <int G, bool PAGED>
+__global__ void __launch_bounds__(kBalThreads, kBalBlocksPerSm)
+decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_constant__ CUtensorMap vmap) {
+    extern __shared__ __align__(1024) unsigned char smem[];   // the swizzled V tiles want 1024-byte alignment
+    constexpr int NT = kBalThreads, NW = kBalWarps;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nblk = (int)gridDim.x, blk = (int)blockIdx.x;
+    const BalSmem lay = bal_smem_layout(G);
+    unsigned char* my_tiles = smem + warp * kBalWarpBytes;
+    const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kBalStages * 8;
+    unsigned char* psm = smem + lay.psm + warp * kTileKeys * 16;
+    BalSeg* segs = reinterpret_cast<BalSeg*>(smem + lay.segs);
+    BalMisc* misc = reinterpret_cast<BalMisc*>(smem + lay.misc);
+    int* s_wsum = misc->wsum;
+    int &s_first_u = misc->first_u, &s_first_P = misc->first_P, &s_nseg = misc->nseg, &s_more = misc->more,
+        &s_next_u = misc->next_u, &s_next_P = misc->next_P, &s_failed = misc->failed;
+    unsigned char* Kl = reinterpret_cast<unsigned char*>(p.K);
+    unsigned char* Vl = reinterpret_cast<unsigned char*>(p.V);
+
+    // ---- set-up that reads nothing the previous step writes ----
+    if (smem_addr(smem) & 1023u) {                          // never expected; reported instead of mis-reading tiles
+        if (tid == 0) atomicCAS(p.status, 0, (int)CORM_ERR_INTERNAL);
+        return;
+    }
+    if (tid == 0) { prefetch_tensormap(&vmap); s_failed = 0; }
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kBalStages; ++s) mbar_init(my_bars + s * 8, 1);
+        fence_mbar_init();
+        fence_async_smem();
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the previous launch on the stream has completed
+
+    // ---- the step's tile list: tiles per unit, block-wide prefix sums, this block's range ----
+    // One round of global loads: every unit's length (and every sequence's token count) is parked in the ring area,
+    // which holds no tile yet, so that locating the block's range and listing its first segments read shared memory.
+    const int U = p.U, n_seq = U / p.Hkv;
+    const bool cached = U <= kBalCacheUnits;
+    int32_t* s_L = reinterpret_cast<int32_t*>(smem);                 // [U] live length incl. the new token, 0 = unit skipped
+    int32_t* s_bt = s_L + kBalCacheUnits;                            // [n_seq] tokens seen before this launch's steps
+    const int per = (U + NT - 1) / NT, lo = min(U, tid * per), hi = min(U, lo + per);
+    auto len_global = [&](int v) -> int {                            // live length incl. the new token, 0 if the unit cannot take it
+        const int l = __ldcg(p.live_in + v) + 1;
+        const int room = PAGED ? __ldcg(p.page_room + v) : 1;
+        return (l <= p.C && room) ? l : 0;
+    };
+    bool use_cache = cached;
+    auto len_of = [&](int v) -> int { return use_cache ? s_L[v] : len_global(v); };
+    auto tokens_of = [&](int v) -> int { return (use_cache ? s_bt[v / p.Hkv] : __ldcg(p.base_tokens + v / p.Hkv)) + p.step + 1; };
+    if (cached)
+        for (int i = tid; i < n_seq; i += NT) s_bt[i] = __ldcg(p.base_tokens + i);
+    int sum = 0;
+    for (int v = lo; v < hi; ++v) {
+        const int l = len_global(v);
+        if (cached) s_L[v] = l;
+        if (!l && blk == 0) {        // a full slab or an exhausted pool: reported, the unit is left as it is
+            const int l_old = __ldcg(p.live_in + v);
+            atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY);
+            p.live_out[v] = l_old;
+            publish_live(p.maxlive, p.step + 1, l_old);
+        }
+        sum += (l + kTileKeys - 1) / kTileKeys;
+    }
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    int excl = incl - sum;
+    long long T = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { if (w < warp) excl += s_wsum[w]; T += s_wsum[w]; }
+    if (T == 0) return;
+    const long long S_b = T * blk / nblk, S_e = T * (blk + 1) / nblk;
+    if (S_b == S_e) return;                                    // more blocks than tiles
+    if (sum > 0 && excl <= S_b && S_b < (long long)excl + sum) {
+        int run = excl;
+        for (int v = lo; v < hi; ++v) {
+            const int tv = (len_of(v) + kTileKeys - 1) / kTileKeys;
+            if (S_b < (long long)run + tv) { s_first_u = v; s_first_P = run; break; }
+            run += tv;
+        }
+    }
+    __syncthreads();
+    int win_u = s_first_u, win_P = s_first_P;
+
+    const int h = lane >> 4, ci = lane & 15;
+    const int key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);     // tile key this lane owns after the fold of qk_tile
+    const double inv_root_d = 0.088388347648318440550;        // 1/sqrt(128)
+    // ldmatrix row addresses of this lane inside a V tile: matrix lane/8 of a 16 x 16 block = keys (lane/16)*8 + lane%8,
+    // channels + 8 for the odd matrices; the chunk index is XORed with the row (lane % 8) by the swizzle
+    const int lm_row = ((lane >> 4) << 3) + (lane & 7), lm_odd = (lane >> 3) & 1, lm_x = lane & 7;
+    int n_consumed = 0;                                        // tiles this warp has consumed: ring slots and parities
+    bool failed = false;
+
+    for (;;) {   // windows of at most kBalSegCap segments (one window unless units are tiny)
+        if (warp == 0) {
+            // lanes look at units win_u + lane; a unit with tiles that starts before the end of the range is a segment
+            const int v = win_u + lane;
+            const int l = v < U ? len_of(v) : 0, tv = (l + kTileKeys - 1) / kTileKeys;
+            int inc = tv;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += up;
+            }
+            const long long Pv = (long long)win_P + inc - tv;   // index of the unit's first tile in the list
+            const bool is_seg = tv > 0 && Pv < S_e && Pv + tv > S_b;
+            const uint32_t segmask = __ballot_sync(0xffffffffu, is_seg);
+            if (is_seg) {
+                BalSeg sg;
+                const long long a = Pv > S_b ? Pv : S_b, e = Pv + tv < S_e ? Pv + tv : S_e;
+                sg.u = v; sg.l = l; sg.tile0 = (int)(a - Pv); sg.n_tiles = (int)(e - a); sg.gtile0 = (int)Pv;
+                sg.t = tokens_of(v); sg.n_unit = tv; sg.pad = 0;
+                segs[__popc(segmask & ((1u << lane) - 1u))] = sg;
+            }
+            const long long P_end = (long long)win_P + __shfl_sync(0xffffffffu, inc, 31);
+            if (lane == 0) {
+                s_nseg = __popc(segmask);
+                s_more = (P_end < S_e && win_u + 32 < U) ? 1 : 0;
+                s_next_u = win_u + 32;
+                s_next_P = (int)P_end;
+            }
+        }
+        __syncthreads();
+        use_cache = false;                                     // the ring is about to receive tiles
+        const int nseg = s_nseg;
+
+        // ---- this warp's tiles: cursor (segment, index among the warp's tiles of that segment) ----
+        struct Cur { int si, it; };
+        auto seg_has = [&](int si) { return segs[si].n_tiles > warp; };
+        auto cur_first = [&]() { Cur c{0, 0}; while (c.si < nseg && !seg_has(c.si)) ++c.si; return c; };
+        auto cur_next = [&](Cur c) {
+            if (c.si >= nseg) return c;
+            ++c.it;
+            if (warp + c.it * NW >= segs[c.si].n_tiles) { c.it = 0; do { ++c.si; } while (c.si < nseg && !seg_has(c.si)); }
+            return c;
+        };
+        // first row of a tile in the layer's K / V storage; a page entry outside the pool (a broken table) is
+        // reported and page 0 is read instead, so that no address is ever formed from it
+        auto tile_row0 = [&](const BalSeg& sg, int ti) -> long long {
+            if (!PAGED) return (long long)sg.u * p.C + (long long)ti * kTileKeys;
+            const int pg = __ldcg(p.page_table + (size_t)sg.u * p.pt_stride + ti);
+            if (pg <= 0 || pg > p.pool_pages) { atomicCAS(p.status, 0, (int)CORM_ERR_INTERNAL); return -1; }
+            return (long long)(pg - 1) * kPageKeys;
+        };
+        auto issue_k = [&](Cur c, int n) {                     // lane 0 only
+            const BalSeg& sg = segs[c.si];
+            const int ti = sg.tile0 + warp + c.it * NW, slot = n % kBalKStages;
+            const uint32_t bytes = (uint32_t)min(kTileKeys, sg.l - ti * kTileKeys) * kRowBytes;
+            long long row0 = tile_row0(sg, ti);
+            if (row0 < 0) row0 = 0;
+            mbar_expect_tx(my_bars + slot * 8, bytes);
+            bulk_load(smem_addr(my_tiles + slot * kTileBytes), Kl + row0 * kRowBytes, bytes, my_bars + slot * 8);
+        };
+        auto issue_v = [&](Cur c) {                            // lane 0 only; the box is always 32 rows
+            const BalSeg& sg = segs[c.si];
+            const int ti = sg.tile0 + warp + c.it * NW;
+            long long row0 = tile_row0(sg, ti);
+            if (row0 < 0) row0 = 0;
+            const uint32_t bar = my_bars + kBalKStages * 8, dst = smem_addr(my_tiles + kBalKStages * kTileBytes);
+            mbar_expect_tx(bar, kTileBytes);
+            tma_load_2d(dst, &vmap, 0, (int)row0, bar);
+            tma_load_2d(dst + kTileBytes / 2, &vmap, 64, (int)row0, bar);
+        };
+        Cur cc = cur_first(), ck = cc, cv = cc;
+        int nk = n_consumed;
+        if (lane == 0) {
+            fence_async_smem();
+            for (int s = 0; s < kBalKStages && ck.si < nseg; ++s) { issue_k(ck, nk); ++nk; ck = cur_next(ck); }
+            if (cv.si < nseg) { issue_v(cv); cv = cur_next(cv); }
+        } else {
+            for (int s = 0; s < kBalKStages && ck.si < nseg; ++s) { ++nk; ck = cur_next(ck); }
+            if (cv.si < nseg) cv = cur_next(cv);
+        }
+        // queries and appended rows of the first segments, fetched while the first tiles are on their way
+        {
+            const int n_pre = min(nseg, lay.n_pre);
+            const int per_seg = G * 16 + 32;
+            for (int x = tid; x < n_pre * per_seg; x += NT) {
+                const int si = x / per_seg, c = x - si * per_seg;
+                const BalSeg& sg = segs[si];
+                if (c < G * 16) {
+                    cp_async16(smem_addr(smem + lay.segq + (si * G * 16 + c) * 16),
+                               reinterpret_cast<const unsigned char*>(p.q) + ((size_t)sg.u * G * 16 + c) * 16);
+                } else if (sg.tile0 + sg.n_tiles == sg.n_unit) {          // the segment holds the unit's last tile
+                    const int cc2 = c - G * 16;
+                    const unsigned char* src = cc2 < 16 ? reinterpret_cast<const unsigned char*>(p.k_new) + ((size_t)sg.u * 16 + cc2) * 16
+                                                        : reinterpret_cast<const unsigned char*>(p.v_new) + ((size_t)sg.u * 16 + cc2 - 16) * 16;
+                    cp_async16(smem_addr(smem + lay.segnew + (si * 32 + cc2) * 16), src);
+                }
+            }
+            cp_async_wait_all();
+        }
+        __syncthreads();
+
+        for (int si = 0; si < nseg; ++si) {
+            const BalSeg sg = segs[si];
+            const int u = sg.u, l = sg.l, l_old = l - 1, t = sg.t;
+            double M[G], Zl[G];
+            float Mref[G];
+            float accd[8][4];
+#pragma unroll
+            for (int g = 0; g < G; ++g) { M[g] = -INFINITY; Zl[g] = 0.0; Mref[g] = -INFINITY; }
+#pragma unroll
+            for (int cb = 0; cb < 8; ++cb)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) accd[cb][e] = 0.f;
+            if (cc.si == si) {
+                // the lane's 8 channels of every query head, widened to fp64
+                double qd[G][8];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const uint4 raw = si < lay.n_pre ? *reinterpret_cast<const uint4*>(smem + lay.segq + ((si * G + g) * 16 + ci) * 16)
+                                                     : __ldcg(reinterpret_cast<const uint4*>(p.q) + ((size_t)u * G + g) * 16 + ci);
+                    unpack8_to_double(raw, qd[g]);
+                }
+                uint32_t* wordu = p.word + (size_t)u * p.C;
+                int32_t* posu = p.pos + (size_t)u * p.C;
+                bool first = true;
+                while (cc.si == si) {
+                    const int ti = sg.tile0 + warp + cc.it * NW;
+                    const int k0 = ti * kTileKeys;
+                    const int n_valid = min(kTileKeys, l - k0);
+                    const bool has_new = (l_old >= k0 && l_old < k0 + kTileKeys);   // this tile holds the appended token
+                    const int kslot = n_consumed % kBalKStages;
+                    unsigned char* ktile = my_tiles + kslot * kTileBytes;
+                    unsigned char* vtile = my_tiles + kBalKStages * kTileBytes;
+                    long long row0 = 0;
+                    uint4 newk = make_uint4(0, 0, 0, 0), newv = make_uint4(0, 0, 0, 0);
+                    if (has_new) {
+                        row0 = tile_row0(sg, ti);
+                        if (lane < 16) {
+                            if (si < lay.n_pre) {
+                                newk = *reinterpret_cast<const uint4*>(smem + lay.segnew + (si * 32 + lane) * 16);
+                                newv = *reinterpret_cast<const uint4*>(smem + lay.segnew + (si * 32 + 16 + lane) * 16);
+                            } else {
+                                newk = __ldcg(reinterpret_cast<const uint4*>(p.k_new) + (size_t)u * 16 + lane);
+                                newv = __ldcg(reinterpret_cast<const uint4*>(p.v_new) + (size_t)u * 16 + lane);
+                            }
+                        }
+                    }
+                    if (!failed && !mbar_wait(my_bars + kslot * 8, (n_consumed / kBalKStages) & 1)) failed = true;   // once one wait has expired the rest are skipped
+                    if (has_new && row0 >= 0) {   // append: the new row goes to the cache and into the arriving tile
+                        if (lane < 16) {
+                            *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = newk;
+                            reinterpret_cast<uint4*>(Kl + (row0 + (l_old - k0)) * kRowBytes)[lane] = newk;
+                        }
+                        if (lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
+                        __syncwarp();
+                    }
+                    double sown[G];
+                    qk_tile<G>(ktile, qd, lane, sown);
+                    __syncwarp();
+                    if (ck.si < nseg) {
+                        if (lane == 0) { fence_async_smem(); issue_k(ck, nk); }
+                        ++nk; ck = cur_next(ck);
+                    }
+
+                    const bool valid = key_own < n_valid;
+                    const int j_own = k0 + key_own;
+                    double sv[G], ex[G];
+#pragma unroll
+                    for (int g = 0; g < G; ++g) sv[g] = valid ? sown[g] * inv_root_d : -INFINITY;   // Eq. 2's exponent
+                    bool over = first;
+#pragma unroll
+                    for (int g = 0; g < G; ++g) over |= ((float)sv[g] > Mref[g] + 16.f);
+                    if (__any_sync(0xffffffffu, over)) {      // the reference moves: first tile, or a logit far above it (rare)
+                        float mt[G];
+#pragma unroll
+                        for (int g = 0; g < G; ++g) mt[g] = (float)sv[g];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                            for (int g = 0; g < G; ++g) mt[g] = fmaxf(mt[g], __shfl_xor_sync(0xffffffffu, mt[g], o));
+                        float scf[G];
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            const float mn = fmaxf(Mref[g], mt[g]);
+                            const double sc = first ? 0.0 : exp_nonpos((double)Mref[g] - (double)mn);
+                            Zl[g] *= sc;
+                            scf[g] = (float)sc;
+                            Mref[g] = mn;
+                        }
+                        // accumulators of this thread belong to head lane % 4
+                        float mine = scf[0];
+#pragma unroll
+                        for (int g = 1; g < G; ++g) mine = (lane & 3) == g ? scf[g] : mine;
+#pragma unroll
+                        for (int cb = 0; cb < 8; ++cb)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) accd[cb][e] *= mine;
+                        first = false;
+                    }
+                    uint32_t pw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        ex[g] = valid ? exp_nonpos(sv[g] - (double)Mref[g]) : 0.0;
+                        Zl[g] += ex[g];
+                        const float pf = (float)ex[g];
+                        const float hi_f = __uint_as_float(pack_bf16x2(0.f, pf) << 16);
+                        pw[g] = pack_bf16x2(pf - hi_f, pf);                 // column 2g = hi, column 2g + 1 = lo
+                    }
+                    *reinterpret_cast<uint4*>(psm + key_own * 16) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+                    if (valid) {
+                        double* dst = p.stash + ((size_t)u * p.C + j_own) * G;
+                        if (G == 4) {
+                            reinterpret_cast<double2*>(dst)[0] = make_double2(sv[0], sv[1]);
+                            reinterpret_cast<double2*>(dst)[1] = make_double2(sv[2 % G], sv[3 % G]);
+                        } else if (G == 2) {
+                            reinterpret_cast<double2*>(dst)[0] = make_double2(sv[0], sv[1 % G]);
+                        } else {
+                            dst[0] = sv[0];
+                        }
+                    }
+                    __syncwarp();
+
+                    if (!failed && !mbar_wait(my_bars + kBalKStages * 8, n_consumed & 1)) failed = true;
+                    if (has_new && row0 >= 0 && lane < 16) {
+                        *reinterpret_cast<uint4*>(vtile + vtile_offset(l_old - k0, lane)) = newv;
+                        reinterpret_cast<uint4*>(Vl + (row0 + (l_old - k0)) * kRowBytes)[lane] = newv;
+                    }
+                    if (n_valid < kTileKeys)     // rows past the unit's end hold whatever the slab had: make them harmless for 0 * v
+                        for (int x = lane; x < (kTileKeys - n_valid) * 16; x += 32) {
+                            const int r = n_valid + (x >> 4), c = x & 15;
+                            *reinterpret_cast<uint4*>(vtile + (c >> 3) * (kTileBytes / 2) + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                    __syncwarp();
+                    {
+                        uint32_t bfr[4];
+                        ldmatrix_x4_trans(bfr, smem_addr(psm + lane * 16));   // keys 0-7 | 8-15 | 16-23 | 24-31 x 8 columns
+                        const uint32_t vbase = smem_addr(vtile) + lm_row * 128;
+#pragma unroll
+                        for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+                            for (int cb = 0; cb < 8; ++cb) {
+                                uint32_t a[4];
+                                const int chunk = ((cb & 3) * 2 + lm_odd) ^ lm_x;
+                                ldmatrix_x4_trans(a, vbase + (cb >> 2) * (kTileBytes / 2) + kb * 16 * 128 + chunk * 16);
+                                mma_bf16_m16n8k16(accd[cb], a, bfr[2 * kb], bfr[2 * kb + 1]);          // Eq. 1
+                            }
+                    }
+                    __syncwarp();
+                    ++n_consumed;
+                    cc = cur_next(cc);
+                    if (cv.si < nseg) {
+                        if (lane == 0) { fence_async_smem(); issue_v(cv); }
+                        cv = cur_next(cv);
+                    }
+                }
+                // fold the warp: Z over the lanes; the accumulators already hold whole-tile sums per (head, channel)
+#pragma unroll
+                for (int g = 0; g < G; ++g) { Zl[g] = warp_sum(Zl[g]); M[g] = (double)Mref[g]; }
+            }
+            // The warp's record {M, Z, acc[128]} per head goes straight to global memory (a warp without a tile in
+            // this segment stores M = -inf, Z = 0, acc = 0), then the warp's arrival: no block-wide step here, the
+            // other warps of the block stream on.
+            const size_t pstride = partial_stride(128);
+            unsigned char* rec_w = p.partials + ((size_t)(blk + u) * NW + warp) * G * pstride;   // blk + u is unique: both grow along the tile list
+            if (lane < G) {
+                double* mz = reinterpret_cast<double*>(rec_w + (size_t)lane * pstride);
+                double Mg = M[0], Zg = Zl[0];
+#pragma unroll
+                for (int g = 1; g < G; ++g) { Mg = lane == g ? M[g] : Mg; Zg = lane == g ? Zl[g] : Zg; }
+                *reinterpret_cast<double2*>(mz) = make_double2(Mg, Zg);
+            }
+            if ((lane & 3) < G) {
+                float* a = reinterpret_cast<float*>(rec_w + (size_t)(lane & 3) * pstride + 16);
+#pragma unroll
+                for (int cb = 0; cb < 8; ++cb) {
+                    a[cb * 16 + (lane >> 2)] = accd[cb][0] + accd[cb][1];       // hi + lo columns of the head
+                    a[cb * 16 + 8 + (lane >> 2)] = accd[cb][2] + accd[cb][3];
+                }
+            }
+            __threadfence();
+            __syncwarp();
+            if (lane == 0) atomicAdd(p.ticket + u, 1u);   // this warp's record and logits of the segment are stored
+        }
+        __syncthreads();
+        if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
+        __syncthreads();
+        if (s_failed) return;                   // a bounded wait expired: reported through the status word
+        // ---- Algorithm 1 for the slots this block streamed; the ring is free now ----
+        bal_finish_block<G, PAGED, NT>(p, segs, nseg, blk, T, nblk, smem, misc);
+        if (s_failed) return;
+        if (!s_more) break;
+        __syncthreads();
+        win_u = s_next_u; win_P = s_next_P;
+        __syncthreads();
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// The V storage of one layer as a 2-D tensor [rows][128] of bf16 with boxes of 32 rows x 64 channels and the
+// 128-byte swizzle; rows = every slab row or every pool row of the layer. The map only ever covers memory of the
+// cache's own device.
+inline corm_status_t make_v_tensor_map(CUtensorMap* out, void* v_layer, unsigned long long rows) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn ||
+            q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return CORM_ERR_UNSUPPORTED;
+        }
+        encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    const cuuint64_t dims[2] = {128, rows};
+    const cuuint64_t strides[1] = {kRowBytes};
+    const cuuint32_t box[2] = {64, kTileKeys};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, v_layer, dims, strides, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CORM_OK : CORM_ERR_CUDA;
+}
+
+// records the balanced kernel may write in one step: one per warp of every (block, unit) pair on the tile list
+__host__ __device__ inline size_t bal_record_count(int n_blocks, int U) { return ((size_t)n_blocks + (size_t)U) * kBalWarps; }
+
+inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& vmap, int G, int upper, int sm_count,
+                                            size_t partial_capacity_records, cudaStream_t st, int* n_launched) {
+    *n_launched = 0;
+    if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
+    if (p.C > kBalMaxTokens) return CORM_ERR_UNSUPPORTED;
+    const int sms = sm_count > 0 ? sm_count : 148;
+    // one block per resident slot, fewer when the step cannot have that many tiles per warp
+    const long long tiles_upper = (long long)((upper + kTileKeys - 1) / kTileKeys) * p.U;
+    long long grid = (long long)sms * kBalBlocksPerSm;
+    if (tiles_upper / kBalWarps + 1 < grid) grid = tiles_upper / kBalWarps + 1;
+    if (bal_record_count((int)grid, p.U) > partial_capacity_records) return CORM_ERR_UNSUPPORTED;
+    const BalSmem lay = bal_smem_layout(G);
+    auto launch = [&](auto kern) -> corm_status_t {
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), (size_t)lay.total);
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kBalThreads);
+        cfg.dynamicSmemBytes = (size_t)lay.total;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set-up overlaps the previous step's tail
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, p, vmap);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        return CORM_OK;
+    };
+    corm_status_t rc;
+    if (p.page_table) rc = G == 1 ? launch(decode_balanced_kernel<1, true>) : G == 2 ? launch(decode_balanced_kernel<2, true>) : launch(decode_balanced_kernel<4, true>);
+    else rc = G == 1 ? launch(decode_balanced_kernel<1, false>) : G == 2 ? launch(decode_balanced_kernel<2, false>) : launch(decode_balanced_kernel<4, false>);
+    if (rc == CORM_OK) *n_launched = 1;
+    return rc;
+}
+
+}  // namespace corm

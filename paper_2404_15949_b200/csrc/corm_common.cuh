@@ -58,6 +58,7 @@ struct DecodeParams {
     const int32_t* base_tokens;  // [B] tokens seen when the step counter was last rebased
     const int32_t* base_obs;     // [B] verdict rows recorded at that time
     uint32_t* ticket;         // [U] arrival counters of the splits of a unit (zero between steps)
+    uint32_t* ticket2;        // [U] second arrival counters (balanced kernel: blocks done with their verdicts)
     unsigned long long* counters;  // [CNT_COUNT]
     int32_t* status;          // sticky device status
     unsigned long long* maxlive;  // (steps done << 32 | longest live length after that step), atomicMax; may be null

@@ -48,8 +48,13 @@ SMALL = [
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, 2),      # units of several splits finished inside the decode launch
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, 3),      # ... by the verdict launch
     ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 64, False),
-    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True),
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True),     # grouped heads: the balanced kernel by default
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, 2),
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, 3),
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 0, 4),       # the balanced kernel forced for one head per KV head
+    ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 0, 4),
+    ("bf16", 128, 4, 5, 3, (1, 40), 60, 8, 4, 0, 4),           # tiny units: many segments per block, units of one tile
+    ("bf16", 128, 4, 1, 1, (3000, 3000), 12, 8, 64, 0, 4),     # one long unit cut over many blocks
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, False),
     ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True),
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 64, True),
