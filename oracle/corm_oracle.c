@@ -343,9 +343,38 @@ int oracle_export_unit(const corm_oracle *o, int layer, int b, int h, double *k,
     return l;
 }
 
-/* Replaces one unit's entries and its sequence counters (used to start both sides from the same state). */
+/* Copies the whole registers of one unit's live entries, in order: regs [live][REG_WORDS], word 0 = newest 32
+ * verdicts (bit b of the register = verdict of the query b steps ago, Algorithm 1's message column). */
+int oracle_export_registers(const corm_oracle *o, int layer, int b, int h, uint32_t *regs) {
+    size_t u = unit_index(o, layer, b, h), C = (size_t)o->max_tokens;
+    int l = o->live[u];
+    memcpy(regs, o->word + u * C * REG_WORDS, (size_t)l * REG_WORDS * sizeof(uint32_t));
+    return l;
+}
+
+int oracle_register_words(void) { return REG_WORDS; }
+
+/* Replaces one unit's entries and its sequence counters (used to start both sides from the same state, and as a
+ * checkpoint restore). regs: [live][REG_WORDS] whole registers as oracle_export_registers gives them. */
+int oracle_import_unit_full(corm_oracle *o, int layer, int b, int h, int live, const double *k, const double *v,
+                            const uint32_t *regs, const int *pos, int n_tokens, int n_obs) {
+    if (live < 0 || live > o->max_tokens) return ORACLE_CAPACITY;
+    size_t u = unit_index(o, layer, b, h), C = (size_t)o->max_tokens, d = (size_t)o->head_dim;
+    memcpy(o->k + u * C * d, k, (size_t)live * d * sizeof(double));
+    memcpy(o->v + u * C * d, v, (size_t)live * d * sizeof(double));
+    memcpy(o->word + u * C * REG_WORDS, regs, (size_t)live * REG_WORDS * sizeof(uint32_t));
+    memcpy(o->pos + u * C, pos, (size_t)live * sizeof(int));
+    o->live[u] = live;
+    o->t[(size_t)layer * o->batch + b] = n_tokens;
+    o->n_obs[(size_t)layer * o->batch + b] = n_obs;
+    return ORACLE_OK;
+}
+
+/* The same with one 32-bit word per entry (the newest 32 verdicts): all of the register only for windows of up to
+ * 32 queries, so wider windows are refused rather than silently losing verdicts. */
 int oracle_import_unit(corm_oracle *o, int layer, int b, int h, int live, const double *k, const double *v,
                        const uint32_t *word, const int *pos, int n_tokens, int n_obs) {
+    if (o->w > 32) return ORACLE_BAD_ARG;
     if (live < 0 || live > o->max_tokens) return ORACLE_CAPACITY;
     size_t u = unit_index(o, layer, b, h), C = (size_t)o->max_tokens, d = (size_t)o->head_dim;
     memcpy(o->k + u * C * d, k, (size_t)live * d * sizeof(double));

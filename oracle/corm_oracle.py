@@ -47,6 +47,11 @@ def _load():
     lib.oracle_export_unit.argtypes = [vp, c_int, c_int, c_int, vp, vp, vp, vp]
     lib.oracle_import_unit.restype = c_int
     lib.oracle_import_unit.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp, vp, vp, c_int, c_int]
+    lib.oracle_import_unit_full.restype = c_int
+    lib.oracle_import_unit_full.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp, vp, vp, c_int, c_int]
+    lib.oracle_export_registers.restype = c_int
+    lib.oracle_export_registers.argtypes = [vp, c_int, c_int, c_int, vp]
+    lib.oracle_register_words.restype = c_int
     lib.oracle_export_age.restype = c_int
     lib.oracle_export_age.argtypes = [vp, c_int, c_int, c_int, vp]
     lib.oracle_counters.argtypes = [vp, vp, vp, vp, vp]
@@ -133,18 +138,28 @@ class CormOracle:
                                     pos.ctypes.data)
         age = np.empty((l,), dtype=np.int32)
         self.lib.oracle_export_age(self.h, layer, b, h, age.ctypes.data)
-        return dict(k=k, v=v, word=word, pos=pos, age=age, live_len=l, n_tokens=self.n_tokens(layer, b),
+        regs = np.empty((l, self.lib.oracle_register_words()), dtype=np.uint32)       # the whole registers
+        self.lib.oracle_export_registers(self.h, layer, b, h, regs.ctypes.data)
+        return dict(k=k, v=v, word=word, pos=pos, age=age, regs=regs, live_len=l, n_tokens=self.n_tokens(layer, b),
                     n_obs=self.n_obs(layer, b))
 
     def import_unit(self, layer, b, h, k, v, word, pos, n_tokens, n_obs):
+        """``word``: [live] newest-32-verdict words (windows of up to 32 queries only) or [live, register words]
+        whole registers as ``export_unit`` returns them under ``regs`` (any window)."""
         k = np.ascontiguousarray(k, dtype=np.float64)
         v = np.ascontiguousarray(v, dtype=np.float64)
         word = np.ascontiguousarray(word, dtype=np.uint32)
         pos = np.ascontiguousarray(pos, dtype=np.int32)
-        rc = self.lib.oracle_import_unit(self.h, layer, b, h, int(k.shape[0]), k.ctypes.data, v.ctypes.data,
-                                         word.ctypes.data, pos.ctypes.data, int(n_tokens), int(n_obs))
+        if word.ndim == 2:
+            assert word.shape == (k.shape[0], self.lib.oracle_register_words())
+            fn = self.lib.oracle_import_unit_full
+        else:
+            assert word.shape == (k.shape[0],)
+            fn = self.lib.oracle_import_unit
+        rc = fn(self.h, layer, b, h, int(k.shape[0]), k.ctypes.data, v.ctypes.data, word.ctypes.data, pos.ctypes.data,
+                int(n_tokens), int(n_obs))
         if rc:
-            raise RuntimeError(f"oracle_import_unit failed with code {rc}")
+            raise RuntimeError(f"oracle import failed with code {rc}")
 
     def counters(self):
         vals = [ctypes.c_longlong(0) for _ in range(4)]

@@ -346,6 +346,75 @@ def test_near_threshold_band_counter():
     assert c["near_threshold"] == c["verdict_evals"] == 1 + 2 + 3 + 4 + 5
 
 
+def test_near_band_width_follows_the_handworked_probabilities():
+    """The counter of verdict evaluations with |p - alpha/t| <= rel * alpha/t, on the hand-worked decode case where every
+    probability is known as a fraction (tests/golden/handworked_decode.txt): the expected counts are taken from those
+    fractions here, for several band widths."""
+    from fractions import Fraction as Fr
+    c = [8, 1, 1, 4, 1, 1]
+    live_before = [[1], [1, 2], [1, 2, 3], [1, 3, 4], [1, 4, 5], [1, 4, 5, 6]]     # keys attended at t = 1..6 (golden file)
+    dist = []                                                   # |p - 1/t| / (1/t) of every evaluation, exactly
+    for t, live in enumerate(live_before, start=1):
+        Z = sum(c[j - 1] for j in live)
+        dist += [abs(Fr(c[j - 1], Z) * t - 1) for j in live]
+    for rel in (Fr(0), Fr(1, 10), Fr(1, 2), Fr(13, 20), Fr(3, 2), Fr(100)):
+        o = CormOracle(1, 1, 1, 1, 64, 8, 2, 1, 1.0)
+        o.set_near_band(float(rel))
+        _empty_prompt(o, 64)
+        q = np.zeros((1, 1, 64), np.float32); q[0, 0, 0] = 8.0
+        for j in range(6):
+            k = np.zeros((1, 1, 64), np.float32); k[0, 0, 0] = np.float32(np.log(c[j]))
+            o.decode_step(0, q, k, np.full((1, 1, 64), j + 1.0, np.float32))
+        n = o.counters()
+        assert n["verdict_evals"] == len(dist) == 16
+        # float32 ln(c_j) moves a probability by ~1e-7 relative: widths are chosen away from every exact distance
+        assert all(abs(float(x - rel)) > 1e-3 for x in dist if x != 0)
+        assert n["near_threshold"] == sum(1 for x in dist if x <= rel), float(rel)
+
+
+@pytest.mark.parametrize("w,G", [(8, 1), (5, 2), (40, 1), (100, 2)])
+def test_export_import_roundtrip_then_identical_future(w, G):
+    from paper_2404_15949_b200.workload import CONFIGS, generate
+    """A unit exported in mid-run (whole registers) and imported into a fresh oracle must have the same future:
+    identical outputs, registers, positions and rows for the next 20 steps. One-word import is for windows of up
+    to 32 queries and is refused beyond."""
+    cfg = CONFIGS[1].with_(batch=2, n_q_heads=2 * G, n_kv_heads=2, head_dim=16, prompt_min=max(40, w + 5),
+                           prompt_max=max(40, w + 5) + 30, steps=45, window_w=w, recent_r=6, alpha=2.0 if w > 32 else 1.0, gqa_rho=0.7 if G > 1 else 0.0,
+                           hh_min=2, hh_max=4, seed=99)
+    data = generate(cfg)
+    mk = lambda: CormOracle(1, 2, 2 * G, 2, 16, cfg.max_tokens, w, 6, cfg.alpha)
+    a, b = mk(), mk()
+    a.compress_prompt(0, data.k_prompt, data.v_prompt, data.q_last, data.prompt_lens)
+    for s in range(25):
+        a.decode_step(0, data.q[s], data.k_new[s], data.v_new[s])
+    assert a.counters()["evicted"] > 0
+    b.compress_prompt(0, None, None, None, np.zeros(2, np.int32))                  # a fresh, empty cache
+    for ib in range(2):
+        for ih in range(2):
+            st = a.export_unit(0, ib, ih)
+            b.import_unit(0, ib, ih, st["k"], st["v"], st["regs"], st["pos"], st["n_tokens"], st["n_obs"])
+            if w > 32:
+                with pytest.raises(RuntimeError):
+                    mk().import_unit(0, ib, ih, st["k"], st["v"], st["word"], st["pos"], st["n_tokens"], st["n_obs"])
+    if w <= 32:                                                                      # the one-word form carries the same state
+        c = mk()
+        c.compress_prompt(0, None, None, None, np.zeros(2, np.int32))
+        for ib in range(2):
+            for ih in range(2):
+                st = a.export_unit(0, ib, ih)
+                c.import_unit(0, ib, ih, st["k"], st["v"], st["word"], st["pos"], st["n_tokens"], st["n_obs"])
+    others = [b] + ([c] if w <= 32 else [])
+    for s in range(25, 45):
+        ref = a.decode_step(0, data.q[s], data.k_new[s], data.v_new[s])
+        for o in others:
+            assert np.array_equal(ref, o.decode_step(0, data.q[s], data.k_new[s], data.v_new[s]))
+            for ib in range(2):
+                for ih in range(2):
+                    x, y = a.export_unit(0, ib, ih), o.export_unit(0, ib, ih)
+                    for key in ("k", "v", "regs", "pos", "age", "live_len", "n_tokens", "n_obs"):
+                        assert np.array_equal(x[key], y[key]), (s, ib, ih, key)
+
+
 def test_bad_arguments_and_capacity():
     with pytest.raises(ValueError):
         CormOracle(1, 1, 3, 2, 4, 8, 2, 1, 1.0)
