@@ -18,7 +18,8 @@
  *
  * The recent-w verdict rows of Algorithm 1 (a bool matrix [m, l]) are held here as one w-bit shift register per
  * key (REG_WORDS 32-bit words, w <= 256): bit b of a key's register is the verdict of the query b steps ago. A
- * literal bool-matrix version lives in alg1_literal.py and is tested equal to this one.
+ * second statement of the policy with another data structure (per key, the set of queries that found it
+ * important) lives in verdict_history.py and is tested equal to this one.
  *
  * Every function below is pinned by tests/test_oracle_pins.py (hand-worked cases, full attention at alpha=0,
  * brute force over subsets, closed forms, invariants); none is "parity unpinned".

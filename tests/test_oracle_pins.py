@@ -1,7 +1,7 @@
 """Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle itself.
 
-Hand-worked cases (tests/golden), full attention at alpha = 0 against a library softmax, agreement with the literal
-bool-matrix form of Algorithm 1, brute force over all subsets on tiny inputs, closed-form special cases and
+Hand-worked cases (tests/golden), full attention at alpha = 0 against a library softmax, agreement with the
+per-key verdict-history statement of the policy (oracle/verdict_history.py), brute force over all subsets on tiny inputs, closed-form special cases and
 per-step invariants. A dropped term, wrong sign/index or transposed operand in the oracle fails at least one.
 """
 import itertools
@@ -13,7 +13,7 @@ import pytest
 import torch
 
 from oracle import CormOracle
-from oracle.alg1_literal import LiteralUnit
+from oracle.verdict_history import HistoryUnit
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -115,8 +115,8 @@ def test_alpha_zero_is_full_attention(seed):
 
 
 @pytest.mark.parametrize("seed", range(40))
-def test_shift_register_equals_literal_algorithm(seed):
-    """C oracle (shift registers) against the literal bool-matrix routine on random tiny cases, prompt included."""
+def test_shift_register_equals_verdict_history(seed):
+    """C oracle (shift registers) against the per-key verdict histories on random tiny cases, prompt included."""
     rng = np.random.default_rng(1000 + seed)
     Hkv = int(rng.integers(1, 3))
     G = int(rng.integers(1, 4))
@@ -132,7 +132,7 @@ def test_shift_register_equals_literal_algorithm(seed):
     units = {}
     for b in range(B):
         for h in range(Hkv):
-            u = LiteralUnit(d, w, r, alpha)
+            u = HistoryUnit(d, w, r, alpha)
             u.compress_prompt(k[b, h, :lens[b]], v[b, h, :lens[b]], q[b, h * G:(h + 1) * G, :w])
             units[b, h] = u
     o.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], lens)
@@ -155,16 +155,16 @@ def test_shift_register_equals_literal_algorithm(seed):
 
 
 @pytest.mark.parametrize("seed", range(10))
-def test_wide_windows_equal_literal_algorithm(seed):
-    """Windows beyond 32 queries (the paper's experiments use up to 256): multi-word registers against the literal
-    bool-matrix routine, compared through the live lists and the age of each key's newest 'important' verdict."""
+def test_wide_windows_equal_verdict_history(seed):
+    """Windows beyond 32 queries (the paper's experiments use up to 256): multi-word registers against the per-key
+    verdict histories, compared through the live lists and the age of each key's newest 'important' verdict."""
     rng = np.random.default_rng(3000 + seed)
     G = int(rng.integers(1, 3))
     d, w, r = 3, int(rng.choice([33, 40, 64, 65, 100])), int(rng.integers(1, 20))
     P, steps = int(rng.integers(0, 150)), int(rng.integers(40, 90))
     k, v, q, _ = _random_case(rng, 1, G, 1, d, P, steps, w, scale=2.5)
     o = CormOracle(1, 1, G, 1, d, P + steps, w, r, 1.0)
-    u = LiteralUnit(d, w, r, 1.0)
+    u = HistoryUnit(d, w, r, 1.0)
     u.compress_prompt(k[0, 0, :P], v[0, 0, :P], q[0, :, :w])
     o.compress_prompt(0, k[:, :, :P], v[:, :, :P], q[:, :, :w], [P])
     evicted = False
