@@ -71,10 +71,18 @@ typedef struct {
     int64_t kv_bytes_live, aux_bytes_live;           /* K+V bytes; register + position bytes */
     int64_t moved_rows;                              /* rows copied by hole-filling compaction so far */
     int64_t attended_keys;                           /* sum over decode steps and units of the live length read */
-    int32_t device_status;                           /* first device-side error (corm_status_t), CORM_OK if none */
+    int32_t device_status;                           /* most severe device-side error so far (the largest
+                                                        corm_status_t code reported), CORM_OK if none. Sticky: once it
+                                                        is non-zero, reset the cache (corm_cache_reset) and run the
+                                                        prompt pass again before trusting any unit */
     int64_t important_keys;                          /* sum over decode steps and units of the keys judged important
                                                         (Definition 3.1, OR over the group): important_keys /
                                                         attended_keys is the sparsity figure of Section 3.1 */
+    int64_t near_threshold;                          /* verdicts (Definition 3.1) whose reduced-precision logit fell
+                                                        inside the proven error bound around its threshold and was
+                                                        formed again in fp64 before it was decided: only the tiled
+                                                        prompt pass places logits in fp32; decode logits are fp64
+                                                        throughout and add nothing here */
 } corm_stats_t;
 
 /* Bytes of device memory a cache with this configuration needs (host, pure). 0 if the configuration is invalid. */
@@ -196,7 +204,6 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
  * it has few; 2 / 3 = those kernels with the first / the second way always. Errors: INVALID_ARG. */
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
-/* Number of kernels this library has launched on behalf of `cache` since create. */
 /* Opt-in monitor of the method's premise (Sections 3.2-3.3: the current query resembles recent ones, which is what
  * lets recent verdicts stand in for future ones, and which the paper reports failing for some models): while
  * enabled, every decode step also forms Eq. 3's cosine similarity between each query head's query and that head's
@@ -213,6 +220,7 @@ corm_status_t corm_cache_similarity(corm_cache_t* cache, double* sum_host, int64
  * Errors: INVALID_ARG. */
 corm_status_t corm_cache_set_bound_scale(corm_cache_t* cache, double scale);
 
+/* Number of kernels this library has launched on behalf of `cache` since create. */
 int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
 
 const char* corm_status_string(corm_status_t status);

@@ -30,7 +30,7 @@ class CormStats(ctypes.Structure):
     _fields_ = [("live_keys", ctypes.c_int64), ("appended_keys", ctypes.c_int64), ("evicted_keys", ctypes.c_int64),
                 ("retention", ctypes.c_double), ("kv_bytes_live", ctypes.c_int64), ("aux_bytes_live", ctypes.c_int64),
                 ("moved_rows", ctypes.c_int64), ("attended_keys", ctypes.c_int64), ("device_status", ctypes.c_int32),
-                ("important_keys", ctypes.c_int64)]
+                ("important_keys", ctypes.c_int64), ("near_threshold", ctypes.c_int64)]
 
 
 class CormError(RuntimeError):
@@ -168,13 +168,19 @@ class CormCache:
             self.handle, layer, ptr(k_prompt), ptr(v_prompt), ptr(q_last), lens.ctypes.data, p_max,
             _stream_ptr(stream)))
 
-    def corm_decode_step(self, layer, q, k_new, v_new, out=None, stream=None):
-        # argument checks kept cheap: this call is on the per-token path and a launch is only a few microseconds
+    def _check_step_args(self, call, q, k_new, v_new, out):
+        # kept cheap: these calls are on the per-token path and a launch is only a few microseconds
         if q.shape != self._q_shape or k_new.shape != self._kv_shape or v_new.shape != self._kv_shape:
-            raise ValueError("corm_decode_step: q / k_new / v_new have the wrong shape")
+            raise ValueError(f"{call}: q / k_new / v_new have the wrong shape")
         if not (q.dtype == k_new.dtype == v_new.dtype == self.dtype and q.is_cuda and k_new.is_cuda and v_new.is_cuda
                 and q.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()):
-            raise ValueError("corm_decode_step: inputs must be contiguous device tensors of the cache dtype")
+            raise ValueError(f"{call}: inputs must be contiguous device tensors of the cache dtype")
+        if out is not None and not (out.shape == self._q_shape and out.dtype == self.dtype and out.is_cuda
+                                    and out.is_contiguous()):
+            raise ValueError(f"{call}: out must be a contiguous device tensor shaped like q")
+
+    def corm_decode_step(self, layer, q, k_new, v_new, out=None, stream=None):
+        self._check_step_args("corm_decode_step", q, k_new, v_new, out)
         if out is None:
             out = torch.empty_like(q)
         rc = self.lib.corm_decode_step(self.handle, layer, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
@@ -187,6 +193,7 @@ class CormCache:
         """corm_decode_step for callers that must not allocate: the step's scratch sits in an array built into the
         library (16 MiB, shared by every cache on the device) instead of the arena. Pass ``out`` to keep this
         wrapper allocation-free as well; calls that overlap on the GPU race on the shared array."""
+        self._check_step_args("corm_decode_step_static", q, k_new, v_new, out)
         if out is None:
             out = torch.empty_like(q)
         _check("corm_decode_step_static", self.lib.corm_decode_step_static(

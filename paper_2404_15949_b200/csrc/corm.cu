@@ -246,6 +246,30 @@ void schedule_live_readback(corm_cache* c, int layer, cudaStream_t st) {
     c->last_readback_step[layer] = c->steps[layer];
 }
 
+// Eq. 3 between this step's queries and the layer's previous decode queries (opt-in; one small launch), after any
+// of the decode entry points: the queries stored as "previous" are always those of the step before.
+corm_status_t monitor_similarity(corm_cache* c, int layer, const void* q, cudaStream_t st) {
+    if (!c->monitor_similarity) return CORM_OK;
+    const corm_config_t& cf = c->cfg;
+    const int n_heads = cf.batch * cf.n_q_heads;
+    const size_t qb = (size_t)n_heads * cf.head_dim * c->e;
+    double* sum = reinterpret_cast<double*>(c->arena + c->lay.sim_acc);
+    unsigned long long* cnt = reinterpret_cast<unsigned long long*>(c->arena + c->lay.sim_acc + 8);
+    corm_status_t rc = dispatch(c, [&](auto* tp, auto dd, auto) -> corm_status_t {
+        using T = std::remove_pointer_t<decltype(tp)>;
+        constexpr int DD = decltype(dd)::value;
+        query_similarity_kernel<T, DD><<<(n_heads + 3) / 4, 128, 0, st>>>(
+            reinterpret_cast<const T*>(q), reinterpret_cast<T*>(layer_ptr(c, c->lay.q_prev, qb, layer)),
+            c->have_q_prev[layer], n_heads, sum, cnt);
+        CORM_CUDA(cudaGetLastError());
+        return CORM_OK;
+    });
+    if (rc != CORM_OK) return rc;
+    c->have_q_prev[layer] = 1;
+    c->launches += 1;
+    return CORM_OK;
+}
+
 corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
                             cudaStream_t st) {
     poll_live_bound(c, layer);
@@ -310,25 +334,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
     if (c->steps[layer] - c->last_readback_step[layer] >= 8) schedule_live_readback(c, layer, st);
-    if (c->monitor_similarity) {
-        const int n_heads = cf.batch * cf.n_q_heads;
-        const size_t qb = (size_t)n_heads * D * c->e;
-        double* sum = reinterpret_cast<double*>(c->arena + c->lay.sim_acc);
-        unsigned long long* cnt = reinterpret_cast<unsigned long long*>(c->arena + c->lay.sim_acc + 8);
-        rc = dispatch(c, [&](auto* tp, auto dd, auto) -> corm_status_t {
-            using T = std::remove_pointer_t<decltype(tp)>;
-            constexpr int DD = decltype(dd)::value;
-            query_similarity_kernel<T, DD><<<(n_heads + 3) / 4, 128, 0, st>>>(
-                reinterpret_cast<const T*>(q), reinterpret_cast<T*>(layer_ptr(c, c->lay.q_prev, qb, layer)),
-                c->have_q_prev[layer], n_heads, sum, cnt);
-            CORM_CUDA(cudaGetLastError());
-            return CORM_OK;
-        });
-        if (rc != CORM_OK) return rc;
-        c->have_q_prev[layer] = 1;
-        c->launches += 1;
-    }
-    return CORM_OK;
+    return monitor_similarity(c, layer, q, st);
 }
 
 }  // namespace
@@ -584,11 +590,13 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 namespace {
 constexpr int kMaxDevices = 64;
 unsigned char* g_static_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_static_scratch_mu;                           // two host threads may make a device's first call together
 
 // The array's name is only a handle on the host; its device address must be asked for, once per device, with that
 // device current. The caller holds a DeviceGuard for `device`.
 corm_status_t static_scratch_address(int device, unsigned char** out) {
     if (device < 0 || device >= kMaxDevices) return CORM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mu);
     if (!g_static_scratch_ptr[device]) {
         void* ptr = nullptr;
         CORM_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
@@ -662,7 +670,7 @@ corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void
     c->parity[layer] ^= 1;
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
-    return CORM_OK;
+    return monitor_similarity(c, layer, q, st);
 }
 
 corm_status_t corm_cache_live_lens(corm_cache_t* c, int32_t layer, int32_t* live_host, void* stream) {
@@ -697,6 +705,7 @@ corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* st
         s.moved_rows += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_MOVED];
         s.attended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_ATTENDED];
         s.important_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_IMPORTANT];
+        s.near_threshold += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_NEAR];
     }
     s.retention = s.appended_keys ? (double)s.live_keys / (double)s.appended_keys : 1.0;
     s.kv_bytes_live = s.live_keys * 2 * c->cfg.head_dim * (int64_t)c->e;

@@ -230,7 +230,7 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
         }
     }
     __syncthreads();
-    if (misc->failed) { if (tid == 0) atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); return; }
+    if (misc->failed) { if (tid == 0) report_status(p.status, CORM_ERR_TIMEOUT); return; }
 
     // ---- B. thresholds: warp w takes the (segment, head) pairs w, w + NW, ... ----
     for (int task = warp; task < nseg * G; task += NW) {
@@ -434,7 +434,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
 
     // ---- set-up that reads nothing the previous step writes ----
     if (smem_addr(smem) & 1023u) {                          // never expected; reported instead of mis-reading tiles
-        if (tid == 0) atomicCAS(p.status, 0, (int)CORM_ERR_INTERNAL);
+        if (tid == 0) report_status(p.status, CORM_ERR_INTERNAL);
         return;
     }
     if (tid == 0) { prefetch_tensormap(&vmap); s_failed = 0; }
@@ -470,7 +470,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
         if (cached) s_L[v] = l;
         if (!l && blk == 0) {        // a full slab or an exhausted pool: reported, the unit is left as it is
             const int l_old = __ldcg(p.live_in + v);
-            atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY);
+            report_status(p.status, CORM_ERR_CAPACITY);
             p.live_out[v] = l_old;
             publish_live(p.maxlive, p.step + 1, l_old);
         }
@@ -559,7 +559,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
         auto tile_row0 = [&](const BalSeg& sg, int ti) -> long long {
             if (!PAGED) return (long long)sg.u * p.C + (long long)ti * kTileKeys;
             const int pg = __ldcg(p.page_table + (size_t)sg.u * p.pt_stride + ti);
-            if (pg <= 0 || pg > p.pool_pages) { atomicCAS(p.status, 0, (int)CORM_ERR_INTERNAL); return -1; }
+            if (pg <= 0 || pg > p.pool_pages) { report_status(p.status, CORM_ERR_INTERNAL); return -1; }
             return (long long)(pg - 1) * kPageKeys;
         };
         auto issue_k = [&](Cur c, int n) {                     // lane 0 only
@@ -795,7 +795,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
             if (lane == 0) atomicAdd(p.ticket + u, 1u);   // this warp's record and logits of the segment are stored
         }
         __syncthreads();
-        if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
+        if (failed) { report_status(p.status, CORM_ERR_TIMEOUT); s_failed = 1; }
         __syncthreads();
         if (s_failed) return;                   // a bounded wait expired: reported through the status word
         // ---- Algorithm 1 for the slots this block streamed; the ring is free now ----

@@ -46,7 +46,7 @@ constexpr double kDotErr = 16.0 / 16777216.0;
 __host__ __device__ constexpr double inv_root_dim(int D) { return D == 128 ? 0.088388347648318440550 : 0.125; }
 
 // Counters kept per layer in the arena (64-bit, updated with atomics by the finalize phase / the prompt pass).
-enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_IMPORTANT = 4, CNT_COUNT = 5 };
+enum { CNT_APPENDED = 0, CNT_EVICTED = 1, CNT_MOVED = 2, CNT_ATTENDED = 3, CNT_IMPORTANT = 4, CNT_NEAR = 5, CNT_COUNT = 6 };
 
 struct DecodeParams {
     void* K;                  // [U][C][D] this layer's key slabs
@@ -149,6 +149,11 @@ template <> __device__ __forceinline__ void load_slice<bf16_t, 2>(const bf16_t* 
     uint32_t v = *reinterpret_cast<const uint32_t*>(p);
     out[0] = __uint_as_float(v << 16); out[1] = __uint_as_float(v & 0xffff0000u);
 }
+
+// Device-side errors are sticky: the status word keeps the numerically largest code reported (a broken invariant
+// outranks an expired wait, which outranks a full slab), so that a later, harmless code cannot hide an earlier severe
+// one nor the other way round. After any non-zero status the cache must be reset before it is used again.
+__device__ __forceinline__ void report_status(int32_t* status, corm_status_t code) { atomicMax(status, (int32_t)code); }
 
 // Adds the warp's total of n to a 64-bit counter (one atomic per warp; all lanes must call).
 __device__ __forceinline__ void warp_count(unsigned long long* counter, int n) {

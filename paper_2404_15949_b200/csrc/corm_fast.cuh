@@ -297,7 +297,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     }
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C || !room) {
-        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
+        if (split == 0 && tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
     const int n_act = (l + p.split_len - 1) / p.split_len;
@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         const int kslot = it % kKStages, vslot = it % kVStages;
         unsigned char* ktile = my_tiles + kslot * kTileBytes;
         unsigned char* vtile = my_tiles + (kKStages + vslot) * kTileBytes;
-        if (!mbar_wait(my_bars + kslot * 8, (it / kKStages) & 1)) failed = true;
+        if (!failed && !mbar_wait(my_bars + kslot * 8, (it / kKStages) & 1)) failed = true;   // after one expired wait the rest are skipped
         if (has_new) {   // append: the new row goes to the slab and replaces whatever the copy fetched for that slot
             cp_async_wait_all();
             __syncwarp();
@@ -474,7 +474,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         }
         __syncwarp();
 
-        if (!mbar_wait(my_bars + (kKStages + vslot) * 8, (it / kVStages) & 1)) failed = true;
+        if (!failed && !mbar_wait(my_bars + (kKStages + vslot) * 8, (it / kVStages) & 1)) failed = true;
         if (has_new) {
             if (lane < 16) {
                 const uint4 x = *reinterpret_cast<const uint4*>(newrow + kRowBytes + lane * 16);
@@ -503,7 +503,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         __syncwarp();
         if (lane == 0 && it + kVStages < my_n) { fence_async_smem(); issue_v(it + kVStages); }
     }
-    if (failed) { atomicCAS(p.status, 0, (int)CORM_ERR_TIMEOUT); s_failed = 1; }
+    if (failed) { report_status(p.status, CORM_ERR_TIMEOUT); s_failed = 1; }
     // The verdict launch that may follow is allowed to become resident once every block of this grid is past its
     // tiles (it waits for this grid to complete before it reads anything written here). Allowing it from the top of
     // the kernel costs 1.4 us per step on 128 units of 1600 keys: its waiting blocks take room next to streaming ones.
@@ -520,7 +520,10 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
         for (int e = 0; e < 8; ++e) acc[g][e] += __shfl_xor_sync(0xffffffffu, acc[g][e], 16);
     }
     __syncthreads();                       // every warp is done with its tiles: the tile area becomes scratch
-    if (s_failed) return;                  // a bounded wait expired: reported through the status word, unit left as is
+    if (s_failed) {                        // a bounded wait expired: reported through the status word; the unit keeps its
+        if (split == 0 && tid == 0) { p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }   // old length
+        return;                            // (its arrival counter is not taken: the cache must be reset after this status)
+    }
     unsigned char* merge = smem + lay.tiles;                      // [NW][G] records {double M, double Z, float acc[128]}
     constexpr int kRec = 16 + 4 * 128;
 #pragma unroll

@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     const int room = pt_u ? __ldcg(p.page_room + u) : 1;
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C || !room) {   // the slab is full (paged: no page for the new row): report, leave the unit untouched
-        if (split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
+        if (split == 0 && tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
         return;
     }
     const int n_act = (l + p.split_len - 1) / p.split_len;
@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     const int b = u / p.Hkv;
     const int P = __ldg(p.prompt_lens + b);
     if (P > p.C) {
-        if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
+        if (tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = 0; }
         return;
     }
     if (P == 0) {
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
     const int kept_total = prefix[nwords];
     const int32_t* pt_u = p.page_table ? p.page_table + (size_t)u * p.pt_stride : nullptr;
     if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, kept_total)) {
-        if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }   // the pool is too small
+        if (tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = 0; }   // the pool is too small
         return;
     }
     T* Kl = reinterpret_cast<T*>(p.K);

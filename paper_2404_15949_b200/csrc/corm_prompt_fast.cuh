@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     const int b = u / p.Hkv, P = __ldg(p.prompt_lens + b), w = p.w, wp = min(P, w);
     const bool last_launch = fp.slot1 == w;
     if (P > p.C) {
-        if (last_launch && split == 0 && tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; }
+        if (last_launch && split == 0 && tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = 0; }
         return;
     }
     if (P == 0) {
@@ -315,6 +315,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
         // verdicts of this launch's queries for the lane's key: a bit per window slot (bit w-1-rho) when the window
         // fits a shift register, else the position of the newest query that found the key important
         uint32_t reg = 0u;
+        int n_near = 0;                                   // logits inside the fp32 bound, placed again in fp64
         for (int gi = 0; gi < groups; ++gi) {
             if (slot0 + (4 * gi + 3) / G < w - wp) continue;                      // none of these queries exists
             // The thresholds are exact (fp64, from the first launch), so a logit only has to be placed on one side of
@@ -333,8 +334,10 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
                 if (exists && pos_own <= qpos) {
                     const double margin = (double)s32[x] * inv_root_d - thr_sm[r], err = err_sm[r] * kn;
                     if (margin >= err) imp = true;
-                    else if (!(margin < -err))
+                    else if (!(margin < -err)) {
                         imp = exact_logit(q_sm + (size_t)r * 128, Kp + (size_t)(k0 + key_own) * kRowBytes) * inv_root_d >= thr_sm[r];
+                        ++n_near;
+                    }
                 }
                 // Definition 3.1 in log form; keys newer than the query keep a 0 bit (Algorithm 1's zero padding)
                 if (imp) {
@@ -343,6 +346,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
                 }
             }
         }
+        warp_count(p.counters + CNT_NEAR, n_near);
         if (key_own < n_valid) {
             uint32_t* dst = tmp_word + k0 + key_own;
             if (slot0 == 0) *dst = reg;                                            // first launch of the window
@@ -376,7 +380,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
     const int kept_total = prefix[nwords];
     const bool paged = p.page_table != nullptr;
     if (!claim_unit_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, kept_total, pt_sm)) {
-        if (tid == 0) { atomicCAS(p.status, 0, (int)CORM_ERR_CAPACITY); p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); }
+        if (tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = 0; publish_live(p.maxlive, 0, 0); }
         return;                                                                       // the pool is too small
     }
     unsigned char* Kl = reinterpret_cast<unsigned char*>(p.K);

@@ -1,14 +1,23 @@
-"""Parity at the benchmark's full sizes and in its launch configuration (automatic tuning, fast path on).
+"""Parity at the benchmark's full sizes and in its launch configuration (automatic tuning, fast path on), over
+the configurations' whole horizons.
 
-The CUDA library steps the whole configuration; the CPU oracle steps a sample of its units (they are independent, and
-the generator yields identical slices for any subset), free-running from the prompt pass with no resynchronisation.
-Outputs of the sampled units must agree within the cache dtype's tolerance and their registers, positions and rows
-must be bit-exact after every checked step. The oracle's count of probabilities within 1e-6 (relative) of the
-threshold is zero on the samples fixed here, except for the 32k-token configuration where ~4e6 evaluations per
-sample make a handful statistically certain; there the count is printed and parity is still required in full.
+The CUDA library steps the whole configuration for every decode step it defines (256 / 512 / 256 / 1024); the CPU
+oracle steps a sample of its units (they are independent, and the generator yields identical slices for any subset),
+free-running from the prompt pass with no resynchronisation. Outputs of the sampled units must agree within the
+cache dtype's tolerance at every step; registers, positions and rows must be bit-exact every 32 steps and at the
+end, with the library enqueued far ahead of the host in between, as in the benchmark. That reaches the launch shapes
+the benchmark spends its time in: one block per unit on the batch-32 workload, the balanced kernel on the grouped
+one, planted-key drift and continuous compaction on the long-context one.
+
+The oracle's count of probabilities within 1e-6 (relative) of the threshold is zero on the samples fixed here
+(chosen by scanning candidate units with the oracle alone) and asserted so, except for the 32k-token configuration:
+there one unit makes 5e7 evaluations over its horizon, 2e6 in the prompt pass alone, at about one in-band evaluation
+per 1.3e6, so no sample of it is free of them; the count is printed and parity is required in full, in-band keys
+included.
 """
 import numpy as np
 import pytest
+import torch
 
 from paper_2404_15949_b200.workload import CONFIGS, generate
 from parity_util import OUT_TOL, make_oracle, sorted_state, to_dev
@@ -16,19 +25,21 @@ from parity_util import OUT_TOL, make_oracle, sorted_state, to_dev
 pytestmark = pytest.mark.gpu
 
 CASES = [
-    # config, layers sampled, sequences sampled, kv heads sampled (per layer), steps, expect zero near-threshold
-    (3, [0], [0, 17], {0: [3, 20]}, 48, True),
-    (4, [0], [1], {0: [4, 7]}, 32, True),
-    (2, [0, 5], [0], {0: [0, 9], 5: [1, 8]}, 32, True),
-    (5, [0], [0], {0: [0]}, 16, False),
+    # config, layers sampled, sequences sampled, kv heads sampled (per layer), expect zero near-threshold
+    (3, [0], [0, 17], {0: [3, 9]}, True),
+    (4, [0], [1, 5], {0: [4, 5]}, True),
+    (2, [0, 5, 31], [0], {0: [0, 9], 5: [1, 8], 31: [0, 3]}, True),
+    (5, [0], [0], {0: [0]}, False),
 ]
+CHECK_EVERY = 32
 
 
 @pytest.mark.parametrize("case", CASES, ids=lambda c: f"config{c[0]}")
 def test_full_size_sampled_units(case):
     from paper_2404_15949_b200.binding import CormCache
-    which, layers, seqs, heads_by_layer, steps, expect_zero_near = case
+    which, layers, seqs, heads_by_layer, expect_zero_near = case
     cfg = CONFIGS[which]
+    steps = cfg.steps
     G, dt = cfg.group, cfg.dtype
     gpu = CormCache(cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.max_tokens,
                     cfg.window_w, cfg.recent_r, cfg.alpha, dt, 0)           # default tuning = what bench.py times
@@ -59,19 +70,25 @@ def test_full_size_sampled_units(case):
 
     check_states("after prompt")
     worst = 0.0
-    for s in range(steps):
+    dev_in = {l: tuple(to_dev(a, dt) for a in (full[l].q, full[l].k_new, full[l].v_new)) for l in layers}
+    for s0 in range(0, steps, CHECK_EVERY):
+        chunk = range(s0, min(steps, s0 + CHECK_EVERY))
+        outs = {l: [] for l in layers}
+        for s in chunk:                                        # the library runs ahead of the host for a whole chunk
+            for l in layers:
+                qd, kd, vd = dev_in[l]
+                outs[l].append(gpu.corm_decode_step(l, qd[s], kd[s], vd[s]))
         for l in layers:
             orc, sub, heads = oracles[l]
-            out = gpu.corm_decode_step(l, to_dev(full[l].q[s], dt), to_dev(full[l].k_new[s], dt),
-                                       to_dev(full[l].v_new[s], dt)).float().cpu().numpy()
-            ref = orc.decode_step(0, sub.q[s], sub.k_new[s], sub.v_new[s])
-            for ib, b in enumerate(seqs):
-                for ih, h in enumerate(heads):
-                    err = np.abs(out[b, h * G:(h + 1) * G] - ref[ib, ih * G:(ih + 1) * G]).max()
-                    worst = max(worst, float(err))
-                    assert err <= OUT_TOL[dt], (s, l, b, h, err)
-        if s % 8 == 7 or s == steps - 1:
-            check_states(f"after step {s}")
+            got = torch.stack(outs[l]).float().cpu().numpy()
+            for i, s in enumerate(chunk):
+                ref = orc.decode_step(0, sub.q[s], sub.k_new[s], sub.v_new[s])
+                for ib, b in enumerate(seqs):
+                    for ih, h in enumerate(heads):
+                        err = np.abs(got[i, b, h * G:(h + 1) * G] - ref[ib, ih * G:(ih + 1) * G]).max()
+                        worst = max(worst, float(err))
+                        assert err <= OUT_TOL[dt], (s, l, b, h, err)
+        check_states(f"after step {chunk[-1]}")
     near = sum(o[0].counters()["near_threshold"] for o in oracles.values())
     print(f"config {which}: max |out - oracle| = {worst:.2e}, near-threshold evaluations in the sample = {near}")
     if expect_zero_near:

@@ -59,6 +59,38 @@ def test_static_scratch_entry_point_matches_on_consecutive_calls():
     assert A[2].corm_cache_stats()["evicted_keys"] == A[1].corm_cache_stats()["evicted_keys"] > 0
 
 
+def test_static_scratch_steps_against_the_oracle_without_allocating():
+    """The entry point against the CPU oracle directly (outputs within tolerance, state bit-exact), and the property
+    it exists for: with `out` supplied, a call makes no request to torch's allocator and takes no memory from the
+    device (one warm-up call first: it looks up the built-in array's address and loads the kernel)."""
+    from parity_util import assert_states_equal, make_oracle
+    cfg = CONFIGS[4].with_(batch=2, n_q_heads=8, n_kv_heads=2, prompt_min=300, prompt_max=420, steps=16, recent_r=32,
+                           seed=777)
+    data = generate(cfg)
+    nb, nh, dt = len(data.seqs), len(data.kv_heads), cfg.dtype
+    gpu, orc = make_gpu_cache(cfg, nb, nh), make_oracle(cfg, nb, nh)
+    gpu.corm_compress_prompt(0, to_dev(data.k_prompt, dt), to_dev(data.v_prompt, dt), to_dev(data.q_last, dt),
+                             data.prompt_lens)
+    orc.compress_prompt(0, data.k_prompt, data.v_prompt, data.q_last, data.prompt_lens)
+    q, k, v = to_dev(data.q, dt), to_dev(data.k_new, dt), to_dev(data.v_new, dt)
+    out = torch.empty_like(q[0])
+    for s in range(cfg.steps):
+        if s >= 1:
+            torch.cuda.synchronize()
+            n_allocs, free = torch.cuda.memory_stats()["allocation.all.allocated"], torch.cuda.mem_get_info()[0]
+        gpu.corm_decode_step_static(0, q[s], k[s], v[s], out)
+        if s >= 1:
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_stats()["allocation.all.allocated"] == n_allocs, f"step {s}: torch allocated"
+            assert torch.cuda.mem_get_info()[0] >= free, f"step {s}: device memory was taken"
+        ref = orc.decode_step(0, data.q[s], data.k_new[s], data.v_new[s])
+        assert np.abs(out.float().cpu().numpy() - ref).max() <= OUT_TOL[dt], f"step {s}"
+        if s % 4 == 3 or s == cfg.steps - 1:
+            assert_states_equal(gpu, orc, 0, nb, nh, f"after step {s}")
+    assert orc.counters()["near_threshold"] == 0 and orc.counters()["evicted"] > 0
+    assert gpu.corm_cache_stats()["device_status"] == 0
+
+
 def test_static_scratch_rejects_oversized_caches():
     from paper_2404_15949_b200.binding import CormError
     cfg = CONFIGS[3].with_(batch=8, prompt_min=64, prompt_max=64, steps=4)                   # 256 units x 4608 slots
