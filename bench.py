@@ -4,7 +4,10 @@
 A "step" is one decode step of the whole batch through every layer of the configuration (one layer for the default
 workload): append, attention over every unit's live keys, verdicts, register update and compaction, one kernel
 launch per layer. Default workload: the batched-throughput
-configuration (batch 32, 32 heads, head_dim 128, bf16, ragged prompts in [2048, 4096]).
+configuration (batch 32, 32 heads, head_dim 128, bf16, ragged prompts in [2048, 4096]); the grouped-query workload is
+measured as well and reported under `also`. Every workload is timed `--repeats` times over the same decode steps,
+each pass from the restored post-prompt state, and the median pass is reported; the end-to-end figure (host buffers
+through corm_decode_step_host) runs over the same steps from the same state.
 
     python bench.py --gpus 1 --steps 256 --warmup 16
     python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...   (independent shards)
@@ -30,12 +33,9 @@ from paper_2404_15949_b200.workload import CONFIGS, generate  # noqa: E402
 METRIC = "corm_decode_step_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per algorithmic byte of the decode kernel, from the ncu capture summarised in
-# profiles/decode_fast_kernel_batch32_bf16.md (243.0 and 240.3 MB moved for 237.4 MB algorithmic at the two captured
-# steps). Set to None whenever the kernel changes until the counters are taken again.
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE = {"batch32_bf16": 1.018}
-# the same for the kernel's paged instance (--pool-pages; 241.5 and 241.0 MB moved for 237.4 MB, same file)
-DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE_PAGED = {"batch32_bf16": 1.016}
+# DRAM traffic of the dominant kernel per launch as ncu counted it, keyed by workload name; None until the counters are
+# taken on the kernel as it stands now (a figure from an older kernel or another launch shape would mislead).
+DRAM_TRAFFIC_BYTES_PER_LAUNCH = {}
 
 
 def log(*a):
@@ -143,61 +143,28 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(cfg, args):
-    return {"workload": f"{cfg.name} (workload {args.workload} of 5, configs[{args.workload - 1}])", "batch": cfg.batch,
+def workload_config(cfg, args, which=None):
+    which = args.workload if which is None else which
+    return {"workload": f"{cfg.name} (workload {which} of 5, configs[{which - 1}])", "batch": cfg.batch,
             "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
             "prompt_len": [cfg.prompt_min, cfg.prompt_max], "window_w": cfg.window_w, "recent_r": cfg.recent_r,
             "alpha": cfg.alpha, "layers_per_step": cfg.n_layers, "seed": cfg.seed,
             "l2": "live K/V read per step exceeds the 126 MB L2 (no flush needed)"}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=256)
-    ap.add_argument("--warmup", type=int, default=16)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
-    ap.add_argument("--e2e-steps", type=int, default=64)
-    ap.add_argument("--ref-seqs", type=int, default=32)
-    ap.add_argument("--ref-steps", type=int, default=512)
-    ap.add_argument("--split-len", type=int, default=0)
-    ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced"],
-                    help="who finishes units of several splits: the decode launch itself or the verdict launch")
-    ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--window", type=int, default=None, help="override the verdict window w (1..256)")
-    ap.add_argument("--recent", type=int, default=None, help="override the protected recent tokens r")
-    ap.add_argument("--pool-pages", type=int, default=0,
-                    help="paged cache with this many 32-key pages per layer (multiple of 32); 0 = one slab per unit")
-    args = ap.parse_args()
-    cfg = CONFIGS[args.workload]
-    if args.alpha is not None:
-        cfg = cfg.with_(alpha=args.alpha, name=cfg.name + f"_alpha{args.alpha:g}")
-    if args.window is not None:
-        cfg = cfg.with_(window_w=args.window, name=cfg.name + f"_w{args.window}")
-    if args.recent is not None:
-        cfg = cfg.with_(recent_r=args.recent, name=cfg.name + f"_r{args.recent}")
-    if args.impl == "reference":
-        return run_reference(args, cfg)
-
+def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
+    """Prompt pass, then `repeats` timed passes over the same decode steps, each from the restored post-prompt state
+    (the prompt pass is run again and the warm-up replayed), and an end-to-end pass over the same steps through the
+    host-buffer entry point. Returns a dict of this rank's and the job's figures."""
     import torch
     import torch.distributed as dist
     from paper_2404_15949_b200.binding import CormCache
-
-    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device; the CORM path has no CPU fallback"
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    # each rank owns an independent shard (its own batch, its own arena): no data-path collective
     from paper_2404_15949_b200.sharding import aggregate_throughput, shard_config
-    cfg_r = shard_config(cfg, rank, world)
-    n_steps = args.warmup + args.steps + args.e2e_steps
+
+    cfg_r = shard_config(cfg, rank, world)              # each rank owns an independent shard: no data-path collective
+    n_steps = args.warmup + args.steps
     cfg_r = cfg_r.with_(steps=max(cfg.steps, n_steps))
-    L = cfg.n_layers                     # a step = one token through every layer of the configuration
+    L = cfg.n_layers                                    # a step = one token through every layer of the configuration
     t0 = time.perf_counter()
     data = [generate(cfg_r, layer=l, n_steps=n_steps) for l in range(L)]
     log(f"[rank {rank}] generated {cfg.name} inputs ({L} layer(s)) in {time.perf_counter() - t0:.1f} s")
@@ -208,123 +175,219 @@ def main():
     cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4}[args.finish])
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
-    prompt_ms = 0.0
-    for l in range(L):
-        kp, vp, ql = dev(data[l].k_prompt), dev(data[l].v_prompt), dev(data[l].q_last)
-        cache.corm_compress_prompt(l, kp, vp, ql, data[l].prompt_lens)     # untimed: first launch loads the kernels
-        torch.cuda.synchronize()
-        a.record()
-        cache.corm_compress_prompt(l, kp, vp, ql, data[l].prompt_lens)     # same inputs, same resulting state
-        b.record()
-        torch.cuda.synchronize()
-        prompt_ms += a.elapsed_time(b)
-        del kp, vp, ql
-    st0 = cache.corm_cache_stats()
+    prompts = [(dev(d.k_prompt), dev(d.v_prompt), dev(d.q_last), d.prompt_lens) for d in data]
     q_d = [dev(d.q) for d in data]
     k_d = [dev(d.k_new) for d in data]
     v_d = [dev(d.v_new) for d in data]
     out = torch.empty_like(q_d[0][0])
-
     # per-step views made once: slicing a tensor costs the host several microseconds, as much as a launch
-    views = [[(q_d[l][s], k_d[l][s], v_d[l][s]) for l in range(L)] for s in range(args.warmup + args.steps)]
+    views = [[(q_d[l][s], k_d[l][s], v_d[l][s]) for l in range(L)] for s in range(n_steps)]
+
+    def restore():
+        """Back to the state right after the prompt pass. Returns the pass's device time (ms)."""
+        torch.cuda.synchronize()
+        a.record()
+        for l in range(L):
+            cache.corm_compress_prompt(l, *prompts[l])
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
 
     def step(s):
         for l in range(L):
             qv, kv, vv = views[s][l]
             cache.corm_decode_step(l, qv, kv, vv, out)
 
-    for s in range(args.warmup):
-        step(s)
-    torch.cuda.synchronize()
-    st1 = cache.corm_cache_stats()
-    launches0 = cache.corm_cache_kernel_launches()
-    sampler = ClockSampler(local)
-    sampler.start()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    a.record()
-    t_issue = time.perf_counter()
-    for s in range(args.warmup, args.warmup + args.steps):
-        step(s)
-    b.record()
-    issue_ms = 1e3 * (time.perf_counter() - t_issue)     # host time to enqueue the timed steps (GPU time hides behind it if larger)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    sampler.stop_flag = True
-    sampler.join()
-    ms = a.elapsed_time(b)
-    launches = cache.corm_cache_kernel_launches() - launches0
-    st2 = cache.corm_cache_stats()
+    restore()                                            # untimed: the first launches load the kernels
+    passes, prompt_ms, sampler = [], 0.0, None
+    for rep in range(args.repeats):
+        prompt_ms = restore()
+        st0 = cache.corm_cache_stats()
+        for s in range(args.warmup):
+            step(s)
+        torch.cuda.synchronize()
+        st1 = cache.corm_cache_stats()
+        launches0 = cache.corm_cache_kernel_launches()
+        if want_clocks and rep == 0:
+            sampler = ClockSampler(local)
+            sampler.start()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        a.record()
+        t_issue = time.perf_counter()
+        for s in range(args.warmup, n_steps):
+            step(s)
+        b.record()
+        issue_ms = 1e3 * (time.perf_counter() - t_issue)  # host time to enqueue the timed steps
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        st2 = cache.corm_cache_stats()
+        passes.append(dict(ms=a.elapsed_time(b), issue_ms=issue_ms, st0=st0, st1=st1, st2=st2,
+                           launches=cache.corm_cache_kernel_launches() - launches0))
+    passes_sorted = sorted(passes, key=lambda x: x["ms"])
+    med = passes_sorted[len(passes_sorted) // 2]
 
-    # end to end through the host-buffer entry point: pinned inputs copied in and the output read back every step
+    # end to end through the host-buffer entry point, over the SAME steps from the same restored state: pinned inputs
+    # read and the output written across the bus every step
     e2e_ms, h2d, d2h = None, 0, 0
-    if args.e2e_steps:
-        base = args.warmup + args.steps
+    if want_e2e:
         pin = lambda t: t.cpu().pin_memory()
-        qh = [pin(x[base:]) for x in q_d]
-        kh = [pin(x[base:]) for x in k_d]
-        vh = [pin(x[base:]) for x in v_d]
+        qh = [pin(x) for x in q_d]
+        kh = [pin(x) for x in k_d]
+        vh = [pin(x) for x in v_d]
         oh = torch.empty_like(qh[0][0]).pin_memory()
         h2d = L * (qh[0][0].numel() + 2 * kh[0][0].numel()) * oh.element_size()
         d2h = L * oh.numel() * oh.element_size()
+        hviews = [[(qh[l][s], kh[l][s], vh[l][s]) for l in range(L)] for s in range(n_steps)]
+        restore()
+        for s in range(args.warmup):
+            for l in range(L):
+                cache.corm_decode_step_host(l, *hviews[s][l], oh)
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         a.record()
-        for s in range(args.e2e_steps):
+        for s in range(args.warmup, n_steps):
             for l in range(L):
-                cache.corm_decode_step_host(l, qh[l][s], kh[l][s], vh[l][s], oh)
+                cache.corm_decode_step_host(l, *hviews[s][l], oh)
         b.record()
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(b)
+    if sampler is not None:
+        sampler.stop_flag = True
+        sampler.join()
     st3 = cache.corm_cache_stats()
     assert st3["device_status"] == 0, f"device status {st3['device_status']}"
 
-    value, ms_max, _ = aggregate_throughput(ms, cfg.batch * args.steps, "cuda")
-    e2e_value = aggregate_throughput(e2e_ms, cfg.batch * args.e2e_steps, "cuda")[0] if e2e_ms else None
+    value, ms_max, _ = aggregate_throughput(med["ms"], cfg.batch * args.steps, "cuda")
+    e2e_value = aggregate_throughput(e2e_ms, cfg.batch * args.steps, "cuda")[0] if e2e_ms else None
+    unit_steps = L * cfg.batch * cfg.n_kv_heads * args.steps
+    attended = med["st2"]["attended_keys"] - med["st1"]["attended_keys"]
+    moved = med["st2"]["moved_rows"] - med["st1"]["moved_rows"]
+    abytes = algorithmic_bytes(cfg, attended, moved, unit_steps)
+    peak, peak_src = measured_peak()
+    achieved = abytes / (med["ms"] * 1e-3) / 1e9
+    launches_per_step = med["launches"] / (args.steps * L)
+    traffic = DRAM_TRAFFIC_BYTES_PER_LAUNCH.get(cfg.name)
+    res = {
+        "value": value, "ms_per_step": ms_max / args.steps,
+        "repeats": {"n": len(passes), "ms_per_step": [x["ms"] / args.steps for x in passes],
+                    "spread": (passes_sorted[-1]["ms"] - passes_sorted[0]["ms"]) / med["ms"],
+                    "reported": "median pass; every pass starts from the restored post-prompt state"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src, "traffic": traffic,
+                     "traffic_note": None if traffic else "no ncu capture of the kernel as it stands at this launch shape",
+                     "target": {"frac_of_nominal_8TBs": 0.60, "met": achieved / 8000.0 >= 0.60},
+                     "kernel": ("decode_balanced_kernel" if launches_per_step < 1.5 and cfg.group > 1 and args.finish in ("auto", "balanced")
+                                else "decode_fast_kernel") + f" ({launches_per_step:.2f} launches per layer per step, all counted in the time)",
+                     "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * med["ms"] / (args.steps * L)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": "the same decode steps as `value`, from the same restored state"},
+        "gpu_launches": med["launches"], "host_issue_us_per_step": 1e3 * med["issue_ms"] / args.steps,
+        "retention": med["st2"]["retention"],
+        "live_keys_per_unit": med["st2"]["live_keys"] / (L * cfg.batch * cfg.n_kv_heads),
+        "evicted_keys_timed": med["st2"]["evicted_keys"] - med["st1"]["evicted_keys"], "moved_rows_timed": moved,
+        "important_key_fraction_timed": (med["st2"]["important_keys"] - med["st1"]["important_keys"]) / max(1, attended),
+        "prompt_pass_ms": prompt_ms, "retention_after_prompt": med["st0"]["retention"],
+        "near_threshold_prompt_pass": med["st0"]["near_threshold"],
+        "arena_bytes": int(cache.arena.numel()),
+    }
+    if sampler is not None:
+        res["clocks"] = sampler.result()
+    if args.pool_pages:
+        res["pool_pages_in_use"] = sum(cache.corm_cache_pool_usage(l)[0] for l in range(L))
+        # the paper's own metric, made physical: K+V bytes of the pages held against K+V bytes of every token seen
+        row = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4)
+        res["kv_bytes_held"] = res["pool_pages_in_use"] * 32 * row
+        res["kv_bytes_full_cache"] = st3["appended_keys"] * row
+        res["kv_memory_reduction"] = 1.0 - res["kv_bytes_held"] / max(1, res["kv_bytes_full_cache"])
+    cache.close()
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--repeats", type=int, default=3, help="timed passes over the same steps; the median is reported")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end pass through the host-buffer entry point")
+    ap.add_argument("--e2e-steps", type=int, default=None, help="0 skips the end-to-end pass (same as --no-e2e)")
+    ap.add_argument("--also", default="4", help="comma-separated workloads measured as well and reported under `also` "
+                                                "(default: the grouped-query target workload); empty = none")
+    ap.add_argument("--ref-seqs", type=int, default=32)
+    ap.add_argument("--ref-steps", type=int, default=512)
+    ap.add_argument("--split-len", type=int, default=0)
+    ap.add_argument("--no-fast", action="store_true")
+    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced"],
+                    help="which decode kernels: automatic, the block-per-split kernels finishing long units inside the "
+                         "decode launch / by the verdict launch, or the balanced single-launch kernel")
+    ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--window", type=int, default=None, help="override the verdict window w (1..256)")
+    ap.add_argument("--recent", type=int, default=None, help="override the protected recent tokens r")
+    ap.add_argument("--pool-pages", type=int, default=0,
+                    help="paged cache with this many 32-key pages per layer (multiple of 32); 0 = one slab per unit")
+    args = ap.parse_args()
+
+    def configured(which):
+        cfg = CONFIGS[which]
+        if args.alpha is not None:
+            cfg = cfg.with_(alpha=args.alpha, name=cfg.name + f"_alpha{args.alpha:g}")
+        if args.window is not None:
+            cfg = cfg.with_(window_w=args.window, name=cfg.name + f"_w{args.window}")
+        if args.recent is not None:
+            cfg = cfg.with_(recent_r=args.recent, name=cfg.name + f"_r{args.recent}")
+        return cfg
+
+    cfg = configured(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, cfg)
+
+    import torch
+    import torch.distributed as dist
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; the CORM path has no CPU fallback"
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    want_e2e = not args.no_e2e and args.e2e_steps != 0
+    main_res = measure_workload(cfg, args, local, world, rank, want_e2e, True)
+    also = []
+    for w in [int(x) for x in args.also.split(",") if x.strip()]:
+        if w == args.workload:
+            continue
+        cfg_w = configured(w)
+        saved = args.steps
+        args.steps = min(args.steps, cfg_w.steps - args.warmup) if cfg_w.steps > args.warmup else args.steps
+        r = measure_workload(cfg_w, args, local, world, rank, False, False)
+        keep = ("value", "ms_per_step", "repeats", "roofline", "gpu_launches", "host_issue_us_per_step", "retention",
+                "live_keys_per_unit", "prompt_pass_ms")
+        also.append(dict({"config": workload_config(cfg_w, args, w), "steps": args.steps, "unit": UNIT},
+                         **{k: r[k] for k in keep}))
+        args.steps = saved
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-    unit_steps = L * cfg.batch * cfg.n_kv_heads * args.steps
-    attended = st2["attended_keys"] - st1["attended_keys"]
-    moved = st2["moved_rows"] - st1["moved_rows"]
-    abytes = algorithmic_bytes(cfg, attended, moved, unit_steps)
-    peak, peak_src = measured_peak()
-    achieved = abytes / (ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64 logits / f32 accumulation over " + cfg.dtype + " cache", "data": "synthetic",
-        "config": workload_config(cfg, args),
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "peak_source": peak_src,
-                     "traffic": ((DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE_PAGED if args.pool_pages else DRAM_TRAFFIC_PER_ALGORITHMIC_BYTE)
-                                 .get(cfg.name) or 0) * abytes / (args.steps * L) or None,
-                     "kernel": "decode_fast_kernel (one launch per layer per step; early steps with units longer than one block add a verdict launch, counted in the time)",
-                     "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * ms / (args.steps * L)},
-        "e2e": {"value": e2e_value, "unit": UNIT,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches, "host_issue_us_per_step": 1e3 * issue_ms / args.steps,
-        "clocks": sampler.result(),
-        "retention": st2["retention"],
-        "live_keys_per_unit": st2["live_keys"] / (L * cfg.batch * cfg.n_kv_heads),
-        "evicted_keys_timed": st2["evicted_keys"] - st1["evicted_keys"], "moved_rows_timed": moved,
-        "important_key_fraction_timed": (st2["important_keys"] - st1["important_keys"]) / max(1, attended),
-        "prompt_pass_ms": prompt_ms, "retention_after_prompt": st0["retention"],
-        "paper_context": "paper reports KV memory only: up to 70% reduction (V100-32GB / A100-80GB), no throughput",
+        "metric": METRIC, "value": main_res.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": main_res.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64 logits / f32 accumulation over " + cfg.dtype + " cache", "data": "synthetic",
+        "config": workload_config(cfg, args, args.workload),
     }
-    line["arena_bytes"] = int(cache.arena.numel())
+    line.update(main_res)
+    line["paper_context"] = "paper reports KV memory only: up to 70% reduction (V100-32GB / A100-80GB), no throughput"
     if args.pool_pages:
         line["config"]["pool_pages"] = args.pool_pages
-        line["pool_pages_in_use"] = sum(cache.corm_cache_pool_usage(l)[0] for l in range(L))
-        # the paper's own metric, made physical: K+V bytes of the pages held against K+V bytes of every token seen
-        row = 2 * cfg.head_dim * (2 if cfg.dtype == "bf16" else 4)
-        line["kv_bytes_held"] = line["pool_pages_in_use"] * 32 * row
-        line["kv_bytes_full_cache"] = st3["appended_keys"] * row
-        line["kv_memory_reduction"] = 1.0 - line["kv_bytes_held"] / max(1, line["kv_bytes_full_cache"])
+    if also:
+        line["also"] = also
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"], _ = oracle_baseline(cfg, args.ref_seqs, args.ref_steps)
     print(json.dumps(line), flush=True)
