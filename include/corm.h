@@ -149,6 +149,18 @@ corm_status_t corm_compress_prompt(corm_cache_t* cache, int32_t layer, const voi
 corm_status_t corm_decode_step(corm_cache_t* cache, int32_t layer, const void* q, const void* k_new,
                                const void* v_new, void* out, void* stream);
 
+/* The same step for n_layers consecutive layers from one host call: layer first_layer + i takes q[i], k_new[i],
+ * v_new[i] and writes out[i] (host arrays of device pointers, each as for corm_decode_step). The paper applies the
+ * policy "on each head at every layer" (footnote to the Approach paragraph) and the layers of a cache are independent
+ * (each has its own token and row counts), so this is exactly n_layers calls of corm_decode_step in layer order on
+ * `stream`; it exists because one launch per layer of a single-sequence model is a few microseconds of GPU work and
+ * a host call per launch costs more than that. In a model the layers' inputs depend on each other's outputs; use
+ * this where they are all known (replay, benchmarking, speculative batches), the per-layer call otherwise.
+ * Errors: as corm_decode_step, all arguments and every layer's state checked before anything is enqueued. */
+corm_status_t corm_decode_step_layers(corm_cache_t* cache, int32_t first_layer, int32_t n_layers,
+                                      const void* const* q, const void* const* k_new, const void* const* v_new,
+                                      void* const* out, void* stream);
+
 /* Same step with HOST buffers, asynchronous on `stream` (out_host is valid once the stream has been synchronised).
  * Pinned buffers the device can address (cudaHostAlloc / cudaHostRegister, 16-byte aligned) are read and written by
  * the kernels directly across the bus, with no copies; any other host memory is copied to staging space inside the

@@ -75,6 +75,8 @@ def load_library():
     lib.corm_decode_step_static.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.corm_decode_step_host.restype = i32
     lib.corm_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.corm_decode_step_layers.restype = i32
+    lib.corm_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.corm_cache_stats.restype = i32
     lib.corm_cache_stats.argtypes = [vp, ctypes.POINTER(CormStats), vp]
     lib.corm_cache_live_lens.restype = i32
@@ -188,6 +190,33 @@ class CormCache:
         if rc != CORM_OK:
             raise CormError("corm_decode_step", rc)
         return out
+
+    def corm_decode_step_layers(self, first_layer, q, k_new, v_new, out, stream=None):
+        """One decode step of ``len(q)`` consecutive layers from a single host call. ``q``, ``k_new``, ``v_new``,
+        ``out``: sequences of per-layer tensors, or ``numpy`` uint64 arrays of their device addresses as
+        ``pointer_table`` builds them (no per-tensor work on the host then; shapes were checked when it was built)."""
+        n = len(q)
+        if not (len(k_new) == len(v_new) == len(out) == n and n >= 1):
+            raise ValueError("corm_decode_step_layers: one q, k_new, v_new and out per layer")
+        tables = []
+        for i, ts in enumerate((q, k_new, v_new, out)):
+            if isinstance(ts, np.ndarray):
+                assert ts.dtype == np.uint64 and ts.flags.c_contiguous
+                tables.append(ts)
+            else:
+                tables.append(self.pointer_table(ts, "q" if i in (0, 3) else "kv"))
+        _check("corm_decode_step_layers", self.lib.corm_decode_step_layers(
+            self.handle, first_layer, n, tables[0].ctypes.data, tables[1].ctypes.data, tables[2].ctypes.data,
+            tables[3].ctypes.data, _stream_ptr(stream)))
+        return out
+
+    def pointer_table(self, tensors, kind):
+        """Device addresses of per-layer tensors as a uint64 array (kind "q": shaped like q / out, "kv": like k_new)."""
+        shape = self._q_shape if kind == "q" else self._kv_shape
+        for t in tensors:
+            if not (t.shape == shape and t.dtype == self.dtype and t.is_cuda and t.is_contiguous()):
+                raise ValueError("pointer_table: contiguous device tensors of the cache dtype with the step's shape")
+        return np.array([t.data_ptr() for t in tensors], dtype=np.uint64)
 
     def corm_decode_step_static(self, layer, q, k_new, v_new, out=None, stream=None):
         """corm_decode_step for callers that must not allocate: the step's scratch sits in an array built into the

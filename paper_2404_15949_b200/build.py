@@ -16,13 +16,21 @@ def _sources():
         os.path.join(os.path.dirname(_HERE), "include", "corm.h")]
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile ``csrc/*.cu`` into ``libcorm.so`` next to this file when it is missing or older than a source."""
+DEBUG_LIB_PATH = os.path.join(_HERE, "libcorm_dbg.so")
+
+
+def build_library(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """Compile ``csrc/*.cu`` into ``libcorm.so`` next to this file when it is missing or older than a source.
+
+    ``debug_bounds=True`` builds ``libcorm_dbg.so`` instead, with -DCORM_DEBUG_BOUNDS: every slot, list, record and
+    mask index is range-checked in the kernels before use (a failed check sets the device status and skips the
+    access). Load it with ``CORM_LIB_PATH=.../libcorm_dbg.so`` and run the GPU tests against it."""
+    lib_path = DEBUG_LIB_PATH if debug_bounds else LIB_PATH
     newest = max(os.path.getmtime(s) for s in _sources())
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= newest:
-        return LIB_PATH
+    if not force and os.path.exists(lib_path) and os.path.getmtime(lib_path) >= newest:
+        return lib_path
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB_PATH] + [
-        s for s in _sources() if s.endswith(".cu")]
+    cmd = [nvcc] + NVCC_FLAGS + (["-DCORM_DEBUG_BOUNDS"] if debug_bounds else []) + (["-Xptxas", "-v"] if verbose else []) + ["-o", lib_path] + [
+        s for s in _sources() if s.endswith(".cu")] + ["-ldl"]      # NVTX (header-only) loads its collector with dlopen
     subprocess.check_call(cmd)
-    return LIB_PATH
+    return lib_path

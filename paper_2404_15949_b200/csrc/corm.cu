@@ -2,6 +2,7 @@
 // path runs in the kernels of corm_fast.cuh / corm_verdict.cuh / corm_prompt_fast.cuh / corm_generic.cuh; nothing
 // here touches tensor data on the CPU.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <algorithm>
 #include <cmath>
@@ -29,7 +30,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, ticket3, move_info, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -89,6 +90,8 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.base_obs = take(Ltot * c.batch * 4);
     L.ticket = take(Ltot * U * 4);
     L.ticket2 = take(Ltot * U * 4);
+    L.ticket3 = take(Ltot * U * 4);
+    L.move_info = take(Ltot * U * 8);
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
@@ -117,6 +120,12 @@ struct DeviceGuard {
         if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
     }
     ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Named range around a boundary call, visible to profilers that collect NVTX (a no-op without one).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
 };
 
 #define CORM_CUDA(expr)                                                         \
@@ -287,6 +296,8 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.base_obs = reinterpret_cast<int32_t*>(layer_ptr(c, c->lay.base_obs, (size_t)cf.batch * 4, layer));
     p.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
     p.ticket2 = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket2, U * 4, layer));
+    p.ticket3 = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket3, U * 4, layer));
+    p.move_info = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.move_info, U * 8, layer));
     p.counters = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer));
     p.status = reinterpret_cast<int32_t*>(c->arena + c->lay.status);
     p.maxlive = maxlive_ptr(c, layer);
@@ -299,7 +310,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.log_alpha = log_alpha_of(c);
     const int upper = std::min(cf.max_tokens, c->live_upper[layer] + 1);   // no unit can hold more live keys
 
-    const bool fast = fast_path_available() && c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
+    const bool fast = c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
     int n_launched = 1;
     // Group sizes above one take the balanced kernel while no unit can be longer than kBalancedAutoLimit keys (its
@@ -451,6 +462,7 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
 
 corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k_prompt, const void* v_prompt,
                                    const void* q_last, const int32_t* prompt_lens_host, int32_t p_max, void* stream) {
+    NvtxRange nvtx_range("corm_compress_prompt");
     if (!layer_ok(c, layer) || !prompt_lens_host || p_max < 0) return CORM_ERR_INVALID_ARG;
     const corm_config_t& cf = c->cfg;
     int max_p = 0;
@@ -476,6 +488,8 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     CORM_CUDA(cudaMemcpyAsync(base_obs, obs.data(), (size_t)cf.batch * 4, cudaMemcpyHostToDevice, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket, U * 4, layer), 0, U * 4, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket2, U * 4, layer), 0, U * 4, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket3, U * 4, layer), 0, U * 4, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.move_info, U * 8, layer), 0, U * 8, st));
     CORM_CUDA(cudaMemsetAsync(maxlive_ptr(c, layer), 0, 8, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer), 0, CNT_COUNT * 8, st));   // a new prompt restarts the layer's statistics
     c->readback_pending[layer] = 0;   // an older read-back no longer describes this layer
@@ -535,6 +549,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
 
 corm_status_t corm_decode_step(corm_cache_t* c, int32_t layer, const void* q, const void* k_new, const void* v_new,
                                void* out, void* stream) {
+    NvtxRange nvtx_range("corm_decode_step");
     if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return CORM_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
          reinterpret_cast<uintptr_t>(out)) % 16) return CORM_ERR_INVALID_ARG;
@@ -544,8 +559,30 @@ corm_status_t corm_decode_step(corm_cache_t* c, int32_t layer, const void* q, co
     return launch_decode(c, layer, q, k_new, v_new, out, static_cast<cudaStream_t>(stream));
 }
 
+corm_status_t corm_decode_step_layers(corm_cache_t* c, int32_t first_layer, int32_t n_layers, const void* const* q,
+                                      const void* const* k_new, const void* const* v_new, void* const* out,
+                                      void* stream) {
+    NvtxRange nvtx_range("corm_decode_step_layers");
+    if (!c || n_layers < 1 || !layer_ok(c, first_layer) || !layer_ok(c, first_layer + n_layers - 1) || !q || !k_new ||
+        !v_new || !out) return CORM_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i) {                 // everything is checked before anything is enqueued
+        if (!q[i] || !k_new[i] || !v_new[i] || !out[i]) return CORM_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(q[i]) | reinterpret_cast<uintptr_t>(k_new[i]) | reinterpret_cast<uintptr_t>(v_new[i]) |
+             reinterpret_cast<uintptr_t>(out[i])) % 16) return CORM_ERR_INVALID_ARG;
+        if (!c->ready[first_layer + i]) return CORM_ERR_STATE;
+    }
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    for (int i = 0; i < n_layers; ++i) {
+        const corm_status_t rc = launch_decode(c, first_layer + i, q[i], k_new[i], v_new[i], out[i], static_cast<cudaStream_t>(stream));
+        if (rc != CORM_OK) return rc;
+    }
+    return CORM_OK;
+}
+
 corm_status_t corm_decode_step_host(corm_cache_t* c, int32_t layer, const void* q_host, const void* k_new_host,
                                     const void* v_new_host, void* out_host, void* stream) {
+    NvtxRange nvtx_range("corm_decode_step_host");
     if (!layer_ok(c, layer) || !q_host || !k_new_host || !v_new_host || !out_host) return CORM_ERR_INVALID_ARG;
     if (!c->ready[layer]) return CORM_ERR_STATE;
     DeviceGuard guard(c->cfg.device);
@@ -609,6 +646,7 @@ corm_status_t static_scratch_address(int device, unsigned char** out) {
 
 corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void* q, const void* k_new,
                                       const void* v_new, void* out, void* stream) {
+    NvtxRange nvtx_range("corm_decode_step_static");
     if (!layer_ok(c, layer) || !q || !k_new || !v_new || !out) return CORM_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
          reinterpret_cast<uintptr_t>(out)) % 16) return CORM_ERR_INVALID_ARG;
@@ -684,6 +722,7 @@ corm_status_t corm_cache_live_lens(corm_cache_t* c, int32_t layer, int32_t* live
 }
 
 corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* stream) {
+    NvtxRange nvtx_range("corm_cache_stats");
     if (!c || !out_host) return CORM_ERR_INVALID_ARG;
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return CORM_ERR_CUDA;

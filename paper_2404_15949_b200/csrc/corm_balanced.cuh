@@ -37,6 +37,7 @@ constexpr int kBalRingBytes = kBalWarps * kBalWarpBytes;       // 96 KiB, reused
 constexpr int kBalBlocksPerSm = 2;
 constexpr int kBalSegCap = 32;                                  // segments listed per window of a block's range
 constexpr int kBalRec = 16 + 4 * 128;                           // {double m, double Z, float acc[128]}
+constexpr int kBalSoloMoves = 32;                               // rows a unit's last block moves alone; more are shared out
 constexpr int kBalCacheUnits = 16384;                            // units whose lengths the prologue parks in shared memory
 constexpr int kBalMaxTokens = 1 << 17;                          // the finish phase keeps 3 bits-per-32 arrays on chip
 
@@ -58,6 +59,7 @@ struct BalMisc {
     int scan[kBalThreads];           // finish phase: scratch of the block-wide prefix sums
     int wsum[kBalWarps];
     int first_u, first_P, nseg, more, next_u, next_P, last, failed;
+    unsigned long long info;         // finish phase: a unit's move word as read by thread 0
 };
 
 // shared-memory carve-up behind the 1024-byte aligned ring
@@ -115,9 +117,17 @@ __device__ __forceinline__ int vtile_offset(int r, int c) {
     return (c >> 3) * (kTileBytes / 2) + r * 128 + ((((c & 7) ^ r) & 7) << 4);
 }
 
+// records the balanced kernel may write in one step: one per warp of every (block, unit) pair on the tile list
+__host__ __device__ inline size_t bal_record_count(int n_blocks, int U) { return ((size_t)n_blocks + (size_t)U) * kBalWarps; }
+
 // block of the balanced partition that owns tile x of the step's list (T tiles, n blocks)
 __device__ __forceinline__ int bal_block_of(long long x, long long T, int n) { return (int)(((x + 1) * n - 1) / T); }
 
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -145,7 +155,7 @@ struct BalFin {
 //      unit's last block scans the mask, fills the holes and publishes the new length.
 // scratch: the block's ring area, free by now.
 template <int G, bool PAGED, int NT>
-__device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
+__device__ __noinline__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
                                  unsigned char* scratch, BalMisc* misc) {
     constexpr int NW = kBalWarps;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -291,7 +301,7 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
 #pragma unroll
                 for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= thr[si * 4 + g]);
                 const uint32_t wd = update_register(wv[k], imp, p.w, sg.t);
-                p.word[(size_t)sg.u * p.C + j] = wd;
+                if (CORM_IN_RANGE(j < p.C, p.status)) p.word[(size_t)sg.u * p.C + j] = wd;
                 keep = !fin[si].evict_on || register_needed(wd, p.w, sg.t) || pv[k] > sg.t - p.r;
                 n_imp += imp ? 1 : 0;
             }
@@ -301,7 +311,9 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
                 const int tile = x0 >> 5;
                 int s2 = 0;
                 while (s2 + 1 < nseg && fin[s2 + 1].tile_prefix <= tile) ++s2;
-                p.keepmask[(size_t)segs[s2].u * keepmask_words(p.C) + segs[s2].tile0 + tile - fin[s2].tile_prefix] = ballot;
+                const int kw = segs[s2].tile0 + tile - fin[s2].tile_prefix;
+                if (CORM_IN_RANGE(kw >= 0 && kw < keepmask_words(p.C), p.status))
+                    p.keepmask[(size_t)segs[s2].u * keepmask_words(p.C) + kw] = ballot;
             }
         }
     }
@@ -345,71 +357,115 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
     }
     __syncthreads();
 
-    // ---- the units this block is the last of: compaction ----
+    // ---- compaction ----
+    // The unit's last block scans the keep mask and lists the holes below the new length and the kept rows above it.
+    // A few rows it moves itself. Many rows (the steps right after a prompt pass, long units) are shared out over all
+    // the unit's blocks: the last block publishes the counts in the unit's move word, the others, which wait for that
+    // word (bounded; the last block needs nobody's help to get there), take every n_blocks-th chunk of 16 rows, and a
+    // third arrival counter tells the block that finishes last to settle the pages and publish the new length.
     for (int si = 0; si < nseg; ++si) {
-        if (!fin[si].last) continue;                                            // uniform
+        const BalFin f = fin[si];
         const BalSeg& sg = segs[si];
-        const int u = sg.u, l = sg.l, t = sg.t, words = (l + 31) / 32 + 2, nwords = (l + 31) / 32;
-        uint32_t* keep_sm = reinterpret_cast<uint32_t*>(comp);
-        int* prefix = reinterpret_cast<int*>(keep_sm + words);
-        int32_t* pt_sm = prefix + words;
+        const int u = sg.u, l = sg.l, words = (l + 31) / 32 + 2, nwords = (l + 31) / 32;
         const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-        const uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
         uint32_t* wordu = p.word + (size_t)u * p.C;
         int32_t* posu = p.pos + (size_t)u * p.C;
-        for (int i = tid; i < nwords; i += NT) {
-            keep_sm[i] = __ldcg(keep_g + i);
-            if (PAGED) pt_sm[i] = __ldcg(pt_u + i);
-        }
-        __syncthreads();
-        int new_len = l, n_moved = 0;
-        if (fin[si].evict_on) {
-            block_popc_scan<NT>(keep_sm, prefix, nwords, misc->scan);
-            new_len = prefix[nwords];
-            if (new_len < l) {
-                const int kept_below = kept_before(keep_sm, prefix, new_len);
-                n_moved = new_len - kept_below;
-                int* holes = reinterpret_cast<int*>(p.stash + (size_t)u * G * p.C);   // every block is done with the logits
-                int* movers = holes + p.C;
-                for (int i = tid; i < nwords; i += NT) {
-                    const uint32_t m = keep_sm[i];
-                    const int w0 = i * 32;
-                    const uint32_t valid = l - w0 >= 32 ? 0xffffffffu : (1u << (l - w0)) - 1u;
-                    const uint32_t below = new_len - w0 >= 32 ? 0xffffffffu : (new_len > w0 ? (1u << (new_len - w0)) - 1u : 0u);
-                    uint32_t hm = ~m & valid & below;                       // evicted slots below the new length
-                    while (hm) {
-                        const int bit = __ffs(hm) - 1;
-                        hm &= hm - 1u;
-                        holes[w0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = w0 + bit;
-                    }
-                    uint32_t km = m & valid & ~below;                       // kept slots at or above it
-                    while (km) {
-                        const int bit = __ffs(km) - 1;
-                        km &= km - 1u;
-                        movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = w0 + bit;
-                    }
-                }
-                __syncthreads();
-                const size_t slab_row0 = (size_t)u * p.C;
-                block_move_rows<bf16_t, 128, NT>(
-                    reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
-                    [&](int slot) -> size_t {
-                        return PAGED ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
-                    },
-                    wordu, posu, movers, holes, n_moved);
+        int* holes = reinterpret_cast<int*>(p.stash + (size_t)u * G * p.C);   // every block is done with the logits
+        int* movers = holes + p.C;
+        const size_t slab_row0 = (size_t)u * p.C;
+        auto row_of = [&](int slot) -> size_t {
+            if (!PAGED) return slab_row0 + (size_t)slot;
+            return page_row(__ldcg(pt_u + (slot >> 5)), slot, p.pool_pages, p.status);
+        };
+        auto publish = [&](int new_len, int n_moved) {                         // whole block
+            if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+            if (tid == 0) {
+                p.live_out[u] = new_len;
+                publish_live(p.maxlive, p.step + 1, new_len);
+                atomicAdd(p.counters + CNT_APPENDED, 1ull);
+                atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+                if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+                if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
             }
+        };
+        unsigned long long info = 0ull;                                        // done bit | rows to share << 32 | new length
+        if (f.last) {
+            uint32_t* keep_sm = reinterpret_cast<uint32_t*>(comp);
+            int* prefix = reinterpret_cast<int*>(keep_sm + words);
+            const uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
+            for (int i = tid; i < nwords; i += NT) keep_sm[i] = __ldcg(keep_g + i);
+            __syncthreads();
+            int new_len = l, n_moved = 0;
+            if (f.evict_on) {
+                block_popc_scan<NT>(keep_sm, prefix, nwords, misc->scan);
+                new_len = prefix[nwords];
+                if (new_len < l) {
+                    const int kept_below = kept_before(keep_sm, prefix, new_len);
+                    n_moved = new_len - kept_below;
+                    for (int i = tid; i < nwords; i += NT) {
+                        const uint32_t m = keep_sm[i];
+                        const int w0 = i * 32;
+                        const uint32_t valid = l - w0 >= 32 ? 0xffffffffu : (1u << (l - w0)) - 1u;
+                        const uint32_t below = new_len - w0 >= 32 ? 0xffffffffu : (new_len > w0 ? (1u << (new_len - w0)) - 1u : 0u);
+                        uint32_t hm = ~m & valid & below;                       // evicted slots below the new length
+                        while (hm) {
+                            const int bit = __ffs(hm) - 1;
+                            hm &= hm - 1u;
+                            holes[w0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = w0 + bit;
+                        }
+                        uint32_t km = m & valid & ~below;                       // kept slots at or above it
+                        while (km) {
+                            const int bit = __ffs(km) - 1;
+                            km &= km - 1u;
+                            movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = w0 + bit;
+                        }
+                    }
+                    __syncthreads();
+                }
+            }
+            const bool shared = f.n_blocks > 1 && n_moved > kBalSoloMoves;
+            if (!shared) {
+                block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), row_of,
+                                                 wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
+                publish(new_len, n_moved);
+            }
+            info = (1ull << 63) | ((unsigned long long)(shared ? n_moved : 0) << 32) | (unsigned)new_len;
+            if (f.n_blocks > 1) {
+                __threadfence();                                               // the lists (and a solo block's moves) before the word
+                __syncthreads();
+                if (tid == 0) atomicExch(p.move_info + u, info);
+            }
+        } else {                                                               // wait for the last block's counts
+            if (tid == 0) {
+                const long long start = clock64();
+                unsigned long long v;
+                while (!((v = ld_acquire_u64(p.move_info + u)) >> 63)) {
+                    if (clock64() - start > kWaitLimitCycles) { misc->failed = 1; break; }
+                    __nanosleep(64);
+                }
+                misc->info = v;
+            }
+            __syncthreads();
+            if (misc->failed) { if (tid == 0) report_status(p.status, CORM_ERR_TIMEOUT); return; }
+            info = misc->info;
         }
-        if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
-        if (tid == 0) {
-            p.live_out[u] = new_len;
-            publish_live(p.maxlive, p.step + 1, new_len);
-            atomicAdd(p.counters + CNT_APPENDED, 1ull);
-            atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
-            if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
-            if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
+        if (f.n_blocks > 1) {
+            const int n_share = (int)((info >> 32) & 0x7fffffffu), new_len = (int)(info & 0xffffffffu);
+            if (n_share)                                                       // this block's chunks of 16 rows
+                block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), row_of,
+                                                 wordu, posu, movers, holes, n_share, blk - (f.rec0 / NW - u), f.n_blocks, l, p.status);
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                const unsigned prev = atomicAdd(p.ticket3 + u, 1u);
+                misc->last = (prev == (unsigned)(f.n_blocks - 1));
+                if (misc->last) { p.ticket3[u] = 0u; atomicExch(p.move_info + u, 0ull); }   // every block has read the word
+                __threadfence();
+            }
+            __syncthreads();
+            if (misc->last && n_share) publish(new_len, n_share);              // all rows are in place
         }
-        __syncthreads();                                                     // the arrays are reused by the next unit
-        (void)t;
+        __syncthreads();                                                       // the arrays are reused by the next unit
     }
 }
 
@@ -644,27 +700,20 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
                     const int kslot = n_consumed % kBalKStages;
                     unsigned char* ktile = my_tiles + kslot * kTileBytes;
                     unsigned char* vtile = my_tiles + kBalKStages * kTileBytes;
-                    long long row0 = 0;
-                    uint4 newk = make_uint4(0, 0, 0, 0), newv = make_uint4(0, 0, 0, 0);
-                    if (has_new) {
-                        row0 = tile_row0(sg, ti);
-                        if (lane < 16) {
-                            if (si < lay.n_pre) {
-                                newk = *reinterpret_cast<const uint4*>(smem + lay.segnew + (si * 32 + lane) * 16);
-                                newv = *reinterpret_cast<const uint4*>(smem + lay.segnew + (si * 32 + 16 + lane) * 16);
-                            } else {
-                                newk = __ldcg(reinterpret_cast<const uint4*>(p.k_new) + (size_t)u * 16 + lane);
-                                newv = __ldcg(reinterpret_cast<const uint4*>(p.v_new) + (size_t)u * 16 + lane);
-                            }
-                        }
-                    }
+                    // the appended token's row (K or V, `which` 0 / 1) as fetched ahead, or from global memory
+                    auto new_row = [&](int which) -> uint4 {
+                        if (si < lay.n_pre) return *reinterpret_cast<const uint4*>(smem + lay.segnew + (si * 32 + which * 16 + (lane & 15)) * 16);
+                        return __ldcg(reinterpret_cast<const uint4*>(which ? p.v_new : p.k_new) + (size_t)u * 16 + (lane & 15));
+                    };
                     if (!failed && !mbar_wait(my_bars + kslot * 8, (n_consumed / kBalKStages) & 1)) failed = true;   // once one wait has expired the rest are skipped
-                    if (has_new && row0 >= 0) {   // append: the new row goes to the cache and into the arriving tile
-                        if (lane < 16) {
+                    if (has_new) {   // append: the new row goes to the cache and into the arriving tile
+                        const long long row0 = tile_row0(sg, ti);
+                        if (row0 >= 0 && lane < 16) {
+                            const uint4 newk = new_row(0);
                             *reinterpret_cast<uint4*>(ktile + (l_old - k0) * kRowBytes + lane * 16) = newk;
                             reinterpret_cast<uint4*>(Kl + (row0 + (l_old - k0)) * kRowBytes)[lane] = newk;
                         }
-                        if (lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
+                        if (row0 >= 0 && lane == 0) { wordu[l_old] = 0u; posu[l_old] = t; }
                         __syncwarp();
                     }
                     double sown[G];
@@ -720,7 +769,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
                         pw[g] = pack_bf16x2(pf - hi_f, pf);                 // column 2g = hi, column 2g + 1 = lo
                     }
                     *reinterpret_cast<uint4*>(psm + key_own * 16) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-                    if (valid) {
+                    if (valid && CORM_IN_RANGE(j_own < p.C, p.status)) {
                         double* dst = p.stash + ((size_t)u * p.C + j_own) * G;
                         if (G == 4) {
                             reinterpret_cast<double2*>(dst)[0] = make_double2(sv[0], sv[1]);
@@ -734,9 +783,13 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
                     __syncwarp();
 
                     if (!failed && !mbar_wait(my_bars + kBalKStages * 8, n_consumed & 1)) failed = true;
-                    if (has_new && row0 >= 0 && lane < 16) {
-                        *reinterpret_cast<uint4*>(vtile + vtile_offset(l_old - k0, lane)) = newv;
-                        reinterpret_cast<uint4*>(Vl + (row0 + (l_old - k0)) * kRowBytes)[lane] = newv;
+                    if (has_new) {
+                        const long long row0 = tile_row0(sg, ti);
+                        if (row0 >= 0 && lane < 16) {
+                            const uint4 newv = new_row(1);
+                            *reinterpret_cast<uint4*>(vtile + vtile_offset(l_old - k0, lane)) = newv;
+                            reinterpret_cast<uint4*>(Vl + (row0 + (l_old - k0)) * kRowBytes)[lane] = newv;
+                        }
                     }
                     if (n_valid < kTileKeys)     // rows past the unit's end hold whatever the slab had: make them harmless for 0 * v
                         for (int x = lane; x < (kTileKeys - n_valid) * 16; x += 32) {
@@ -775,6 +828,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
             // other warps of the block stream on.
             const size_t pstride = partial_stride(128);
             unsigned char* rec_w = p.partials + ((size_t)(blk + u) * NW + warp) * G * pstride;   // blk + u is unique: both grow along the tile list
+            if (!CORM_IN_RANGE((size_t)(blk + u) * NW + warp < bal_record_count(nblk, p.U), p.status)) continue;
             if (lane < G) {
                 double* mz = reinterpret_cast<double*>(rec_w + (size_t)lane * pstride);
                 double Mg = M[0], Zg = Zl[0];
@@ -837,8 +891,6 @@ inline corm_status_t make_v_tensor_map(CUtensorMap* out, void* v_layer, unsigned
     return r == CUDA_SUCCESS ? CORM_OK : CORM_ERR_CUDA;
 }
 
-// records the balanced kernel may write in one step: one per warp of every (block, unit) pair on the tile list
-__host__ __device__ inline size_t bal_record_count(int n_blocks, int U) { return ((size_t)n_blocks + (size_t)U) * kBalWarps; }
 
 inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& vmap, int G, int upper, int sm_count,
                                             size_t partial_capacity_records, cudaStream_t st, int* n_launched) {

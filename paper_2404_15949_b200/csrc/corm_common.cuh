@@ -59,6 +59,8 @@ struct DecodeParams {
     const int32_t* base_obs;     // [B] verdict rows recorded at that time
     uint32_t* ticket;         // [U] arrival counters of the splits of a unit (zero between steps)
     uint32_t* ticket2;        // [U] second arrival counters (balanced kernel: blocks done with their verdicts)
+    uint32_t* ticket3;        // [U] third arrival counters (balanced kernel: blocks done with their share of the row moves)
+    unsigned long long* move_info;   // [U] balanced kernel: the unit's move word (zero between steps)
     unsigned long long* counters;  // [CNT_COUNT]
     int32_t* status;          // sticky device status
     unsigned long long* maxlive;  // (steps done << 32 | longest live length after that step), atomicMax; may be null
@@ -155,6 +157,17 @@ template <> __device__ __forceinline__ void load_slice<bf16_t, 2>(const bf16_t* 
 // one nor the other way round. After any non-zero status the cache must be reset before it is used again.
 __device__ __forceinline__ void report_status(int32_t* status, corm_status_t code) { atomicMax(status, (int32_t)code); }
 
+// Range checks. compute-sanitizer cannot be run where this library is developed, so the kernels can check themselves:
+// a build with -DCORM_DEBUG_BOUNDS tests every slot, list entry, record and mask index before it is used; a failed
+// test reports CORM_ERR_INTERNAL through the status word and SKIPS the access (the kernel goes on and returns
+// normally). The release build compiles the tests away, except for page-table entries (page_row below): those come
+// from memory, and a bad one would otherwise become a wild address.
+#ifdef CORM_DEBUG_BOUNDS
+#define CORM_IN_RANGE(cond, status) ((cond) ? true : (corm::report_status((status), CORM_ERR_INTERNAL), false))
+#else
+#define CORM_IN_RANGE(cond, status) true
+#endif
+
 // Adds the warp's total of n to a 64-bit counter (one atomic per warp; all lanes must call).
 __device__ __forceinline__ void warp_count(unsigned long long* counter, int n) {
 #pragma unroll
@@ -199,9 +212,17 @@ __device__ __forceinline__ bool register_needed(uint32_t reg, int w, int t) {
 // untouched, like a full slab.
 constexpr int kPageKeys = 32;
 
+// Row of a slot whose page-table entry is `entry` (page + 1). An entry outside the pool means the table is broken:
+// it is reported and the slot's row inside page 0 is returned, so that no address is ever formed from a bad entry
+// (checked in every build). The data is wrong from then on; the status tells the caller to reset the cache.
+__device__ __forceinline__ size_t page_row(int entry, int slot, int pool_pages, int32_t* status) {
+    if (entry <= 0 || entry > pool_pages) { report_status(status, CORM_ERR_INTERNAL); entry = 1; }
+    return (size_t)(entry - 1) * kPageKeys + (slot & 31);
+}
+
 // row of slot `slot` in the layer's K / V storage: through the unit's page table, or inside its slab
-__device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, int slot) {
-    return pt_u ? (size_t)(__ldcg(pt_u + (slot >> 5)) - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
+__device__ __forceinline__ size_t kv_row(const int32_t* pt_u, size_t slab_row0, int slot, int pool_pages, int32_t* status) {
+    return pt_u ? page_row(__ldcg(pt_u + (slot >> 5)), slot, pool_pages, status) : slab_row0 + (size_t)slot;
 }
 
 // Claims one free page for page-table entry `index` of unit u (of n_units). Every unit has a home region of the
@@ -319,12 +340,15 @@ __device__ __forceinline__ int kept_before(const uint32_t* mask, const int* pref
 // four rows at a time and issues all their loads before the first store (the copies are latency-, not
 // bandwidth-limited). Rows are D*sizeof(T) bytes = a multiple of 16.
 // row_of(slot) gives the slot's row in the layer's K / V storage (Kl, Vl).
+// part / n_parts: this block takes the chunks of NT / 8 rows numbered part, part + n_parts, ... (several blocks
+// sharing one unit's moves); the default is every chunk.
 template <typename T, int D, int NT, typename RowOf>
 __device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, RowOf row_of, uint32_t* wordu, int32_t* posu,
-                                                const int* movers, const int* holes, int n_moved) {
+                                                const int* movers, const int* holes, int n_moved, int part = 0,
+                                                int n_parts = 1, int slot_limit = 0x7fffffff, int32_t* status = nullptr) {
     constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = 4, NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i0 = warp * kRows; i0 < n_moved; i0 += NW * kRows) {
+    for (int i0 = (part * NW + warp) * kRows; i0 < n_moved; i0 += n_parts * NW * kRows) {
         int src[kRows], dst[kRows];
         size_t srow[kRows], drow[kRows];                 // rows of the layer's K / V storage (Kl, Vl)
         uint4 buf[kRows][kIter];
@@ -335,6 +359,8 @@ __device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, RowOf row_of, uint
             const bool on = i0 + r < n_moved;
             src[r] = on ? movers[i0 + r] : -1;
             dst[r] = on ? holes[i0 + r] : -1;
+            if (on && !CORM_IN_RANGE(src[r] >= 0 && src[r] < slot_limit && dst[r] >= 0 && dst[r] < slot_limit, status))
+                src[r] = dst[r] = -1;                      // the row is left where it is
             srow[r] = on ? row_of(src[r]) : 0;
             drow[r] = on ? row_of(dst[r]) : 0;
         }
@@ -454,12 +480,13 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
 #pragma unroll
                 for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
                 const uint32_t wd = update_register(wv[k], imp, p.w, t);
-                wordu[j] = wd;
+                if (CORM_IN_RANGE(j < p.C, p.status)) wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
                 n_imp += imp ? 1 : 0;
             }
             const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
-            if (lane == 0 && base + warp * 32 < l) keepmask[(base >> 5) + warp] = ballot;
+            if (lane == 0 && base + warp * 32 < l && CORM_IN_RANGE((base >> 5) + warp < cap_words, p.status))
+                keepmask[(base >> 5) + warp] = ballot;
         }
     }
     warp_count(p.counters + CNT_IMPORTANT, n_imp);         // Section 3.1's sparsity: keys judged important this step
@@ -485,8 +512,8 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
             const size_t slab_row0 = (size_t)u * p.C;
             block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
                                       [&](int slot) -> size_t {
-                                          return pt_u ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
-                                      }, wordu, posu, movers, holes, n_moved);
+                                          return pt_u ? page_row(pt_sm[slot >> 5], slot, p.pool_pages, p.status) : slab_row0 + (size_t)slot;
+                                      }, wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
         }
     }
     settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);

@@ -44,8 +44,6 @@ constexpr long long kWaitLimitCycles = 4000000000ll;   // bounded mbarrier waits
 // longest unit that may finish inside one block (bounded by the registers that carry its verdict words)
 __host__ __device__ constexpr int fast_max_single_cap(int G) { return (G == 1 ? 8 : 2) * kFastThreads; }
 
-inline bool fast_path_available() { return true; }
-
 // ---- shared-memory carve-up (bytes), all offsets multiples of 128 ----
 struct FastSmem {
     int tiles, psm, stash, bars, newrow, total;
@@ -255,10 +253,10 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
                 reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
                 [&](int slot) -> size_t {      // the unit is one split: its pages are the ones the warps fetched for their tiles
                     const int tile = slot >> 5;
-                    return PAGED ? (size_t)(tile_pages[tile % kFastWarps][tile / kFastWarps] - 1) * kPageKeys + (slot & 31)
+                    return PAGED ? page_row(tile_pages[tile % kFastWarps][tile / kFastWarps], slot, p.pool_pages, p.status)
                                  : slab_row0 + (size_t)slot;
                 },
-                wordu, posu, movers, holes, n_moved);
+                wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
         }
     }
     if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
@@ -289,6 +287,9 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     // without a page for the appended row (pool exhausted) is treated like a full slab.
     __shared__ int32_t s_pt[kFastWarps][32];
     const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+    // launched with programmatic stream serialization: the block may start while the previous launch on the stream
+    // drains and reads nothing before that launch has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     int32_t my_page = 0, room = 1;
     if (PAGED) {
         const int idx = split * (p.split_len >> 5) + warp + lane * kFastWarps;
@@ -327,7 +328,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     auto tile_row0 = [&](int it) -> size_t {
         if (!PAGED) return slab_row0 + (size_t)(begin + (warp + it * NW) * kTileKeys);
         const int pg = it < 32 ? s_pt[warp][it] : __ldcg(pt_u + (begin >> 5) + warp + it * NW);
-        return (size_t)(pg - 1) * kPageKeys;
+        return page_row(pg, 0, p.pool_pages, p.status);
     };
     auto tile_keys = [&](int it) { return min(kTileKeys, end - (begin + (warp + it * NW) * kTileKeys)); };
     auto issue_k = [&](int it) {
@@ -468,8 +469,8 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
             M[g] = Mn[g];
             psm[key_own * G + g] = (float)ex[g];
             if (valid) {
-                if (single) stash_sm[g * p.single_cap + j_own] = sv[g];
-                else p.stash[((size_t)u * G + g) * p.C + j_own] = sv[g];
+                if (single) { if (CORM_IN_RANGE(j_own < p.single_cap, p.status)) stash_sm[g * p.single_cap + j_own] = sv[g]; }
+                else if (CORM_IN_RANGE(j_own < p.C, p.status)) p.stash[((size_t)u * G + g) * p.C + j_own] = sv[g];
             }
         }
         __syncwarp();
@@ -668,8 +669,18 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     auto launch = [&](auto kern) -> corm_status_t {
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
-        kern<<<dim3(n_splits, (unsigned)p.U), kFastThreads, smem, st>>>(p);
-        e = cudaGetLastError();
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(n_splits, (unsigned)p.U);
+        cfg.blockDim = dim3(kFastThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // launch latency hides behind the previous launch's tail
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, p);
+        if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;
     };

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     if (l_old >= begin && l_old < end) {
         const T* kn = reinterpret_cast<const T*>(p.k_new) + (size_t)u * D;
         const T* vn = reinterpret_cast<const T*>(p.v_new) + (size_t)u * D;
-        const size_t row = kv_row(pt_u, slab_row0, l_old);
+        const size_t row = kv_row(pt_u, slab_row0, l_old, p.pool_pages, p.status);
         for (int c = tid; c < D; c += NT) { Kl[row * D + c] = kn[c]; Vl[row * D + c] = vn[c]; }
         if (tid == 0) { p.word[(size_t)u * p.C + l_old] = 0u; p.pos[(size_t)u * p.C + l_old] = t; }
         __syncthreads();
@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(kGenericThreads) decode_generic_kernel(const _
     const double root_d = sqrt((double)D);
     for (int j = begin + warp; j < end; j += NW) {
         float kf[NPL], vf[NPL];
-        const size_t row = kv_row(pt_u, slab_row0, j);
+        const size_t row = kv_row(pt_u, slab_row0, j, p.pool_pages, p.status);
         load_slice<T, NPL>(Kl + row * D + c0, kf);
         load_slice<T, NPL>(Vl + row * D + c0, vf);
 #pragma unroll
@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(kPromptThreads) prompt_generic_kernel(const __
         const int dst = kept_before(keepmask, prefix, j);
         const uint4* ks = reinterpret_cast<const uint4*>(Kp + (size_t)j * D);
         const uint4* vs = reinterpret_cast<const uint4*>(Vp + (size_t)j * D);
-        const size_t drow = kv_row(pt_u, (size_t)u * p.C, dst);
+        const size_t drow = kv_row(pt_u, (size_t)u * p.C, dst, p.pool_pages, p.status);
         uint4* kd = reinterpret_cast<uint4*>(Kl + drow * D);
         uint4* vd = reinterpret_cast<uint4*>(Vl + drow * D);
         for (int c = lane; c < 2 * kChunks; c += 32) {

@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
             const int j = j0 + x;
             const bool kept = j < P && ((keepmask[j >> 5] >> (j & 31)) & 1u);
             dst[x] = kept ? kept_before(keepmask, prefix, j) : -1;
-            drow[x] = !kept ? 0 : paged ? (size_t)(pt_sm[dst[x] >> 5] - 1) * kPageKeys + (dst[x] & 31) : (size_t)u * p.C + dst[x];
+            drow[x] = !kept ? 0 : paged ? page_row(pt_sm[dst[x] >> 5], dst[x], p.pool_pages, p.status) : (size_t)u * p.C + dst[x];
             if (kept) buf[x] = __ldg(reinterpret_cast<const uint4*>((lane < 16 ? Kp : Vp) + (size_t)j * kRowBytes) + (lane & 15));
         }
 #pragma unroll

@@ -124,12 +124,13 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
 #pragma unroll
                 for (int g = 0; g < G; ++g) imp |= (sv[k][g] >= s_thr[g]);
                 const uint32_t wd = update_register(wv[k], imp, p.w, t);
-                wordu[j] = wd;
+                if (CORM_IN_RANGE(j < p.C, p.status)) wordu[j] = wd;
                 keep = !evict_on || register_needed(wd, p.w, t) || pv[k] > t - p.r;
                 n_imp += imp ? 1 : 0;
             }
             const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
-            if (lane == 0 && base + warp * 32 < l) keep_g[(base >> 5) + warp] = ballot;
+            if (lane == 0 && base + warp * 32 < l && CORM_IN_RANGE((base >> 5) + warp < keepmask_words(p.C), p.status))
+                keep_g[(base >> 5) + warp] = ballot;
         }
     }
 
@@ -208,8 +209,8 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
             const size_t slab_row0 = (size_t)u * p.C;
             block_move_rows<T, D, NT>(reinterpret_cast<T*>(p.K), reinterpret_cast<T*>(p.V),
                                       [&](int slot) -> size_t {
-                                          return pt_u ? (size_t)(pt_sm[slot >> 5] - 1) * kPageKeys + (slot & 31) : slab_row0 + (size_t)slot;
-                                      }, wordu, posu, movers, holes, n_moved);
+                                          return pt_u ? page_row(pt_sm[slot >> 5], slot, p.pool_pages, p.status) : slab_row0 + (size_t)slot;
+                                      }, wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
         }
     }
     settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l_old, new_len);

@@ -168,6 +168,42 @@ def test_multi_layer_independent_and_deterministic():
     assert 2 * 3 + 3 * cfg.steps <= n <= 2 * 3 + 2 * 3 * cfg.steps and n == gpu2.corm_cache_kernel_launches()
 
 
+def test_all_layers_from_one_call_equal_per_layer_calls():
+    """corm_decode_step_layers is n per-layer calls in layer order: identical output bits and states, checked against
+    the oracle as well; pointer tables built once per step; bad arguments enqueue nothing."""
+    from paper_2404_15949_b200.binding import CormError
+    cfg = CONFIGS[2].with_(n_layers=4, n_q_heads=4, n_kv_heads=4, prompt_min=260, prompt_max=260, steps=10,
+                           recent_r=32, dense_layers=1)
+    one, many = make_gpu_cache(cfg, 1, 4, n_layers=4), make_gpu_cache(cfg, 1, 4, n_layers=4)
+    orc = make_oracle(cfg, 1, 4, n_layers=4)
+    datas = [generate(cfg, layer=l) for l in range(4)]
+    dt = cfg.dtype
+    for l, d in enumerate(datas):
+        for g in (one, many):
+            g.corm_compress_prompt(l, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+        orc.compress_prompt(l, d.k_prompt, d.v_prompt, d.q_last, d.prompt_lens)
+    for s in range(cfg.steps):
+        q = [to_dev(d.q[s], dt) for d in datas]
+        k = [to_dev(d.k_new[s], dt) for d in datas]
+        v = [to_dev(d.v_new[s], dt) for d in datas]
+        outs = [torch.empty_like(x) for x in q]
+        if s % 2:                                                      # tensors one step, address tables the next
+            many.corm_decode_step_layers(0, q, k, v, outs)
+        else:
+            many.corm_decode_step_layers(0, many.pointer_table(q, "q"), many.pointer_table(k, "kv"),
+                                         many.pointer_table(v, "kv"), many.pointer_table(outs, "q"))
+        for l in range(4):
+            a = one.corm_decode_step(l, q[l], k[l], v[l])
+            assert torch.equal(a, outs[l])
+            assert np.abs(a.float().cpu().numpy() - orc.decode_step(l, datas[l].q[s], datas[l].k_new[s], datas[l].v_new[s])).max() <= OUT_TOL[dt]
+    for l in range(4):
+        assert_states_equal(many, orc, l, 1, 4, f"layer {l}")
+    before = many.corm_cache_kernel_launches()
+    with pytest.raises(CormError):
+        many.corm_decode_step_layers(2, q, k, v, outs)                 # layers 2..5 of 4
+    assert many.corm_cache_kernel_launches() == before
+
+
 WIDE = [
     # dtype, d, G, n_kv, B, prompt range, steps, w, r, split_len, fast, alpha, seed
     ("bf16", 128, 1, 4, 2, (300, 520), 80, 40, 16, 0, True, 1.0, 4242),      # tiled prompt pass, one launch pair
