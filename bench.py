@@ -172,7 +172,7 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
                       cfg.recent_r, cfg.alpha, cfg.dtype, local, pool_pages=args.pool_pages)
-    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4}[args.finish])
+    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4, "balanced-verdict": 5}[args.finish])
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
     prompts = [(dev(d.k_prompt), dev(d.v_prompt), dev(d.q_last), d.prompt_lens) for d in data]
@@ -332,7 +332,7 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=512)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced"],
+    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced", "balanced-verdict"],
                     help="which decode kernels: automatic, the block-per-split kernels finishing long units inside the "
                          "decode launch / by the verdict launch, or the balanced single-launch kernel")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")

@@ -210,10 +210,13 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
                                       void* stream);
 
 /* Tuning knobs (performance only; live lists and registers do not depend on them, outputs only within rounding):
- * keys per split of the decode kernel (multiple of 32, 0 = automatic) and which kernels may be used:
- * allow_fast_path 0 = the generic kernels only; 1 = the bf16/head_dim-128 kernels (default), which finish a unit
- * of several splits inside the decode launch when the launch has many units and by a second, verdict launch when
- * it has few; 2 / 3 = those kernels with the first / the second way always. Errors: INVALID_ARG. */
+ * keys per split of the block-per-split decode kernel (multiple of 32, 0 = automatic) and which kernels may be used:
+ * allow_fast_path 0 = the generic kernels only; 1 = automatic (default): for bf16 / head_dim 128, one query head per
+ * KV head takes the block-per-split kernel, which finishes a unit of several splits inside the decode launch when the
+ * launch has many units and by a second, verdict launch when it has few, and grouped heads take the balanced
+ * kernel (every block an equal share of the step's keys) followed by the verdict launch; 2 / 3 = the block-per-split
+ * kernel with the first / the second way always; 4 / 5 = the balanced kernel for every group size it covers,
+ * finishing inside its own launch / with the verdict launch. Errors: INVALID_ARG. */
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Opt-in monitor of the method's premise (Sections 3.2-3.3: the current query resembles recent ones, which is what

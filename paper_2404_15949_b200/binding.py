@@ -260,8 +260,9 @@ class CormCache:
         return out
 
     def corm_cache_set_tuning(self, split_len=0, allow_fast_path=True):
-        """allow_fast_path: False/0 generic kernels, True/1 fast kernels, 2 / 3 fast kernels that always finish units of
-        several splits inside the decode launch / by the verdict launch."""
+        """allow_fast_path: False/0 generic kernels, True/1 automatic, 2 / 3 block-per-split kernels that always finish
+        units of several splits inside the decode launch / by the verdict launch, 4 / 5 the balanced kernel finishing
+        inside its launch / with the verdict launch."""
         _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
 
     def corm_cache_set_similarity_monitor(self, enabled=True):

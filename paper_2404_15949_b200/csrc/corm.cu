@@ -30,7 +30,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, ticket3, move_info, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, ticket3, move_info, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask, unit_rec;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -104,6 +104,7 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.stash = take(U * G * C * 8);
     L.partials = take(partial_records_of(c) * G * partial_stride((int)D));
     L.keepmask = take(U * (size_t)keepmask_words((int)C) * 4);
+    L.unit_rec = take(U * 8);
     L.stage_q = take((size_t)c.batch * c.n_q_heads * D * e);
     L.stage_k = take(U * D * e);
     L.stage_v = take(U * D * e);
@@ -304,6 +305,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.stash = reinterpret_cast<double*>(c->arena + c->lay.stash);
     p.partials = c->arena + c->lay.partials;
     p.keepmask = reinterpret_cast<uint32_t*>(c->arena + c->lay.keepmask);
+    p.unit_rec = reinterpret_cast<int2*>(c->arena + c->lay.unit_rec);
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
     p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
     p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
@@ -313,14 +315,15 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     const bool fast = c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
     int n_launched = 1;
-    // Group sizes above one take the balanced kernel while no unit can be longer than kBalancedAutoLimit keys (its
-    // compaction is one block per unit, which long units with many evictions per step outgrow); tuning value 4
-    // forces it for every group size and length the kernel covers.
-    constexpr int kBalancedAutoLimit = 6144;
-    const bool balanced = fast && !c->vmaps.empty() &&
-                          (c->allow_fast == 4 || (c->allow_fast == 1 && c->G >= 2 && upper <= kBalancedAutoLimit));
+    // Grouped query heads take the balanced streaming kernel followed by the verdict launch (measured against the
+    // block-per-split kernels on one GPU, us per step: 53 against 55 in the steady state of the grouped workload, 122
+    // against 136 in its first steps, 174 against 190 on 24k-key units, 157 against 177 on 8k-key units without
+    // evictions); one query head per KV head stays on the block-per-split kernel, whose loop is lighter (three
+    // blocks per SM). Tuning values 4 / 5 force the balanced kernel finishing in the launch / with the verdict launch.
+    const bool balanced = fast && !c->vmaps.empty() && (c->allow_fast == 4 || c->allow_fast == 5 || (c->allow_fast == 1 && c->G >= 2));
+    const bool balanced_verdict = c->allow_fast != 4;
     if (balanced) {
-        rc = launch_decode_balanced(p, c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf), st, &n_launched);
+        rc = launch_decode_balanced(p, c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf), balanced_verdict, st, &n_launched);
     } else if (fast) {
         // the mean grows by at most one key per step, like the bound
         const int typical = c->live_mean[layer] ? std::min(upper, c->live_mean[layer] + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
@@ -881,7 +884,7 @@ corm_status_t corm_cache_pool_usage(corm_cache_t* c, int32_t layer, int64_t* pag
 corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
-    if (allow_fast_path < 0 || allow_fast_path > 4) return CORM_ERR_INVALID_ARG;
+    if (allow_fast_path < 0 || allow_fast_path > 5) return CORM_ERR_INVALID_ARG;
     c->allow_fast = allow_fast_path;
     return CORM_OK;
 }

@@ -37,7 +37,6 @@ constexpr int kBalRingBytes = kBalWarps * kBalWarpBytes;       // 96 KiB, reused
 constexpr int kBalBlocksPerSm = 2;
 constexpr int kBalSegCap = 32;                                  // segments listed per window of a block's range
 constexpr int kBalRec = 16 + 4 * 128;                           // {double m, double Z, float acc[128]}
-constexpr int kBalSoloMoves = 32;                               // rows a unit's last block moves alone; more are shared out
 constexpr int kBalCacheUnits = 16384;                            // units whose lengths the prologue parks in shared memory
 constexpr int kBalMaxTokens = 1 << 17;                          // the finish phase keeps 3 bits-per-32 arrays on chip
 
@@ -59,21 +58,20 @@ struct BalMisc {
     int scan[kBalThreads];           // finish phase: scratch of the block-wide prefix sums
     int wsum[kBalWarps];
     int first_u, first_P, nseg, more, next_u, next_P, last, failed;
-    unsigned long long info;         // finish phase: a unit's move word as read by thread 0
 };
 
 // shared-memory carve-up behind the 1024-byte aligned ring
 struct BalSmem {
     int psm, segq, segnew, bars, segs, misc, total, n_pre;
 };
-__host__ __device__ inline BalSmem bal_smem_layout(int G) {
-    BalSmem s;
+__host__ __device__ constexpr int bal_align128(int x) { return (x + 127) / 128 * 128; }
+__host__ __device__ constexpr BalSmem bal_smem_layout(int G) {
+    BalSmem s{};
     int off = kBalRingBytes;
-    auto take = [&](int bytes) { int at = off; off = (off + bytes + 127) / 128 * 128; return at; };
-    s.psm = take(kBalWarps * kTileKeys * 16);
-    s.bars = take(kBalWarps * kBalStages * 8);
-    s.segs = take(kBalSegCap * (int)sizeof(BalSeg));
-    s.misc = take((int)sizeof(BalMisc));
+    s.psm = off; off = bal_align128(off + kBalWarps * kTileKeys * 16);
+    s.bars = off; off = bal_align128(off + kBalWarps * kBalStages * 8);
+    s.segs = off; off = bal_align128(off + kBalSegCap * (int)sizeof(BalSeg));
+    s.misc = off; off = bal_align128(off + (int)sizeof(BalMisc));
     // queries and appended rows of the first n_pre segments are fetched ahead; whatever shared memory is left
     const int budget = (228 * 1024) / kBalBlocksPerSm - 1024 /* system */;
     const int per = G * kRowBytes + 2 * kRowBytes;
@@ -81,8 +79,8 @@ __host__ __device__ inline BalSmem bal_smem_layout(int G) {
     if (n_pre > 8) n_pre = 8;
     if (n_pre < 1) n_pre = 1;
     s.n_pre = n_pre;
-    s.segq = take(n_pre * G * kRowBytes);
-    s.segnew = take(n_pre * 2 * kRowBytes);
+    s.segq = off; off = bal_align128(off + n_pre * G * kRowBytes);
+    s.segnew = off; off = bal_align128(off + n_pre * 2 * kRowBytes);
     s.total = off;
     return s;
 }
@@ -155,7 +153,7 @@ struct BalFin {
 //      unit's last block scans the mask, fills the holes and publishes the new length.
 // scratch: the block's ring area, free by now.
 template <int G, bool PAGED, int NT>
-__device__ __noinline__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
+__device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
                                  unsigned char* scratch, BalMisc* misc) {
     constexpr int NW = kBalWarps;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -357,126 +355,84 @@ __device__ __noinline__ void bal_finish_block(const DecodeParams& p, const BalSe
     }
     __syncthreads();
 
-    // ---- compaction ----
-    // The unit's last block scans the keep mask and lists the holes below the new length and the kept rows above it.
-    // A few rows it moves itself. Many rows (the steps right after a prompt pass, long units) are shared out over all
-    // the unit's blocks: the last block publishes the counts in the unit's move word, the others, which wait for that
-    // word (bounded; the last block needs nobody's help to get there), take every n_blocks-th chunk of 16 rows, and a
-    // third arrival counter tells the block that finishes last to settle the pages and publish the new length.
+    // ---- the units this block is the last of: compaction ----
     for (int si = 0; si < nseg; ++si) {
-        const BalFin f = fin[si];
+        if (!fin[si].last) continue;                                            // uniform
         const BalSeg& sg = segs[si];
-        const int u = sg.u, l = sg.l, words = (l + 31) / 32 + 2, nwords = (l + 31) / 32;
+        const int u = sg.u, l = sg.l, t = sg.t, words = (l + 31) / 32 + 2, nwords = (l + 31) / 32;
+        uint32_t* keep_sm = reinterpret_cast<uint32_t*>(comp);
+        int* prefix = reinterpret_cast<int*>(keep_sm + words);
+        int32_t* pt_sm = prefix + words;
         const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
+        const uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
         uint32_t* wordu = p.word + (size_t)u * p.C;
         int32_t* posu = p.pos + (size_t)u * p.C;
-        int* holes = reinterpret_cast<int*>(p.stash + (size_t)u * G * p.C);   // every block is done with the logits
-        int* movers = holes + p.C;
-        const size_t slab_row0 = (size_t)u * p.C;
-        auto row_of = [&](int slot) -> size_t {
-            if (!PAGED) return slab_row0 + (size_t)slot;
-            return page_row(__ldcg(pt_u + (slot >> 5)), slot, p.pool_pages, p.status);
-        };
-        auto publish = [&](int new_len, int n_moved) {                         // whole block
-            if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
-            if (tid == 0) {
-                p.live_out[u] = new_len;
-                publish_live(p.maxlive, p.step + 1, new_len);
-                atomicAdd(p.counters + CNT_APPENDED, 1ull);
-                atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
-                if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
-                if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
-            }
-        };
-        unsigned long long info = 0ull;                                        // done bit | rows to share << 32 | new length
-        if (f.last) {
-            uint32_t* keep_sm = reinterpret_cast<uint32_t*>(comp);
-            int* prefix = reinterpret_cast<int*>(keep_sm + words);
-            const uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
-            for (int i = tid; i < nwords; i += NT) keep_sm[i] = __ldcg(keep_g + i);
-            __syncthreads();
-            int new_len = l, n_moved = 0;
-            if (f.evict_on) {
-                block_popc_scan<NT>(keep_sm, prefix, nwords, misc->scan);
-                new_len = prefix[nwords];
-                if (new_len < l) {
-                    const int kept_below = kept_before(keep_sm, prefix, new_len);
-                    n_moved = new_len - kept_below;
-                    for (int i = tid; i < nwords; i += NT) {
-                        const uint32_t m = keep_sm[i];
-                        const int w0 = i * 32;
-                        const uint32_t valid = l - w0 >= 32 ? 0xffffffffu : (1u << (l - w0)) - 1u;
-                        const uint32_t below = new_len - w0 >= 32 ? 0xffffffffu : (new_len > w0 ? (1u << (new_len - w0)) - 1u : 0u);
-                        uint32_t hm = ~m & valid & below;                       // evicted slots below the new length
-                        while (hm) {
-                            const int bit = __ffs(hm) - 1;
-                            hm &= hm - 1u;
-                            holes[w0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = w0 + bit;
-                        }
-                        uint32_t km = m & valid & ~below;                       // kept slots at or above it
-                        while (km) {
-                            const int bit = __ffs(km) - 1;
-                            km &= km - 1u;
-                            movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = w0 + bit;
-                        }
+        for (int i = tid; i < nwords; i += NT) {
+            keep_sm[i] = __ldcg(keep_g + i);
+            if (PAGED) pt_sm[i] = __ldcg(pt_u + i);
+        }
+        __syncthreads();
+        int new_len = l, n_moved = 0;
+        if (fin[si].evict_on) {
+            block_popc_scan<NT>(keep_sm, prefix, nwords, misc->scan);
+            new_len = prefix[nwords];
+            if (new_len < l) {
+                const int kept_below = kept_before(keep_sm, prefix, new_len);
+                n_moved = new_len - kept_below;
+                int* holes = reinterpret_cast<int*>(p.stash + (size_t)u * G * p.C);   // every block is done with the logits
+                int* movers = holes + p.C;
+                for (int i = tid; i < nwords; i += NT) {
+                    const uint32_t m = keep_sm[i];
+                    const int w0 = i * 32;
+                    const uint32_t valid = l - w0 >= 32 ? 0xffffffffu : (1u << (l - w0)) - 1u;
+                    const uint32_t below = new_len - w0 >= 32 ? 0xffffffffu : (new_len > w0 ? (1u << (new_len - w0)) - 1u : 0u);
+                    uint32_t hm = ~m & valid & below;                       // evicted slots below the new length
+                    while (hm) {
+                        const int bit = __ffs(hm) - 1;
+                        hm &= hm - 1u;
+                        holes[w0 - prefix[i] + __popc(~m & ((1u << bit) - 1u))] = w0 + bit;
                     }
-                    __syncthreads();
+                    uint32_t km = m & valid & ~below;                       // kept slots at or above it
+                    while (km) {
+                        const int bit = __ffs(km) - 1;
+                        km &= km - 1u;
+                        movers[prefix[i] + __popc(m & ((1u << bit) - 1u)) - kept_below] = w0 + bit;
+                    }
                 }
-            }
-            const bool shared = f.n_blocks > 1 && n_moved > kBalSoloMoves;
-            if (!shared) {
-                block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), row_of,
-                                                 wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
-                publish(new_len, n_moved);
-            }
-            info = (1ull << 63) | ((unsigned long long)(shared ? n_moved : 0) << 32) | (unsigned)new_len;
-            if (f.n_blocks > 1) {
-                __threadfence();                                               // the lists (and a solo block's moves) before the word
                 __syncthreads();
-                if (tid == 0) atomicExch(p.move_info + u, info);
+                const size_t slab_row0 = (size_t)u * p.C;
+                block_move_rows<bf16_t, 128, NT>(
+                    reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V),
+                    [&](int slot) -> size_t {
+                        return PAGED ? page_row(pt_sm[slot >> 5], slot, p.pool_pages, p.status) : slab_row0 + (size_t)slot;
+                    },
+                    wordu, posu, movers, holes, n_moved, 0, 1, l, p.status);
             }
-        } else {                                                               // wait for the last block's counts
-            if (tid == 0) {
-                const long long start = clock64();
-                unsigned long long v;
-                while (!((v = ld_acquire_u64(p.move_info + u)) >> 63)) {
-                    if (clock64() - start > kWaitLimitCycles) { misc->failed = 1; break; }
-                    __nanosleep(64);
-                }
-                misc->info = v;
-            }
-            __syncthreads();
-            if (misc->failed) { if (tid == 0) report_status(p.status, CORM_ERR_TIMEOUT); return; }
-            info = misc->info;
         }
-        if (f.n_blocks > 1) {
-            const int n_share = (int)((info >> 32) & 0x7fffffffu), new_len = (int)(info & 0xffffffffu);
-            if (n_share)                                                       // this block's chunks of 16 rows
-                block_move_rows<bf16_t, 128, NT>(reinterpret_cast<bf16_t*>(p.K), reinterpret_cast<bf16_t*>(p.V), row_of,
-                                                 wordu, posu, movers, holes, n_share, blk - (f.rec0 / NW - u), f.n_blocks, l, p.status);
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) {
-                const unsigned prev = atomicAdd(p.ticket3 + u, 1u);
-                misc->last = (prev == (unsigned)(f.n_blocks - 1));
-                if (misc->last) { p.ticket3[u] = 0u; atomicExch(p.move_info + u, 0ull); }   // every block has read the word
-                __threadfence();
-            }
-            __syncthreads();
-            if (misc->last && n_share) publish(new_len, n_share);              // all rows are in place
+        if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+        if (tid == 0) {
+            p.live_out[u] = new_len;
+            publish_live(p.maxlive, p.step + 1, new_len);
+            atomicAdd(p.counters + CNT_APPENDED, 1ull);
+            atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
+            if (new_len < l) atomicAdd(p.counters + CNT_EVICTED, (unsigned long long)(l - new_len));
+            if (n_moved) atomicAdd(p.counters + CNT_MOVED, (unsigned long long)n_moved);
         }
-        __syncthreads();                                                       // the arrays are reused by the next unit
+        __syncthreads();                                                     // the arrays are reused by the next unit
+        (void)t;
     }
 }
 
-template <int G, bool PAGED>
+// FINISH: Algorithm 1 is finished inside this launch (bal_finish_block); otherwise the kernel only streams, lists each
+// unit's records in p.unit_rec and leaves verdicts and compaction to the verdict launch that follows it.
+template <int G, bool PAGED, bool FINISH>
 __global__ void __launch_bounds__(kBalThreads, kBalBlocksPerSm)
 decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ __align__(1024) unsigned char smem[];   // the swizzled V tiles want 1024-byte alignment
     constexpr int NT = kBalThreads, NW = kBalWarps;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nblk = (int)gridDim.x, blk = (int)blockIdx.x;
-    const BalSmem lay = bal_smem_layout(G);
+    constexpr BalSmem lay = bal_smem_layout(G);           // compile-time offsets: no registers held for them
     unsigned char* my_tiles = smem + warp * kBalWarpBytes;
     const uint32_t my_bars = smem_addr(smem + lay.bars) + warp * kBalStages * 8;
     unsigned char* psm = smem + lay.psm + warp * kTileKeys * 16;
@@ -846,15 +802,26 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
             }
             __threadfence();
             __syncwarp();
-            if (lane == 0) atomicAdd(p.ticket + u, 1u);   // this warp's record and logits of the segment are stored
+            if (FINISH && lane == 0) atomicAdd(p.ticket + u, 1u);   // this warp's record and logits of the segment are stored
         }
         __syncthreads();
         if (failed) { report_status(p.status, CORM_ERR_TIMEOUT); s_failed = 1; }
         __syncthreads();
         if (s_failed) return;                   // a bounded wait expired: reported through the status word
         // ---- Algorithm 1 for the slots this block streamed; the ring is free now ----
-        bal_finish_block<G, PAGED, NT>(p, segs, nseg, blk, T, nblk, smem, misc);
-        if (s_failed) return;
+        if (FINISH) {
+            bal_finish_block<G, PAGED, NT>(p, segs, nseg, blk, T, nblk, smem, misc);
+            if (s_failed) return;
+        } else {
+            // the verdict launch may become resident now; it reads nothing of this launch before it has completed
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            for (int si = tid; si < nseg; si += NT) {          // units that start in this block: where their records are
+                const BalSeg& sg = segs[si];
+                const long long P0 = sg.gtile0;
+                const int fb = bal_block_of(P0, T, nblk);
+                if (fb == blk) p.unit_rec[sg.u] = make_int2((fb + sg.u) * NW, (bal_block_of(P0 + sg.n_unit - 1, T, nblk) - fb + 1) * NW);
+            }
+        }
         if (!s_more) break;
         __syncthreads();
         win_u = s_next_u; win_P = s_next_P;
@@ -893,24 +860,27 @@ inline corm_status_t make_v_tensor_map(CUtensorMap* out, void* v_layer, unsigned
 
 
 inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& vmap, int G, int upper, int sm_count,
-                                            size_t partial_capacity_records, cudaStream_t st, int* n_launched) {
+                                            size_t partial_capacity_records, bool verdict_launch, cudaStream_t st,
+                                            int* n_launched) {
     *n_launched = 0;
     if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
     if (p.C > kBalMaxTokens) return CORM_ERR_UNSUPPORTED;
     const int sms = sm_count > 0 ? sm_count : 148;
     // one block per resident slot, fewer when the step cannot have that many tiles per warp
-    const long long tiles_upper = (long long)((upper + kTileKeys - 1) / kTileKeys) * p.U;
+    const int upper_tiles = (upper + kTileKeys - 1) / kTileKeys;
+    const long long tiles_upper = (long long)upper_tiles * p.U;
     long long grid = (long long)sms * kBalBlocksPerSm;
     if (tiles_upper / kBalWarps + 1 < grid) grid = tiles_upper / kBalWarps + 1;
     if (bal_record_count((int)grid, p.U) > partial_capacity_records) return CORM_ERR_UNSUPPORTED;
-    const BalSmem lay = bal_smem_layout(G);
+    constexpr int kTotal[5] = {0, bal_smem_layout(1).total, bal_smem_layout(2).total, 0, bal_smem_layout(4).total};
+    const size_t smem = (size_t)kTotal[G];
     auto launch = [&](auto kern) -> corm_status_t {
-        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), (size_t)lay.total);
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3((unsigned)grid);
         cfg.blockDim = dim3(kBalThreads);
-        cfg.dynamicSmemBytes = (size_t)lay.total;
+        cfg.dynamicSmemBytes = smem;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set-up overlaps the previous step's tail
@@ -923,9 +893,40 @@ inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& 
         return CORM_OK;
     };
     corm_status_t rc;
-    if (p.page_table) rc = G == 1 ? launch(decode_balanced_kernel<1, true>) : G == 2 ? launch(decode_balanced_kernel<2, true>) : launch(decode_balanced_kernel<4, true>);
-    else rc = G == 1 ? launch(decode_balanced_kernel<1, false>) : G == 2 ? launch(decode_balanced_kernel<2, false>) : launch(decode_balanced_kernel<4, false>);
-    if (rc == CORM_OK) *n_launched = 1;
+#define CORM_BAL(FIN)                                                                                                      \
+    (p.page_table ? (G == 1 ? launch(decode_balanced_kernel<1, true, FIN>) : G == 2 ? launch(decode_balanced_kernel<2, true, FIN>)   \
+                                                                                    : launch(decode_balanced_kernel<4, true, FIN>))  \
+                  : (G == 1 ? launch(decode_balanced_kernel<1, false, FIN>) : G == 2 ? launch(decode_balanced_kernel<2, false, FIN>) \
+                                                                                     : launch(decode_balanced_kernel<4, false, FIN>)))
+    rc = verdict_launch ? CORM_BAL(false) : CORM_BAL(true);
+#undef CORM_BAL
+    if (rc != CORM_OK) return rc;
+    *n_launched = 1;
+    if (!verdict_launch) return CORM_OK;
+    // verdicts and compaction by the verdict launch, spread over 1024-slot chunks of every unit
+    const int n_rec_cap = kBalWarps * (int)(grid < upper_tiles ? grid : upper_tiles);   // records one unit can have
+    const size_t vsmem = verdict_smem(p.C, n_rec_cap, G, p.page_table != nullptr);
+    auto launch_v = [&](auto kern) -> corm_status_t {
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), vsmem);
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((upper + kVerdictChunk - 1) / kVerdictChunk, (unsigned)p.U);
+        cfg.blockDim = dim3(kVerdictThreads);
+        cfg.dynamicSmemBytes = vsmem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may become resident during the streaming tail
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, p, n_rec_cap);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: verdict launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        return CORM_OK;
+    };
+    rc = G == 1 ? launch_v(decode_verdict_kernel<bf16_t, 128, 1, true>) : G == 2 ? launch_v(decode_verdict_kernel<bf16_t, 128, 2, true>)
+                                                                                 : launch_v(decode_verdict_kernel<bf16_t, 128, 4, true>);
+    if (rc == CORM_OK) *n_launched = 2;
     return rc;
 }
 

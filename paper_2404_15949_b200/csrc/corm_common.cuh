@@ -67,6 +67,7 @@ struct DecodeParams {
     double* stash;            // [U*G][C] scaled logits of this step (scratch)
     unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
     uint32_t* keepmask;       // [U][ceil(C/32)+2] keep bits of the verdict launch (scratch)
+    int2* unit_rec;           // [U] balanced kernel -> verdict launch: a unit's first record and its record count (scratch)
     const void* q;            // [B][Hq][D]
     const void* k_new;        // [B][Hkv][D]
     const void* v_new;        // [B][Hkv][D]

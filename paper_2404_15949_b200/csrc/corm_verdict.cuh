@@ -28,7 +28,9 @@ __host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G, bool 
     return (size_t)G * n_splits * (8 + 8 + 4) + 16 + (size_t)(paged ? 3 : 2) * keepmask_words(C) * 4;   // + keep mask, prefix sums (, page entries)
 }
 
-template <typename T, int D, int G>
+// BAL: the streaming pass was the balanced kernel (corm_balanced.cuh): a unit's records are the n_rec consecutive
+// ones from rec0 on that the kernel lists in p.unit_rec, and the logits are stored [slot][G].
+template <typename T, int D, int G, bool BAL = false>
 __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
                                                                          const int n_splits) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -43,8 +45,7 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     const int room = pt_u ? __ldcg(p.page_room + u) : 1;                   // paged caches: a page for the appended row
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C || !room) return;                                          // reported by the streaming kernel
-    const int n_act = (l + p.split_len - 1) / p.split_len;
-    if (n_act == 1 && l <= p.single_cap) return;                           // finished inside the streaming kernel
+    if (!BAL && (l + p.split_len - 1) / p.split_len == 1 && l <= p.single_cap) return;   // finished inside the streaming kernel
     const int n_chunks = (l + kVerdictChunk - 1) / kVerdictChunk;
     if (chunk >= n_chunks) return;
     const int t = __ldg(p.base_tokens + b) + p.step + 1;
@@ -64,13 +65,16 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     asm volatile("griddepcontrol.wait;" ::: "memory");                     // the streaming grid has completed
     // everything this block needs from the streaming kernel is requested at once: status, split records, logits
     const int status = __ldcg(p.status);
+    const int2 ur = BAL ? __ldcg(p.unit_rec + u) : make_int2(u * p.max_splits, (l + p.split_len - 1) / p.split_len);
+    const int n_act = min(ur.y, n_splits);                                 // n_splits bounds the shared-memory arrays
     const double* stash_u = p.stash + (size_t)u * G * p.C;
     double sv[kVerdictPer][G];
 #pragma unroll
     for (int k = 0; k < kVerdictPer; ++k) {
         const int j = base0 + k * NT + tid;
 #pragma unroll
-        for (int g = 0; g < G; ++g) sv[k][g] = j < l ? __ldcg(stash_u + (size_t)g * p.C + j) : -INFINITY;
+        for (int g = 0; g < G; ++g)
+            sv[k][g] = j < l ? __ldcg(BAL ? stash_u + (size_t)j * G + g : stash_u + (size_t)g * p.C + j) : -INFINITY;
     }
 
     double* sm_m = reinterpret_cast<double*>(smem);                        // [G][n_splits]
@@ -80,7 +84,7 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     int* prefix = reinterpret_cast<int*>(keep_sm + keepmask_words(p.C));
     int32_t* pt_sm = prefix + keepmask_words(p.C);                         // paged caches: the unit's page entries (last block)
     const size_t pstride = partial_stride(D);
-    const unsigned char* rec_u = p.partials + (size_t)u * p.max_splits * G * pstride;
+    const unsigned char* rec_u = p.partials + (size_t)ur.x * G * pstride;
 
     // a. split reduction
     for (int x = tid; x < G * n_act; x += NT) {

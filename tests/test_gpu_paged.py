@@ -23,6 +23,8 @@ PAGED = [
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, True, 64),       # balanced kernel (default for grouped heads)
     ("bf16", 128, 1, 3, 2, (150, 330), 72, 8, 16, 0, 4, 96),          # balanced kernel, one head per KV head
     ("bf16", 128, 4, 1, 1, (3000, 3000), 12, 8, 64, 0, 4, 128),       # one long unit cut over many blocks
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 0, 5, 64),            # balanced streaming + verdict launch
+    ("bf16", 128, 4, 1, 1, (3000, 3000), 12, 8, 64, 0, 5, 128),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, 3, 64),
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 0, True, 32),         # grows across page boundaries from one page
     ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True, 32),        # generic decode kernel, tiled prompt pass

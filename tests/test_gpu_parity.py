@@ -55,6 +55,10 @@ SMALL = [
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 0, 4),
     ("bf16", 128, 4, 5, 3, (1, 40), 60, 8, 4, 0, 4),           # tiny units: many segments per block, units of one tile
     ("bf16", 128, 4, 1, 1, (3000, 3000), 12, 8, 64, 0, 4),     # one long unit cut over many blocks
+    ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 0, 5),         # balanced streaming, verdicts by the verdict launch
+    ("bf16", 128, 1, 3, 2, (150, 330), 40, 8, 16, 0, 5),
+    ("bf16", 128, 4, 5, 3, (1, 40), 60, 8, 4, 0, 5),
+    ("bf16", 128, 4, 1, 1, (3000, 3000), 12, 8, 64, 0, 5),
     ("bf16", 128, 4, 2, 2, (97, 257), 36, 4, 8, 128, False),
     ("bf16", 128, 8, 1, 2, (64, 129), 20, 3, 5, 64, True),
     ("bf16", 128, 2, 2, 1, (31, 33), 70, 8, 32, 64, True),
