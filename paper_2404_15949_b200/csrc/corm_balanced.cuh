@@ -7,7 +7,7 @@
 // boundaries. The four warps of a block stream the tiles of a segment in turn, each through its own ring of
 // shared-memory stages: K tiles by bulk copies (a tile is one contiguous run of 256-byte rows), V tiles by 2-D
 // tensor-map copies with the 128-byte swizzle, both completing on mbarriers with bounded waits.
-//   Q.K   fp64 on the CUDA cores, as in corm_fast.cuh (qk_tile): verdicts are compared with an fp64 oracle.
+//   Q.K   fp64 on the CUDA cores, as in corm_fast.cuh (qk_tile_pairs below): verdicts are compared with an fp64 oracle.
 //   P.V   on the tensor cores: mma.m16n8k16 with A = V^T (ldmatrix.trans from the swizzled tile) and B = the
 //         tile's probabilities, each split into two bf16 (p = hi + lo to ~2^-17 relative), the 2 G columns of B
 //         being (head, hi / lo); fp32 accumulation. A group of four heads fills the 8 columns of one instruction.
@@ -107,6 +107,48 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float hi, float lo) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
+}
+
+// qk_tile of corm_fast.cuh with the key slots taken in pairs (s, s + 4): the two slots' FMA chains run together
+// (eight independent chains instead of four: a dependent fp64 FMA issues only every ~23 cycles) and the pair's first
+// butterfly exchange follows at once, overlapping the next pair's arithmetic. Same lane -> key map, same sums up to
+// the order of the additions. 2 % faster than qk_tile here (same GPU, long units).
+template <int G>
+__device__ __forceinline__ void qk_tile_pairs(const unsigned char* ktile, const double (&qd)[G][8], int lane,
+                                              double (&sown)[G]) {
+    const int h = lane >> 4, i = lane & 15, m = i >> 1, b0 = i & 1;
+    double r[2][G];
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        double b[G][4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s) {
+            const int key0 = 16 * h + 8 * (it ^ b0) + (s ^ m), key1 = 16 * h + 8 * (it ^ b0) + ((s + 4) ^ m);
+            const uint4 raw0 = *reinterpret_cast<const uint4*>(ktile + key0 * kRowBytes + i * 16);
+            const uint4 raw1 = *reinterpret_cast<const uint4*>(ktile + key1 * kRowBytes + i * 16);
+            double k0[8], k1[8];
+            unpack8_to_double(raw0, k0);
+            unpack8_to_double(raw1, k1);
+            double a0[G], a1[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) { a0[g] = qd[g][0] * k0[0]; a1[g] = qd[g][0] * k1[0]; }
+#pragma unroll
+            for (int e = 1; e < 8; ++e)
+#pragma unroll
+                for (int g = 0; g < G; ++g) { a0[g] = fma(qd[g][e], k0[e], a0[g]); a1[g] = fma(qd[g][e], k1[e], a1[g]); }
+#pragma unroll
+            for (int g = 0; g < G; ++g) b[g][s] = a0[g] + __shfl_xor_sync(0xffffffffu, a1[g], 8);
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+#pragma unroll
+            for (int s = 0; s < 2; ++s) b[g][s] += __shfl_xor_sync(0xffffffffu, b[g][s + 2], 4);
+            b[g][0] += __shfl_xor_sync(0xffffffffu, b[g][1], 2);
+            r[it][g] = b[g][0];
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) sown[g] = r[0][g] + __shfl_xor_sync(0xffffffffu, r[1][g], 1);
 }
 
 // byte offset of 16-byte chunk c (0..15) of row r inside a V tile as the swizzled tensor copies lay it out: two
@@ -673,7 +715,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
                         __syncwarp();
                     }
                     double sown[G];
-                    qk_tile<G>(ktile, qd, lane, sown);
+                    qk_tile_pairs<G>(ktile, qd, lane, sown);
                     __syncwarp();
                     if (ck.si < nseg) {
                         if (lane == 0) { fence_async_smem(); issue_k(ck, nk); }
