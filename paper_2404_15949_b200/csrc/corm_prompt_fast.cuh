@@ -315,7 +315,6 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
         // verdicts of this launch's queries for the lane's key: a bit per window slot (bit w-1-rho) when the window
         // fits a shift register, else the position of the newest query that found the key important
         uint32_t reg = 0u;
-        int n_near = 0;                                   // logits inside the fp32 bound, placed again in fp64
         for (int gi = 0; gi < groups; ++gi) {
             if (slot0 + (4 * gi + 3) / G < w - wp) continue;                      // none of these queries exists
             // The thresholds are exact (fp64, from the first launch), so a logit only has to be placed on one side of
@@ -336,7 +335,7 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
                     if (margin >= err) imp = true;
                     else if (!(margin < -err)) {
                         imp = exact_logit(q_sm + (size_t)r * 128, Kp + (size_t)(k0 + key_own) * kRowBytes) * inv_root_d >= thr_sm[r];
-                        ++n_near;
+                        atomicAdd(p.counters + CNT_NEAR, 1ull);      // rare: a few hundred per pass
                     }
                 }
                 // Definition 3.1 in log form; keys newer than the query keep a 0 bit (Algorithm 1's zero padding)
@@ -346,7 +345,6 @@ __global__ void __launch_bounds__(kPromptFastThreads) prompt_verdict_kernel(cons
                 }
             }
         }
-        warp_count(p.counters + CNT_NEAR, n_near);
         if (key_own < n_valid) {
             uint32_t* dst = tmp_word + k0 + key_own;
             if (slot0 == 0) *dst = reg;                                            // first launch of the window
