@@ -945,14 +945,15 @@ inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& 
     if (rc != CORM_OK) return rc;
     *n_launched = 1;
     if (!verdict_launch) return CORM_OK;
-    // verdicts and compaction by the verdict launch, spread over 1024-slot chunks of every unit
+    // verdicts and compaction by the verdict launch, spread over 1024- or 2048-slot chunks of every unit
     const int n_rec_cap = kBalWarps * (int)(grid < upper_tiles ? grid : upper_tiles);   // records one unit can have
     const size_t vsmem = verdict_smem(p.C, n_rec_cap, G, p.page_table != nullptr);
     auto launch_v = [&](auto kern) -> corm_status_t {
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), vsmem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((upper + kVerdictChunk - 1) / kVerdictChunk, (unsigned)p.U);
+        const int batches = verdict_batches(upper, p.U, sms);
+        cfg.gridDim = dim3((upper + batches * kVerdictBatch - 1) / (batches * kVerdictBatch), (unsigned)p.U);
         cfg.blockDim = dim3(kVerdictThreads);
         cfg.dynamicSmemBytes = vsmem;
         cfg.stream = st;
@@ -961,7 +962,7 @@ inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& 
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, kern, p, n_rec_cap);
+        e = cudaLaunchKernelEx(&cfg, kern, p, n_rec_cap, batches);
         if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: verdict launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;

@@ -696,7 +696,8 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
         cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), vsmem);
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3((upper + kVerdictChunk - 1) / kVerdictChunk, (unsigned)p.U);
+        const int batches = verdict_batches(upper, p.U, sms);
+        cfg.gridDim = dim3((upper + batches * kVerdictBatch - 1) / (batches * kVerdictBatch), (unsigned)p.U);
         cfg.blockDim = dim3(kVerdictThreads);
         cfg.dynamicSmemBytes = vsmem;
         cfg.stream = st;
@@ -705,7 +706,7 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, kern, p, n_splits);
+        e = cudaLaunchKernelEx(&cfg, kern, p, n_splits, batches);
         if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) { std::fprintf(stderr, "corm: verdict launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
         return CORM_OK;

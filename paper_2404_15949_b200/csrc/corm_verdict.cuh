@@ -2,7 +2,7 @@
 // (Algorithm 1's verdict row, register update, keep decision, compaction), spread over many blocks instead of one.
 //
 // The streaming kernel leaves, per unit, one partial record {m, Z, acc[D]} per split and query head and the scaled
-// logits of every live key. Here a block owns 1024 consecutive slots of one unit:
+// logits of every live key. Here a block owns 1024 or 2048 consecutive slots of one unit (one or two batches):
 //   a. every block reduces the (m, Z) of the unit's splits to lse_g and the threshold of Definition 3.1 in log form
 //      (a few dozen values; the same arithmetic in the same order in every block, so all blocks agree bit for bit);
 //      block 0 of the unit also reduces the accumulators to the attention output of Eq. 1;
@@ -19,8 +19,17 @@
 namespace corm {
 
 constexpr int kVerdictThreads = 256;
-constexpr int kVerdictChunk = 1024;                       // slots per block
-constexpr int kVerdictPer = kVerdictChunk / kVerdictThreads;
+constexpr int kVerdictPer = 4;                            // slots per thread and batch
+constexpr int kVerdictBatch = kVerdictThreads * kVerdictPer;
+constexpr int kVerdictMaxBatches = 2;                     // a block judges its slots in one or two batches of 1024: with two, the
+                                                          // block's fixed chain of round trips (records, thresholds, arrival) is
+                                                          // paid once per 2048 slots, which pays when one batch per block would
+                                                          // need more than one wave of blocks (long units)
+// batches per block for a launch over units of up to `upper` keys
+inline int verdict_batches(int upper, int n_units, int sm_count) {
+    const long long blocks = (long long)((upper + kVerdictBatch - 1) / kVerdictBatch) * n_units;
+    return blocks > 4ll * sm_count ? kVerdictMaxBatches : 1;
+}
 
 __host__ __device__ inline int keepmask_words(int C) { return (C + 31) / 32 + 2; }
 
@@ -32,7 +41,7 @@ __host__ __device__ inline size_t verdict_smem(int C, int n_splits, int G, bool 
 // ones from rec0 on that the kernel lists in p.unit_rec, and the logits are stored [slot][G].
 template <typename T, int D, int G, bool BAL = false>
 __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(const __grid_constant__ DecodeParams p,
-                                                                         const int n_splits) {
+                                                                         const int n_splits, const int batches) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ double s_thr[G], s_Z[G];
     __shared__ int s_scan[kVerdictThreads];
@@ -46,22 +55,26 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
     if (l > p.C || !room) return;                                          // reported by the streaming kernel
     if (!BAL && (l + p.split_len - 1) / p.split_len == 1 && l <= p.single_cap) return;   // finished inside the streaming kernel
-    const int n_chunks = (l + kVerdictChunk - 1) / kVerdictChunk;
+    const int chunk_slots = batches * kVerdictBatch;
+    const int n_chunks = (l + chunk_slots - 1) / chunk_slots;
     if (chunk >= n_chunks) return;
     const int t = __ldg(p.base_tokens + b) + p.step + 1;
     const int n_obs = min(p.w, __ldg(p.base_obs + b) + p.step + 1);
     const bool evict_on = n_obs >= p.w;
     uint32_t* wordu = p.word + (size_t)u * p.C;
     int32_t* posu = p.pos + (size_t)u * p.C;
-    const int base0 = chunk * kVerdictChunk;
+    const int base0 = chunk * chunk_slots;
     uint32_t wv[kVerdictPer];
     int32_t pv[kVerdictPer];
+    auto load_regs = [&](int bbase) {                                      // registers and positions: not written by the streaming kernel
 #pragma unroll
-    for (int k = 0; k < kVerdictPer; ++k) {                                // the appended slot l_old starts as (0, t)
-        const int j = base0 + k * NT + tid;
-        wv[k] = j < l_old ? __ldcg(wordu + j) : 0u;
-        pv[k] = j < l_old ? __ldcg(posu + j) : t;
-    }
+        for (int k = 0; k < kVerdictPer; ++k) {                            // the appended slot l_old starts as (0, t)
+            const int j = bbase + k * NT + tid;
+            wv[k] = j < l_old ? __ldcg(wordu + j) : 0u;
+            pv[k] = j < l_old ? __ldcg(posu + j) : t;
+        }
+    };
+    load_regs(base0);
     asm volatile("griddepcontrol.wait;" ::: "memory");                     // the streaming grid has completed
     // everything this block needs from the streaming kernel is requested at once: status, split records, logits
     const int status = __ldcg(p.status);
@@ -69,13 +82,16 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     const int n_act = min(ur.y, n_splits);                                 // n_splits bounds the shared-memory arrays
     const double* stash_u = p.stash + (size_t)u * G * p.C;
     double sv[kVerdictPer][G];
+    auto load_logits = [&](int bbase) {
 #pragma unroll
-    for (int k = 0; k < kVerdictPer; ++k) {
-        const int j = base0 + k * NT + tid;
+        for (int k = 0; k < kVerdictPer; ++k) {
+            const int j = bbase + k * NT + tid;
 #pragma unroll
-        for (int g = 0; g < G; ++g)
-            sv[k][g] = j < l ? __ldcg(BAL ? stash_u + (size_t)j * G + g : stash_u + (size_t)g * p.C + j) : -INFINITY;
-    }
+            for (int g = 0; g < G; ++g)
+                sv[k][g] = j < l ? __ldcg(BAL ? stash_u + (size_t)j * G + g : stash_u + (size_t)g * p.C + j) : -INFINITY;
+        }
+    };
+    load_logits(base0);
 
     double* sm_m = reinterpret_cast<double*>(smem);                        // [G][n_splits]
     double* sm_Z = sm_m + (size_t)G * n_splits;
@@ -117,10 +133,13 @@ __global__ void __launch_bounds__(kVerdictThreads, 4) decode_verdict_kernel(cons
     // b. verdicts, register update, keep flags of this block's slots
     uint32_t* keep_g = p.keepmask + (size_t)u * keepmask_words(p.C);
     int n_imp = 0;                                                         // keys this thread judged important
-    {
+    for (int bt = 0; bt < batches; ++bt) {
+        const int bbase = base0 + bt * kVerdictBatch;
+        if (bbase >= l) break;                                             // uniform
+        if (bt) { load_regs(bbase); load_logits(bbase); }
 #pragma unroll
         for (int k = 0; k < kVerdictPer; ++k) {
-            const int base = base0 + k * NT, j = base + tid;
+            const int base = bbase + k * NT, j = base + tid;
             if (base >= l) break;                                          // uniform
             bool keep = false;
             if (j < l) {
