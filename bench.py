@@ -176,12 +176,18 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
     prompts = [(dev(d.k_prompt), dev(d.v_prompt), dev(d.q_last), d.prompt_lens) for d in data]
-    q_d = [dev(d.q) for d in data]
-    k_d = [dev(d.k_new) for d in data]
-    v_d = [dev(d.v_new) for d in data]
-    out = torch.empty_like(q_d[0][0])
+    # [step][layer][...]: the layers' inputs of a step are contiguous, so that a configuration of several layers can be
+    # stepped by one launch (corm_decode_step_layers)
+    q_all = torch.stack([dev(d.q) for d in data], dim=1).contiguous()
+    k_all = torch.stack([dev(d.k_new) for d in data], dim=1).contiguous()
+    v_all = torch.stack([dev(d.v_new) for d in data], dim=1).contiguous()
+    q_d = [q_all[:, l] for l in range(L)]
+    k_d = [k_all[:, l] for l in range(L)]
+    v_d = [v_all[:, l] for l in range(L)]
+    out_all = torch.empty_like(q_all[0])
+    out = out_all[0]
     # per-step views made once: slicing a tensor costs the host several microseconds, as much as a launch
-    views = [[(q_d[l][s], k_d[l][s], v_d[l][s]) for l in range(L)] for s in range(n_steps)]
+    views = [[(q_all[s, l], k_all[s, l], v_all[s, l]) for l in range(L)] for s in range(n_steps)]
 
     def restore():
         """Back to the state right after the prompt pass. Returns the pass's device time (ms)."""
@@ -194,7 +200,7 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
         return a.elapsed_time(b)
 
     # configurations of several layers step them all from one host call; the address tables are built once
-    outs = [torch.empty_like(out) for _ in range(L)]
+    outs = [out_all[l] for l in range(L)]
     if L > 1:
         tabs = [tuple(cache.pointer_table([views[s][l][i] for l in range(L)], "q" if i == 0 else "kv") for i in range(3))
                 for s in range(n_steps)]
@@ -242,7 +248,7 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
     # read and the output written across the bus every step
     e2e_ms, h2d, d2h = None, 0, 0
     if want_e2e:
-        pin = lambda t: t.cpu().pin_memory()
+        pin = lambda t: t.contiguous().cpu().pin_memory()
         qh = [pin(x) for x in q_d]
         kh = [pin(x) for x in k_d]
         vh = [pin(x) for x in v_d]

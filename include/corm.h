@@ -152,10 +152,15 @@ corm_status_t corm_decode_step(corm_cache_t* cache, int32_t layer, const void* q
 /* The same step for n_layers consecutive layers from one host call: layer first_layer + i takes q[i], k_new[i],
  * v_new[i] and writes out[i] (host arrays of device pointers, each as for corm_decode_step). The paper applies the
  * policy "on each head at every layer" (footnote to the Approach paragraph) and the layers of a cache are independent
- * (each has its own token and row counts), so this is exactly n_layers calls of corm_decode_step in layer order on
- * `stream`; it exists because one launch per layer of a single-sequence model is a few microseconds of GPU work and
- * a host call per launch costs more than that. In a model the layers' inputs depend on each other's outputs; use
- * this where they are all known (replay, benchmarking, speculative batches), the per-layer call otherwise.
+ * (each has its own token and row counts), so the result is exactly that of n_layers calls of corm_decode_step in
+ * layer order on `stream` (outputs within rounding: blocks may be cut differently). It exists because one launch per
+ * layer of a single-sequence model is a few microseconds of GPU work behind a chain of launch and memory latencies:
+ * when the layers' buffers are contiguous in layer order (q[i + 1] directly behind q[i], likewise k_new, v_new, out),
+ * the cache is a slab cache on the bf16 / head_dim-128 kernels, and all the layers are at the same step, ALL layers
+ * run as one launch (the layers' units are one array to the kernels); otherwise the per-layer launches are enqueued
+ * one after the other. The step's counters are then added to the first layer's (totals in corm_cache_stats are
+ * the same). In a model the layers' inputs depend on each other's outputs; use this where they are all known
+ * (replay, benchmarking, speculative batches), the per-layer call otherwise.
  * Errors: as corm_decode_step, all arguments and every layer's state checked before anything is enqueued. */
 corm_status_t corm_decode_step_layers(corm_cache_t* cache, int32_t first_layer, int32_t n_layers,
                                       const void* const* q, const void* const* k_new, const void* const* v_new,

@@ -59,8 +59,13 @@ int max_splits_of(const corm_config_t& c) { return (c.max_tokens + kMinSplit - 1
 // Split partial records the arena holds: one per (unit, split) of the block-per-split kernels, and enough for the
 // balanced kernel's one record per (block, unit) pair of its tile list at up to kMaxBalancedBlocks blocks.
 constexpr int kMaxBalancedBlocks = 1024;
-size_t partial_records_of(const corm_config_t& c) {
-    const size_t U = (size_t)c.batch * c.n_kv_heads;
+// layers whose units one launch may cover: all of a slab cache's layers if their units fit a grid dimension, else one
+size_t fused_layers_of(const corm_config_t& c, int pool_pages) {
+    const long long U = (long long)c.batch * c.n_kv_heads;
+    return (pool_pages == 0 && c.n_layers > 1 && U * c.n_layers <= 65535) ? (size_t)c.n_layers : 1;
+}
+size_t partial_records_of(const corm_config_t& c, int pool_pages) {
+    const size_t U = (size_t)c.batch * c.n_kv_heads * fused_layers_of(c, pool_pages);
     return std::max(U * (size_t)max_splits_of(c), bal_record_count(kMaxBalancedBlocks, (int)U));
 }
 
@@ -101,10 +106,13 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.page_room = take(pool_pages ? Ltot * U * 4 : 0);
     L.bookkeeping_end = off;
     L.q_prev = take(Ltot * (size_t)c.batch * c.n_q_heads * D * e);
-    L.stash = take(U * G * C * 8);
-    L.partials = take(partial_records_of(c) * G * partial_stride((int)D));
-    L.keepmask = take(U * (size_t)keepmask_words((int)C) * 4);
-    L.unit_rec = take(U * 8);
+    // scratch of one launch; a launch covers one layer's units, or all layers' units when corm_decode_step_layers
+    // steps them together (slab caches): 8 G bytes per slot against the 2 D e bytes of its K and V rows
+    const size_t Us = U * fused_layers_of(c, pool_pages);
+    L.stash = take(Us * G * C * 8);
+    L.partials = take(partial_records_of(c, pool_pages) * G * partial_stride((int)D));
+    L.keepmask = take(Us * (size_t)keepmask_words((int)C) * 4);
+    L.unit_rec = take(Us * 8);
     L.stage_q = take((size_t)c.batch * c.n_q_heads * D * e);
     L.stage_k = take(U * D * e);
     L.stage_v = take(U * D * e);
@@ -161,6 +169,11 @@ struct corm_cache {
     long long launches = 0;
     int pool_pages = 0, pt_stride = 0;            // paged cache: pages per layer, page-table entries per unit
     std::vector<CUtensorMap> vmaps;               // per layer: the V storage as a tiled tensor (balanced kernel); empty = unavailable
+    CUtensorMap vmap_all;                         // the V storage of all layers of a slab cache as one tensor (layers stepped together)
+    bool have_vmap_all = false;
+    // per layer: the group of layers (first layer * 65536 + count) it has been stepped with ever since its prompt pass
+    // (-1: not stepped yet, -2: alone or in different groups); only then does the group's length read-back describe it
+    std::vector<int> step_group;
 };
 
 namespace {
@@ -210,7 +223,8 @@ template <typename P> void set_paging(const corm_cache* c, int layer, P& p) {
 }
 
 int32_t* live_buf(const corm_cache* c, int layer, int parity) {
-    return reinterpret_cast<int32_t*>(c->arena + c->lay.live) + ((size_t)layer * 2 + parity) * c->U;
+    // [2][L][U]: the layers' buffers of one parity are contiguous, so that layers stepped together form one array
+    return reinterpret_cast<int32_t*>(c->arena + c->lay.live) + ((size_t)parity * c->cfg.n_layers + layer) * c->U;
 }
 
 bool layer_ok(const corm_cache* c, int layer) { return c && layer >= 0 && layer < c->cfg.n_layers; }
@@ -280,9 +294,25 @@ corm_status_t monitor_similarity(corm_cache* c, int layer, const void* q, cudaSt
     return CORM_OK;
 }
 
+// One decode step of layers [layer, layer + n_fused) as ONE launch (pair): the layers' units are consecutive in every
+// per-unit array of the arena, so n_fused layers of U units are one array of n_fused * U units to the kernels. The
+// caller has checked that the layers are at the same step with the same buffer parity and that q, k_new, v_new and
+// out of consecutive layers are contiguous. Counters of the step go to the first layer's slots (totals are unchanged).
 corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
-                            cudaStream_t st) {
-    poll_live_bound(c, layer);
+                            cudaStream_t st, int n_fused = 1) {
+    for (int i = 0; i < n_fused; ++i) poll_live_bound(c, layer + i);
+    {   // A launch publishes its longest unit in its first layer's word. That bounds every layer of the group, but only
+        // while that word has only ever been written by launches over this same group of layers.
+        const int now = n_fused > 1 ? layer * 65536 + n_fused : -2;           // this launch's group (solo launches: none)
+        bool same_group = n_fused > 1;
+        for (int i = 0; i < n_fused; ++i) {
+            int& g = c->step_group[layer + i];
+            g = (g == -1 || g == now) ? now : -2;
+            same_group &= g == now && now != -2;
+        }
+        if (same_group && c->steps[layer] > 0)
+            for (int i = 1; i < n_fused; ++i) c->live_upper[layer + i] = std::min(c->live_upper[layer + i], c->live_upper[layer]);
+    }
     const corm_config_t& cf = c->cfg;
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
     DecodeParams p{};
@@ -307,10 +337,16 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.keepmask = reinterpret_cast<uint32_t*>(c->arena + c->lay.keepmask);
     p.unit_rec = reinterpret_cast<int2*>(c->arena + c->lay.unit_rec);
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
-    p.U = (int)U; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
+    p.U = (int)U * n_fused; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
     p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
     p.log_alpha = log_alpha_of(c);
-    const int upper = std::min(cf.max_tokens, c->live_upper[layer] + 1);   // no unit can hold more live keys
+    int bound = 0, mean_sum = 0, mean_known = 1;
+    for (int i = 0; i < n_fused; ++i) {
+        bound = std::max(bound, c->live_upper[layer + i]);
+        mean_known &= c->live_mean[layer + i] > 0;
+        mean_sum += c->live_mean[layer + i];
+    }
+    const int upper = std::min(cf.max_tokens, bound + 1);   // no unit can hold more live keys
 
     const bool fast = c->allow_fast && cf.kv_dtype == CORM_BF16 && cf.head_dim == 128 && c->G <= 4;
     corm_status_t rc;
@@ -323,10 +359,10 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     const bool balanced = fast && !c->vmaps.empty() && (c->allow_fast == 4 || c->allow_fast == 5 || (c->allow_fast == 1 && c->G >= 2));
     const bool balanced_verdict = c->allow_fast != 4;
     if (balanced) {
-        rc = launch_decode_balanced(p, c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf), balanced_verdict, st, &n_launched);
+        rc = launch_decode_balanced(p, n_fused > 1 ? c->vmap_all : c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf, c->pool_pages), balanced_verdict, st, &n_launched);
     } else if (fast) {
         // the mean grows by at most one key per step, like the bound
-        const int typical = c->live_mean[layer] ? std::min(upper, c->live_mean[layer] + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
+        const int typical = mean_known ? std::min(upper, mean_sum / n_fused + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
         rc = launch_decode_fast(p, c->G, upper, typical, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
@@ -337,18 +373,21 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
             const size_t smem = generic_decode_smem(DD, GG, cf.max_tokens, c->pool_pages != 0);
             auto kern = decode_generic_kernel<T, DD, GG>;
             CORM_CUDA(ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem));
-            kern<<<dim3(n_splits, (unsigned)U), kGenericThreads, smem, st>>>(p);
+            kern<<<dim3(n_splits, (unsigned)p.U), kGenericThreads, smem, st>>>(p);
             CORM_CUDA(cudaGetLastError());
             return CORM_OK;
         });
     }
     if (rc != CORM_OK) return rc;
     c->launches += n_launched;
-    c->parity[layer] ^= 1;
-    c->steps[layer] += 1;
-    c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
-    if (c->steps[layer] - c->last_readback_step[layer] >= 8) schedule_live_readback(c, layer, st);
-    return monitor_similarity(c, layer, q, st);
+    for (int i = 0; i < n_fused; ++i) {
+        const int l = layer + i;
+        c->parity[l] ^= 1;
+        c->steps[l] += 1;
+        c->live_upper[l] = std::min(cf.max_tokens, c->live_upper[l] + 1);
+        if (c->steps[l] - c->last_readback_step[l] >= 8) schedule_live_readback(c, l, st);
+    }
+    return n_fused == 1 ? monitor_similarity(c, layer, q, st) : CORM_OK;
 }
 
 }  // namespace
@@ -395,6 +434,7 @@ corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pag
     c->live_upper.assign(cfg->n_layers, 0);
     c->live_mean.assign(cfg->n_layers, 0);
     c->have_q_prev.assign(cfg->n_layers, 0);
+    c->step_group.assign(cfg->n_layers, -1);
     c->readback_pending.assign(cfg->n_layers, 0);
     c->last_readback_step.assign(cfg->n_layers, 0);
     c->readback_ev.assign(cfg->n_layers, nullptr);
@@ -425,6 +465,8 @@ corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pag
                 c->vmaps.clear();                 // the block-per-split kernels serve the cache instead
                 break;
             }
+        if (!c->vmaps.empty() && !pool_pages && cfg->n_layers > 1)
+            c->have_vmap_all = make_v_tensor_map(&c->vmap_all, layer_ptr(c, lay.V, kv_layer_bytes(c), 0), rows * cfg->n_layers) == CORM_OK;
     }
     cudaError_t e = cudaMemset(c->arena + lay.bookkeeping_begin, 0, lay.bookkeeping_end - lay.bookkeeping_begin);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -458,7 +500,7 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
                               static_cast<cudaStream_t>(stream)));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; c->live_mean[l] = 0; c->have_q_prev[l] = 0;
-        c->readback_pending[l] = 0; c->last_readback_step[l] = 0;
+        c->readback_pending[l] = 0; c->last_readback_step[l] = 0; c->step_group[l] = -1;
     }
     return CORM_OK;
 }
@@ -524,7 +566,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
         fp.p = p;
         fp.partials = c->arena + c->lay.partials;
         fp.ticket = reinterpret_cast<uint32_t*>(layer_ptr(c, c->lay.ticket, U * 4, layer));
-        const size_t cap = U * (size_t)max_splits_of(cf) * c->G * partial_stride((int)D);
+        const size_t cap = U * (size_t)max_splits_of(cf) * c->G * partial_stride((int)D);   // one layer's share is enough here
         rc = launch_prompt_fast(fp, c->G, max_p, c->sm_count, cap, st);
         n_launched = prompt_fast_launches(c->G, cf.window_w);
     }
@@ -545,6 +587,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     c->launches += n_launched;
     c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p; c->live_mean[layer] = 0;
     c->have_q_prev[layer] = 0;                    // the previous decode query belonged to the old text
+    c->step_group[layer] = -1;
     c->last_readback_step[layer] = 0;
     schedule_live_readback(c, layer, st);
     return CORM_OK;
@@ -576,6 +619,22 @@ corm_status_t corm_decode_step_layers(corm_cache_t* c, int32_t first_layer, int3
     }
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return CORM_ERR_CUDA;
+    // One launch for all the layers when the kernels can see them as one array of units: a slab cache on the
+    // bf16 / head_dim-128 kernels, every layer at the same step with the same buffer parity, and the layers' q,
+    // k_new, v_new and out contiguous in layer order. (Grouped heads also need the tensor map over all layers, which
+    // starts at layer 0.)
+    const corm_config_t& cf = c->cfg;
+    const size_t qb = (size_t)cf.batch * cf.n_q_heads * cf.head_dim * c->e, kb = (size_t)c->U * cf.head_dim * c->e;
+    bool fuse = n_layers > 1 && fused_layers_of(cf, c->pool_pages) > 1 && c->allow_fast && cf.kv_dtype == CORM_BF16 &&
+                cf.head_dim == 128 && c->G <= 4 && !c->monitor_similarity &&
+                (c->G == 1 || c->allow_fast == 2 || c->allow_fast == 3 || (c->have_vmap_all && first_layer == 0));
+    for (int i = 1; fuse && i < n_layers; ++i) {
+        const auto at = [](const void* ptr, size_t off) { return static_cast<const unsigned char*>(ptr) + off; };
+        fuse = c->steps[first_layer + i] == c->steps[first_layer] && c->parity[first_layer + i] == c->parity[first_layer] &&
+               q[i] == at(q[0], i * qb) && out[i] == at(out[0], i * qb) && k_new[i] == at(k_new[0], i * kb) &&
+               v_new[i] == at(v_new[0], i * kb);
+    }
+    if (fuse) return launch_decode(c, first_layer, q[0], k_new[0], v_new[0], out[0], static_cast<cudaStream_t>(stream), n_layers);
     for (int i = 0; i < n_layers; ++i) {
         const corm_status_t rc = launch_decode(c, first_layer + i, q[i], k_new[i], v_new[i], out[i], static_cast<cudaStream_t>(stream));
         if (rc != CORM_OK) return rc;
@@ -740,7 +799,7 @@ corm_status_t corm_cache_stats(corm_cache_t* c, corm_stats_t* out_host, void* st
     CORM_CUDA(cudaStreamSynchronize(st));
     corm_stats_t s{};
     for (int l = 0; l < L; ++l) {
-        const int32_t* lv = live.data() + ((size_t)l * 2 + c->parity[l]) * c->U;
+        const int32_t* lv = live.data() + ((size_t)c->parity[l] * L + l) * c->U;
         for (int u = 0; u < c->U; ++u) s.live_keys += lv[u];
         s.appended_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_APPENDED];
         s.evicted_keys += (int64_t)cnt[(size_t)l * CNT_COUNT + CNT_EVICTED];
@@ -863,6 +922,7 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     c->readback_pending[layer] = 0;   // a read-back enqueued before this import knows nothing of it
     c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
     c->live_mean[layer] = 0;                      // unknown until the next read-back
+    c->step_group[layer] = -2;                    // lengths changed behind the kernels' backs: the layer keeps its own bound
     return CORM_OK;
 }
 
