@@ -172,7 +172,7 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
     dev = lambda a: torch.from_numpy(a).cuda().to(tdt).contiguous()
     cache = CormCache(L, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg_r.max_tokens, cfg.window_w,
                       cfg.recent_r, cfg.alpha, cfg.dtype, local, pool_pages=args.pool_pages)
-    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4, "balanced-verdict": 5}[args.finish])
+    cache.corm_cache_set_tuning(args.split_len, 0 if args.no_fast else {"auto": 1, "inline": 2, "verdict": 3, "balanced": 4, "balanced-verdict": 5, "units": 6}[args.finish])
     ev = lambda: torch.cuda.Event(enable_timing=True)
     a, b = ev(), ev()
     prompts = [(dev(d.k_prompt), dev(d.v_prompt), dev(d.q_last), d.prompt_lens) for d in data]
@@ -213,13 +213,26 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
             qv, kv, vv = views[s][0]
             cache.corm_decode_step(0, qv, kv, vv, out)
 
+    out_steps = torch.empty_like(q_all) if args.api == "steps" else None
+
+    def run(s0, s1, api):
+        """Enqueue decode steps [s0, s1): one corm_decode_steps call, or one call per step."""
+        if s1 <= s0:
+            return
+        if api == "steps":
+            cache.corm_decode_steps(0, L, q_all[s0:s1], k_all[s0:s1], v_all[s0:s1], out_steps[s0:s1])
+        else:
+            for s in range(s0, s1):
+                step(s)
+
     restore()                                            # untimed: the first launches load the kernels
     passes, prompt_ms, sampler = [], 0.0, None
-    for rep in range(args.repeats):
+    # with --api steps one more pass times the same steps through one call per step, reported as `per_step_calls`
+    plan = [args.api] * args.repeats + (["step"] if args.api == "steps" else [])
+    for rep, api in enumerate(plan):
         prompt_ms = restore()
         st0 = cache.corm_cache_stats()
-        for s in range(args.warmup):
-            step(s)
+        run(0, args.warmup, api)
         torch.cuda.synchronize()
         st1 = cache.corm_cache_stats()
         launches0 = cache.corm_cache_kernel_launches()
@@ -231,8 +244,8 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
         torch.cuda.synchronize()
         a.record()
         t_issue = time.perf_counter()
-        for s in range(args.warmup, n_steps):
-            step(s)
+        chained0 = cache.corm_cache_chained_launches()
+        run(args.warmup, n_steps, api)
         b.record()
         issue_ms = 1e3 * (time.perf_counter() - t_issue)  # host time to enqueue the timed steps
         torch.cuda.synchronize()
@@ -240,7 +253,9 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
             dist.barrier()
         st2 = cache.corm_cache_stats()
         passes.append(dict(ms=a.elapsed_time(b), issue_ms=issue_ms, st0=st0, st1=st1, st2=st2,
-                           launches=cache.corm_cache_kernel_launches() - launches0))
+                           launches=cache.corm_cache_kernel_launches() - launches0,
+                           chained=cache.corm_cache_chained_launches() - chained0))
+    per_step_pass = passes.pop() if args.api == "steps" else None
     passes_sorted = sorted(passes, key=lambda x: x["ms"])
     med = passes_sorted[len(passes_sorted) // 2]
 
@@ -301,6 +316,9 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": "the same decode steps as `value`, from the same restored state"},
         "gpu_launches": med["launches"], "host_issue_us_per_step": 1e3 * med["issue_ms"] / args.steps,
+        "api": ("corm_decode_steps: the timed steps enqueued by one call" if args.api == "steps" else
+                "one corm_decode_step" + ("_layers" if L > 1 else "") + " call per step"),
+        "chained_launches": med["chained"],
         "retention": med["st2"]["retention"],
         "live_keys_per_unit": med["st2"]["live_keys"] / (L * cfg.batch * cfg.n_kv_heads),
         "evicted_keys_timed": med["st2"]["evicted_keys"] - med["st1"]["evicted_keys"], "moved_rows_timed": moved,
@@ -309,6 +327,11 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
         "near_threshold_prompt_pass": med["st0"]["near_threshold"],
         "arena_bytes": int(cache.arena.numel()),
     }
+    if per_step_pass is not None:       # the same steps, one host call per step (no launch is chained to the one before)
+        res["per_step_calls"] = {
+            "value": aggregate_throughput(per_step_pass["ms"], cfg.batch * args.steps, "cuda")[0], "unit": UNIT,
+            "ms_per_step": per_step_pass["ms"] / args.steps,
+            "host_issue_us_per_step": 1e3 * per_step_pass["issue_ms"] / args.steps}
     if sampler is not None:
         res["clocks"] = sampler.result()
     if args.pool_pages:
@@ -329,6 +352,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=16)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--api", default="steps", choices=["steps", "step"],
+                    help="steps: the timed steps are enqueued by one corm_decode_steps call (consecutive launches chained "
+                         "where the kernels allow it); step: one corm_decode_step / corm_decode_step_layers call per step")
     ap.add_argument("--repeats", type=int, default=3, help="timed passes over the same steps; the median is reported")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end pass through the host-buffer entry point")
     ap.add_argument("--e2e-steps", type=int, default=None, help="0 skips the end-to-end pass (same as --no-e2e)")
@@ -338,7 +364,7 @@ def main():
     ap.add_argument("--ref-steps", type=int, default=512)
     ap.add_argument("--split-len", type=int, default=0)
     ap.add_argument("--no-fast", action="store_true")
-    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced", "balanced-verdict"],
+    ap.add_argument("--finish", default="auto", choices=["auto", "inline", "verdict", "balanced", "balanced-verdict", "units"],
                     help="which decode kernels: automatic, the block-per-split kernels finishing long units inside the "
                          "decode launch / by the verdict launch, or the balanced single-launch kernel")
     ap.add_argument("--alpha", type=float, default=None, help="override the threshold scale (0 keeps every key)")
@@ -383,7 +409,7 @@ def main():
         args.steps = min(args.steps, cfg_w.steps - args.warmup) if cfg_w.steps > args.warmup else args.steps
         r = measure_workload(cfg_w, args, local, world, rank, False, False)
         keep = ("value", "ms_per_step", "repeats", "roofline", "gpu_launches", "host_issue_us_per_step", "retention",
-                "live_keys_per_unit", "prompt_pass_ms")
+                "live_keys_per_unit", "prompt_pass_ms", "api", "chained_launches", "per_step_calls")
         also.append(dict({"config": workload_config(cfg_w, args, w), "steps": args.steps, "unit": UNIT},
                          **{k: r[k] for k in keep}))
         args.steps = saved

@@ -166,6 +166,25 @@ corm_status_t corm_decode_step_layers(corm_cache_t* cache, int32_t first_layer, 
                                       const void* const* q, const void* const* k_new, const void* const* v_new,
                                       void* const* out, void* stream);
 
+/* n_steps consecutive decode steps of n_layers consecutive layers from one host call, for callers that hold the
+ * inputs of all those steps before the first one runs: scoring a given text (the paper's language-modelling
+ * experiments feed known tokens; a layer's queries, keys and values for all positions can be formed before its cache
+ * is stepped through them), replay, benchmarking. Buffers are device arrays laid out [n_steps][n_layers] of the
+ * per-layer tensors of corm_decode_step:
+ *   q, out        [n_steps][n_layers][batch, n_q_heads, head_dim]
+ *   k_new, v_new  [n_steps][n_layers][batch, n_kv_heads, head_dim]
+ * Every input must be complete in stream order before the call; the result is that of calling corm_decode_step_layers
+ * once per step (registers, live lists and positions identical, outputs within rounding).
+ * What the call adds: the units of a cache are independent (Algorithm 1 runs "on each head at every layer"), so
+ * step s + 1 of a unit needs step s of that unit only. When a step's launch finishes every unit inside the streaming
+ * kernel (one query head per KV head, or tuning value 2), the next step's launch is chained to it: its blocks start
+ * as soon as a multiprocessor has room and each waits (bounded, like every wait here) for its own unit's previous
+ * step instead of the whole previous launch, so consecutive steps fill one another's last waves. Steps that need the
+ * verdict launch, and caches with the similarity monitor on, run as with the per-step calls.
+ * Errors: as corm_decode_step_layers; n_steps == 0 is a no-op. A failing step leaves the steps before it enqueued. */
+corm_status_t corm_decode_steps(corm_cache_t* cache, int32_t first_layer, int32_t n_layers, int32_t n_steps,
+                                const void* q, const void* k_new, const void* v_new, void* out, void* stream);
+
 /* Same step with HOST buffers, asynchronous on `stream` (out_host is valid once the stream has been synchronised).
  * Pinned buffers the device can address (cudaHostAlloc / cudaHostRegister, 16-byte aligned) are read and written by
  * the kernels directly across the bus, with no copies; any other host memory is copied to staging space inside the
@@ -242,6 +261,9 @@ corm_status_t corm_cache_set_bound_scale(corm_cache_t* cache, double scale);
 
 /* Number of kernels this library has launched on behalf of `cache` since create. */
 int64_t corm_cache_kernel_launches(const corm_cache_t* cache);
+
+/* How many of them were chained to the previous step's launch (corm_decode_steps). */
+int64_t corm_cache_chained_launches(const corm_cache_t* cache);
 
 const char* corm_status_string(corm_status_t status);
 

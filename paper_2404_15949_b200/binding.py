@@ -77,6 +77,10 @@ def load_library():
     lib.corm_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.corm_decode_step_layers.restype = i32
     lib.corm_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.corm_decode_steps.restype = i32
+    lib.corm_decode_steps.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.corm_cache_chained_launches.restype = i64
+    lib.corm_cache_chained_launches.argtypes = [vp]
     lib.corm_cache_stats.restype = i32
     lib.corm_cache_stats.argtypes = [vp, ctypes.POINTER(CormStats), vp]
     lib.corm_cache_live_lens.restype = i32
@@ -209,6 +213,31 @@ class CormCache:
             self.handle, first_layer, n, tables[0].ctypes.data, tables[1].ctypes.data, tables[2].ctypes.data,
             tables[3].ctypes.data, _stream_ptr(stream)))
         return out
+
+    def corm_decode_steps(self, first_layer, n_layers, q, k_new, v_new, out=None, stream=None):
+        """``q.shape[0]`` consecutive decode steps of ``n_layers`` consecutive layers from one host call. ``q`` and
+        ``out``: device tensors ``[n_steps, n_layers, batch, n_q_heads, head_dim]``; ``k_new``, ``v_new``:
+        ``[n_steps, n_layers, batch, n_kv_heads, head_dim]`` (the layer axis may be left out for one layer)."""
+        if n_layers == 1 and q.dim() == 1 + len(self._q_shape):
+            q, k_new, v_new = q.unsqueeze(1), k_new.unsqueeze(1), v_new.unsqueeze(1)
+            out = out.unsqueeze(1) if out is not None else None
+            squeeze = True
+        else:
+            squeeze = False
+        n_steps = q.shape[0]
+        if out is None:
+            out = torch.empty_like(q)
+        for t, shape in ((q, self._q_shape), (out, self._q_shape), (k_new, self._kv_shape), (v_new, self._kv_shape)):
+            if not (tuple(t.shape) == (n_steps, n_layers) + tuple(shape) and t.dtype == self.dtype and t.is_cuda and
+                    t.is_contiguous()):
+                raise ValueError("corm_decode_steps: contiguous device tensors [n_steps, n_layers, ...] of the cache dtype")
+        _check("corm_decode_steps", self.lib.corm_decode_steps(
+            self.handle, first_layer, n_layers, n_steps, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+            _stream_ptr(stream)))
+        return out.squeeze(1) if squeeze else out
+
+    def corm_cache_chained_launches(self):
+        return int(self.lib.corm_cache_chained_launches(self.handle))
 
     def pointer_table(self, tensors, kind):
         """Device addresses of per-layer tensors as a uint64 array (kind "q": shaped like q / out, "kv": like k_new)."""

@@ -6,6 +6,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <climits>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -30,7 +31,7 @@ constexpr int kMinSplit = 64;
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Layout {
-    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, ticket3, move_info, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask, unit_rec;
+    size_t K, V, word, pos, live, base_tokens, base_obs, ticket, ticket2, ticket3, move_info, unit_stamp, counters, status, maxlive, sim_acc, page_table, page_bits, page_room, q_prev, stash, partials, keepmask, unit_rec;
     size_t stage_q, stage_k, stage_v, stage_out, total, bookkeeping_begin, bookkeeping_end;
 };
 
@@ -97,6 +98,7 @@ Layout make_layout(const corm_config_t& c, int pool_pages) {
     L.ticket2 = take(Ltot * U * 4);
     L.ticket3 = take(Ltot * U * 4);
     L.move_info = take(Ltot * U * 8);
+    L.unit_stamp = take(Ltot * U * 8);
     L.counters = take(Ltot * CNT_COUNT * 8);
     L.status = take(4);
     L.maxlive = take(Ltot * 8);
@@ -174,6 +176,14 @@ struct corm_cache {
     // per layer: the group of layers (first layer * 65536 + count) it has been stepped with ever since its prompt pass
     // (-1: not stepped yet, -2: alone or in different groups); only then does the group's length read-back describe it
     std::vector<int> step_group;
+    // per layer, meaningful for the first layer of a group: bound on the longest unit of ALL the group's layers, taken
+    // from a length word that a launch over the whole group wrote (INT_MAX = none yet). The first layer's own
+    // live_upper may be smaller: right after the prompt pass it describes that layer alone.
+    std::vector<int> group_upper;
+    // per layer: its latest decode launch finished every unit inside the streaming kernel and left the units' stamps,
+    // so the next step's launch may be chained to it (corm_decode_steps)
+    std::vector<int> chain_ok;
+    long long chained_launches = 0;
 };
 
 namespace {
@@ -255,6 +265,8 @@ void poll_live_bound(corm_cache* c, int layer) {
     if (steps_done > c->steps[layer]) return;   // stale word from before a reset / new prompt
     const int bound = len + (c->steps[layer] - steps_done);
     if (bound < c->live_upper[layer]) c->live_upper[layer] = bound;
+    // a word written by a decode launch over the layer's group covers every layer of the group
+    if (steps_done >= 1 && c->step_group[layer] >= 0 && bound < c->group_upper[layer]) c->group_upper[layer] = bound;
     long long sum = 0;                            // the lengths themselves came with the same read-back
     for (int u = 0; u < c->U; ++u) sum += c->live_host[(size_t)layer * c->U + u];
     c->live_mean[layer] = (int)(sum / c->U);
@@ -298,8 +310,10 @@ corm_status_t monitor_similarity(corm_cache* c, int layer, const void* q, cudaSt
 // per-unit array of the arena, so n_fused layers of U units are one array of n_fused * U units to the kernels. The
 // caller has checked that the layers are at the same step with the same buffer parity and that q, k_new, v_new and
 // out of consecutive layers are contiguous. Counters of the step go to the first layer's slots (totals are unchanged).
+// chain: the caller enqueued this layer's (these layers') previous step immediately before and nothing since, and
+// this step's inputs were complete before that; more: the next step follows in the same way.
 corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void* k_new, const void* v_new, void* out,
-                            cudaStream_t st, int n_fused = 1) {
+                            cudaStream_t st, int n_fused = 1, bool chain = false, bool more = false) {
     for (int i = 0; i < n_fused; ++i) poll_live_bound(c, layer + i);
     {   // A launch publishes its longest unit in its first layer's word. That bounds every layer of the group, but only
         // while that word has only ever been written by launches over this same group of layers.
@@ -310,8 +324,8 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
             g = (g == -1 || g == now) ? now : -2;
             same_group &= g == now && now != -2;
         }
-        if (same_group && c->steps[layer] > 0)
-            for (int i = 1; i < n_fused; ++i) c->live_upper[layer + i] = std::min(c->live_upper[layer + i], c->live_upper[layer]);
+        if (same_group && c->group_upper[layer] != INT_MAX)
+            for (int i = 0; i < n_fused; ++i) c->live_upper[layer + i] = std::min(c->live_upper[layer + i], c->group_upper[layer]);
     }
     const corm_config_t& cf = c->cfg;
     const size_t C = cf.max_tokens, D = cf.head_dim, U = c->U;
@@ -336,6 +350,7 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     p.partials = c->arena + c->lay.partials;
     p.keepmask = reinterpret_cast<uint32_t*>(c->arena + c->lay.keepmask);
     p.unit_rec = reinterpret_cast<int2*>(c->arena + c->lay.unit_rec);
+    p.unit_stamp = reinterpret_cast<unsigned long long*>(layer_ptr(c, c->lay.unit_stamp, U * 8, layer));
     p.q = q; p.k_new = k_new; p.v_new = v_new; p.out = out;
     p.U = (int)U * n_fused; p.Hkv = cf.n_kv_heads; p.C = cf.max_tokens; p.max_splits = max_splits_of(cf);
     p.step = c->steps[layer]; p.w = cf.window_w; p.r = cf.recent_r;
@@ -356,14 +371,35 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     // against 136 in its first steps, 174 against 190 on 24k-key units, 157 against 177 on 8k-key units without
     // evictions); one query head per KV head stays on the block-per-split kernel, whose loop is lighter (three
     // blocks per SM). Tuning values 4 / 5 force the balanced kernel finishing in the launch / with the verdict launch.
-    const bool balanced = fast && !c->vmaps.empty() && (c->allow_fast == 4 || c->allow_fast == 5 || (c->allow_fast == 1 && c->G >= 2));
+    // Inside a call of several steps (corm_decode_steps) grouped heads take that kernel's loop with a block per split
+    // and the unit finished by its last split instead, because such launches can be chained: 43 against 51 us per step
+    // on 128 units of 1660 keys, 132 against 142 on 8200-key units. Not with few long units, whose finishing block
+    // walks the whole unit alone (32 units of 12-24k keys: 133 against 103 us). Tuning value 6 forces it.
+    const bool units = fast && !c->vmaps.empty() &&
+                       (c->allow_fast == 6 || (c->allow_fast == 1 && c->G >= 2 && (chain || more) && !c->monitor_similarity &&
+                                               (long long)upper <= 96ll * (long long)p.U));
+    const bool balanced = !units && fast && !c->vmaps.empty() &&
+                          (c->allow_fast == 4 || c->allow_fast == 5 || (c->allow_fast == 1 && c->G >= 2));
     const bool balanced_verdict = c->allow_fast != 4;
-    if (balanced) {
+    bool chain_ok_before = chain && !c->monitor_similarity;
+    for (int i = 0; i < n_fused; ++i) chain_ok_before &= c->chain_ok[layer + i] != 0;
+    bool self_finishing = false;
+    if (!(fast && !balanced) && !units) p.unit_stamp = nullptr;    // only the block-per-split kernels keep stamps
+    if (units) {
+        const int typical = mean_known ? std::min(upper, mean_sum / n_fused + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
+        rc = launch_decode_balanced_units(p, n_fused > 1 ? c->vmap_all : c->vmaps[layer], c->G, upper, typical, c->tune_split_len,
+                                          c->sm_count, partial_records_of(cf, c->pool_pages), st, &n_launched,
+                                          chain_ok_before, more && !c->monitor_similarity);
+        self_finishing = rc == CORM_OK;
+        if (rc == CORM_OK && p.chain_wait) c->chained_launches += 1;
+    } else if (balanced) {
         rc = launch_decode_balanced(p, n_fused > 1 ? c->vmap_all : c->vmaps[layer], c->G, upper, c->sm_count, partial_records_of(cf, c->pool_pages), balanced_verdict, st, &n_launched);
     } else if (fast) {
         // the mean grows by at most one key per step, like the bound
         const int typical = mean_known ? std::min(upper, mean_sum / n_fused + c->steps[layer] - c->last_readback_step[layer] + 1) : 0;
-        rc = launch_decode_fast(p, c->G, upper, typical, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast);
+        rc = launch_decode_fast(p, c->G, upper, typical, c->tune_split_len, c->sm_count, st, &n_launched, c->allow_fast,
+                                chain_ok_before, more && !c->monitor_similarity, &self_finishing);
+        if (rc == CORM_OK && p.chain_wait) c->chained_launches += 1;
     } else {
         p.split_len = c->tune_split_len ? c->tune_split_len : 256;
         const int n_splits = (upper + p.split_len - 1) / p.split_len;
@@ -382,9 +418,11 @@ corm_status_t launch_decode(corm_cache* c, int layer, const void* q, const void*
     c->launches += n_launched;
     for (int i = 0; i < n_fused; ++i) {
         const int l = layer + i;
+        c->chain_ok[l] = self_finishing ? 1 : 0;
         c->parity[l] ^= 1;
         c->steps[l] += 1;
         c->live_upper[l] = std::min(cf.max_tokens, c->live_upper[l] + 1);
+        if (c->group_upper[l] != INT_MAX) c->group_upper[l] += 1;
         if (c->steps[l] - c->last_readback_step[l] >= 8) schedule_live_readback(c, l, st);
     }
     return n_fused == 1 ? monitor_similarity(c, layer, q, st) : CORM_OK;
@@ -435,6 +473,8 @@ corm_status_t corm_cache_create_paged(const corm_config_t* cfg, int32_t pool_pag
     c->live_mean.assign(cfg->n_layers, 0);
     c->have_q_prev.assign(cfg->n_layers, 0);
     c->step_group.assign(cfg->n_layers, -1);
+    c->group_upper.assign(cfg->n_layers, INT_MAX);
+    c->chain_ok.assign(cfg->n_layers, 0);
     c->readback_pending.assign(cfg->n_layers, 0);
     c->last_readback_step.assign(cfg->n_layers, 0);
     c->readback_ev.assign(cfg->n_layers, nullptr);
@@ -500,7 +540,7 @@ corm_status_t corm_cache_reset(corm_cache_t* c, void* stream) {
                               static_cast<cudaStream_t>(stream)));
     for (int l = 0; l < c->cfg.n_layers; ++l) {
         c->parity[l] = 0; c->steps[l] = 0; c->ready[l] = 0; c->live_upper[l] = 0; c->live_mean[l] = 0; c->have_q_prev[l] = 0;
-        c->readback_pending[l] = 0; c->last_readback_step[l] = 0; c->step_group[l] = -1;
+        c->readback_pending[l] = 0; c->last_readback_step[l] = 0; c->step_group[l] = -1; c->chain_ok[l] = 0; c->group_upper[l] = INT_MAX;
     }
     return CORM_OK;
 }
@@ -535,6 +575,8 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket2, U * 4, layer), 0, U * 4, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.ticket3, U * 4, layer), 0, U * 4, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.move_info, U * 8, layer), 0, U * 8, st));
+    CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.unit_stamp, U * 8, layer), 0, U * 8, st));   // step counts restart
+    c->chain_ok[layer] = 0;
     CORM_CUDA(cudaMemsetAsync(maxlive_ptr(c, layer), 0, 8, st));
     CORM_CUDA(cudaMemsetAsync(layer_ptr(c, c->lay.counters, CNT_COUNT * 8, layer), 0, CNT_COUNT * 8, st));   // a new prompt restarts the layer's statistics
     c->readback_pending[layer] = 0;   // an older read-back no longer describes this layer
@@ -588,6 +630,7 @@ corm_status_t corm_compress_prompt(corm_cache_t* c, int32_t layer, const void* k
     c->parity[layer] = 0; c->steps[layer] = 0; c->ready[layer] = 1; c->live_upper[layer] = max_p; c->live_mean[layer] = 0;
     c->have_q_prev[layer] = 0;                    // the previous decode query belonged to the old text
     c->step_group[layer] = -1;
+    c->group_upper[layer] = INT_MAX;
     c->last_readback_step[layer] = 0;
     schedule_live_readback(c, layer, st);
     return CORM_OK;
@@ -627,7 +670,7 @@ corm_status_t corm_decode_step_layers(corm_cache_t* c, int32_t first_layer, int3
     const size_t qb = (size_t)cf.batch * cf.n_q_heads * cf.head_dim * c->e, kb = (size_t)c->U * cf.head_dim * c->e;
     bool fuse = n_layers > 1 && fused_layers_of(cf, c->pool_pages) > 1 && c->allow_fast && cf.kv_dtype == CORM_BF16 &&
                 cf.head_dim == 128 && c->G <= 4 && !c->monitor_similarity &&
-                (c->G == 1 || c->allow_fast == 2 || c->allow_fast == 3 || (c->have_vmap_all && first_layer == 0));
+                ((c->allow_fast != 6 && (c->G == 1 || c->allow_fast == 2 || c->allow_fast == 3)) || (c->have_vmap_all && first_layer == 0));
     for (int i = 1; fuse && i < n_layers; ++i) {
         const auto at = [](const void* ptr, size_t off) { return static_cast<const unsigned char*>(ptr) + off; };
         fuse = c->steps[first_layer + i] == c->steps[first_layer] && c->parity[first_layer + i] == c->parity[first_layer] &&
@@ -641,6 +684,55 @@ corm_status_t corm_decode_step_layers(corm_cache_t* c, int32_t first_layer, int3
     }
     return CORM_OK;
 }
+
+corm_status_t corm_decode_steps(corm_cache_t* c, int32_t first_layer, int32_t n_layers, int32_t n_steps, const void* q,
+                                const void* k_new, const void* v_new, void* out, void* stream) {
+    NvtxRange nvtx_range("corm_decode_steps");
+    if (!c || n_layers < 1 || n_steps < 0 || !layer_ok(c, first_layer) || !layer_ok(c, first_layer + n_layers - 1))
+        return CORM_ERR_INVALID_ARG;
+    if (n_steps == 0) return CORM_OK;
+    if (!q || !k_new || !v_new || !out) return CORM_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) |
+         reinterpret_cast<uintptr_t>(out)) % 16) return CORM_ERR_INVALID_ARG;
+    for (int i = 0; i < n_layers; ++i)
+        if (!c->ready[first_layer + i]) return CORM_ERR_STATE;
+    const corm_config_t& cf = c->cfg;
+    DeviceGuard guard(cf.device);
+    if (!guard.ok) return CORM_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t qb = (size_t)cf.batch * cf.n_q_heads * cf.head_dim * c->e, kb = (size_t)c->U * cf.head_dim * c->e;
+    // all layers of a step as one launch under the same conditions as corm_decode_step_layers (the buffers are
+    // contiguous by this call's layout)
+    bool fuse = n_layers > 1 && fused_layers_of(cf, c->pool_pages) > 1 && c->allow_fast && cf.kv_dtype == CORM_BF16 &&
+                cf.head_dim == 128 && c->G <= 4 && !c->monitor_similarity &&
+                ((c->allow_fast != 6 && (c->G == 1 || c->allow_fast == 2 || c->allow_fast == 3)) || (c->have_vmap_all && first_layer == 0));
+    for (int i = 1; fuse && i < n_layers; ++i)
+        fuse = c->steps[first_layer + i] == c->steps[first_layer] && c->parity[first_layer + i] == c->parity[first_layer];
+    const auto at = [](const void* ptr, size_t off) { return static_cast<const unsigned char*>(ptr) + off; };
+    const auto at_out = [](void* ptr, size_t off) { return static_cast<unsigned char*>(ptr) + off; };
+    for (int s = 0; s < n_steps; ++s) {
+        // A step is chained to the one before it when that one was enqueued by this call (nothing of the caller's can
+        // sit between them on the stream, and every step's inputs precede the call) and neither is the last word on
+        // its units' lengths for the host: a length read-back between two launches separates them anyway.
+        const bool chain = s > 0, more = s + 1 < n_steps;
+        if (fuse || n_layers == 1) {
+            const size_t i0 = (size_t)s * n_layers;
+            const corm_status_t rc = launch_decode(c, first_layer, at(q, i0 * qb), at(k_new, i0 * kb), at(v_new, i0 * kb),
+                                                   at_out(out, i0 * qb), st, n_layers, chain, more);
+            if (rc != CORM_OK) return rc;
+            continue;
+        }
+        for (int i = 0; i < n_layers; ++i) {   // separate launches per layer: another layer's launch sits between two steps of one
+            const size_t ix = (size_t)s * n_layers + i;
+            const corm_status_t rc = launch_decode(c, first_layer + i, at(q, ix * qb), at(k_new, ix * kb), at(v_new, ix * kb),
+                                                   at_out(out, ix * qb), st);
+            if (rc != CORM_OK) return rc;
+        }
+    }
+    return CORM_OK;
+}
+
+int64_t corm_cache_chained_launches(const corm_cache_t* c) { return c ? c->chained_launches : 0; }
 
 corm_status_t corm_decode_step_host(corm_cache_t* c, int32_t layer, const void* q_host, const void* k_new_host,
                                     const void* v_new_host, void* out_host, void* stream) {
@@ -767,6 +859,7 @@ corm_status_t corm_decode_step_static(corm_cache_t* c, int32_t layer, const void
     });
     if (rc != CORM_OK) return rc;
     c->launches += 1;
+    c->chain_ok[layer] = 0;
     c->parity[layer] ^= 1;
     c->steps[layer] += 1;
     c->live_upper[layer] = std::min(cf.max_tokens, c->live_upper[layer] + 1);
@@ -923,6 +1016,8 @@ corm_status_t corm_cache_import_state(corm_cache_t* c, int32_t layer, int32_t se
     c->live_upper[layer] = std::max(c->live_upper[layer], live_len);
     c->live_mean[layer] = 0;                      // unknown until the next read-back
     c->step_group[layer] = -2;                    // lengths changed behind the kernels' backs: the layer keeps its own bound
+    c->group_upper[layer] = INT_MAX;
+    c->chain_ok[layer] = 0;                       // ... and its units' stamps no longer describe them
     return CORM_OK;
 }
 
@@ -944,7 +1039,7 @@ corm_status_t corm_cache_pool_usage(corm_cache_t* c, int32_t layer, int64_t* pag
 corm_status_t corm_cache_set_tuning(corm_cache_t* c, int32_t split_len, int32_t allow_fast_path) {
     if (!c || split_len < 0 || (split_len % 32) || (split_len && split_len < kMinSplit)) return CORM_ERR_INVALID_ARG;
     c->tune_split_len = split_len;
-    if (allow_fast_path < 0 || allow_fast_path > 5) return CORM_ERR_INVALID_ARG;
+    if (allow_fast_path < 0 || allow_fast_path > 6) return CORM_ERR_INVALID_ARG;
     c->allow_fast = allow_fast_path;
     return CORM_OK;
 }

@@ -54,6 +54,7 @@ struct BalSeg {
 // Small block-wide variables. The kernel declares no static shared memory at all: its dynamic shared memory then
 // starts at the block's first usable byte, which is 1024-byte aligned, as the swizzled V tiles need (checked at entry).
 struct BalMisc {
+    unsigned long long stamp;     // kBalUnits, chained launch: the unit's stamp as tid 0 read it
     double thr[4], Zg[4];            // finish phase: thresholds and normalisers per head
     int scan[kBalThreads];           // finish phase: scratch of the block-wide prefix sums
     int wsum[kBalWarps];
@@ -160,6 +161,11 @@ __device__ __forceinline__ int vtile_offset(int r, int c) {
 // records the balanced kernel may write in one step: one per warp of every (block, unit) pair on the tile list
 __host__ __device__ inline size_t bal_record_count(int n_blocks, int U) { return ((size_t)n_blocks + (size_t)U) * kBalWarps; }
 
+// A block per split (kBalUnits): unit u keeps its records (one per warp and split) at a place that does not depend on
+// the launch, because chained launches overlap: another unit's previous step may still be reading its own. A quarter
+// of the splits the arena provides records for, times four warps.
+__host__ __device__ inline int bal_unit_splits(int max_splits) { return max_splits >= 4 ? max_splits / 4 : 1; }
+
 // block of the balanced partition that owns tile x of the step's list (T tiles, n blocks)
 __device__ __forceinline__ int bal_block_of(long long x, long long T, int n) { return (int)(((x + 1) * n - 1) / T); }
 
@@ -194,7 +200,9 @@ struct BalFin {
 //   D. the unit's first block reduces the accumulators to the output of Eq. 1; after a second arrival counter the
 //      unit's last block scans the mask, fills the holes and publishes the new length.
 // scratch: the block's ring area, free by now.
-template <int G, bool PAGED, int NT>
+// UNIT: the block is the last-arriving split of the one unit in segs[0] (a block per split, kBalUnits) and finishes
+// the whole unit alone: all the unit's records are stored, nothing is waited for, and the unit's stamp is left.
+template <int G, bool PAGED, int NT, bool UNIT>
 __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int nseg, int blk, long long T, int nblk,
                                  unsigned char* scratch, BalMisc* misc) {
     constexpr int NW = kBalWarps;
@@ -210,14 +218,14 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
         for (int si = 0; si < nseg; ++si) {
             const BalSeg& sg = segs[si];
             const long long P0 = sg.gtile0;
-            const int fb = bal_block_of(P0, T, nblk);
+            const int fb = UNIT ? 0 : bal_block_of(P0, T, nblk);
             BalFin f;
-            f.n_blocks = bal_block_of(P0 + sg.n_unit - 1, T, nblk) - fb + 1;
-            f.rec0 = (fb + sg.u) * NW;
+            f.n_blocks = UNIT ? sg.pad : bal_block_of(P0 + sg.n_unit - 1, T, nblk) - fb + 1;
+            f.rec0 = UNIT ? sg.u * bal_unit_splits(p.max_splits) * NW : (fb + sg.u) * NW;
             f.tile_prefix = tp;
             f.evict_on = min(p.w, __ldcg(p.base_obs + sg.u / p.Hkv) + p.step + 1) >= p.w;
-            f.last = 0;
-            f.first = fb == blk;
+            f.last = UNIT ? 1 : 0;
+            f.first = UNIT || fb == blk;
             f.sc_off = off;
             f.pad = 0;
             if (f.first) off += G * f.n_blocks * NW;
@@ -268,7 +276,7 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
         }
     };
     load_batch(0);
-    if (tid == 0) {
+    if (!UNIT && tid == 0) {
         const long long start = clock64();
         for (int si = 0; si < nseg && !misc->failed; ++si) {
             if (fin[si].n_blocks == 1) continue;                               // a block's own warps arrived before its last barrier
@@ -360,7 +368,7 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
     warp_count(p.counters + CNT_IMPORTANT, n_imp);                             // Section 3.1's sparsity
     __threadfence();
     __syncthreads();
-    if (tid < nseg) {
+    if (!UNIT && tid < nseg) {
         const int si = tid, u = segs[si].u;
         const unsigned prev = atomicAdd(p.ticket2 + u, 1u);
         if (prev == (unsigned)(fin[si].n_blocks - 1)) {
@@ -452,8 +460,10 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
             }
         }
         if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+        if (UNIT && p.unit_stamp) __syncthreads();                      // every warp's row moves come before the stamp
         if (tid == 0) {
             p.live_out[u] = new_len;
+            if (UNIT) publish_unit_stamp(p, u, new_len);
             publish_live(p.maxlive, p.step + 1, new_len);
             atomicAdd(p.counters + CNT_APPENDED, 1ull);
             atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
@@ -465,11 +475,17 @@ __device__ void bal_finish_block(const DecodeParams& p, const BalSeg* segs, int 
     }
 }
 
-// FINISH: Algorithm 1 is finished inside this launch (bal_finish_block); otherwise the kernel only streams, lists each
-// unit's records in p.unit_rec and leaves verdicts and compaction to the verdict launch that follows it.
-template <int G, bool PAGED, bool FINISH>
+// MODE kBalStream: the kernel only streams, lists each unit's records in p.unit_rec and leaves verdicts and compaction
+// to the verdict launch that follows it. kBalFinish: Algorithm 1 is finished inside this launch by the blocks that
+// streamed a unit (bal_finish_block). kBalUnits: no balanced partition; grid (splits, units), a block streams one split
+// of one unit (p.split_len keys) and the unit's last-arriving block finishes it alone. No block of such a launch waits
+// for another, a finished unit leaves its stamp, and the launch may be chained to the previous step's (see
+// decode_fast_kernel): with many short units the steps then overlap unit by unit.
+constexpr int kBalStream = 0, kBalFinish = 1, kBalUnits = 2;
+template <int G, bool PAGED, int MODE>
 __global__ void __launch_bounds__(kBalThreads, kBalBlocksPerSm)
 decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_constant__ CUtensorMap vmap) {
+    constexpr bool FINISH = MODE == kBalFinish;
     extern __shared__ __align__(1024) unsigned char smem[];   // the swizzled V tiles want 1024-byte alignment
     constexpr int NT = kBalThreads, NW = kBalWarps;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -498,7 +514,47 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
         fence_mbar_init();
         fence_async_smem();
     }
-    asm volatile("griddepcontrol.wait;" ::: "memory");       // the previous launch on the stream has completed
+    if (MODE == kBalUnits) {
+        // ---- one split of one unit ----
+        const int u = (int)blockIdx.y, split = (int)blockIdx.x;
+        int l_old;
+        if (p.chain_wait) {                                   // this unit's previous step, not the previous launch
+            if (tid == 0) misc->stamp = wait_unit_stamp(p.unit_stamp + u, (uint32_t)p.step, p.status);
+            __syncthreads();
+            const unsigned long long sw = misc->stamp;
+            if ((uint32_t)(sw >> 32) != (uint32_t)p.step) return;   // the wait gave up (reported), or a block without a split
+            l_old = (int)(uint32_t)sw;
+            asm volatile("fence.proxy.async.global;" ::: "memory");   // the tile copies read rows that ordinary stores wrote
+        } else {
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            l_old = __ldcg(p.live_in + u);
+        }
+        const int l = l_old + 1;
+        const int room = PAGED ? __ldcg(p.page_room + u) : 1;
+        if (l > p.C || !room) {                               // a full slab or an exhausted pool: reported, the unit is left as it is
+            if (split == 0 && tid == 0) {
+                report_status(p.status, CORM_ERR_CAPACITY);
+                p.live_out[u] = l_old;
+                publish_unit_stamp(p, u, l_old);
+                publish_live(p.maxlive, p.step + 1, l_old);
+            }
+            return;
+        }
+        const int n_unit = (l + kTileKeys - 1) / kTileKeys, tps = p.split_len / kTileKeys;
+        const int n_act = (n_unit + tps - 1) / tps;
+        if (split >= n_act) return;
+        if (n_act > (int)gridDim.x && split == 0 && tid == 0) report_status(p.status, CORM_ERR_INTERNAL);   // the host's bound on the unit was wrong
+        if (p.early_trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // every block has its length by now
+        if (tid == 0) {
+            BalSeg sg;
+            sg.u = u; sg.l = l; sg.tile0 = split * tps; sg.n_tiles = min(tps, n_unit - split * tps); sg.gtile0 = 0;
+            sg.t = __ldcg(p.base_tokens + u / p.Hkv) + p.step + 1; sg.n_unit = n_unit; sg.pad = n_act;
+            segs[0] = sg;
+            s_nseg = 1; s_more = 0;
+        }
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the previous launch on the stream has completed
+    }
 
     // ---- the step's tile list: tiles per unit, block-wide prefix sums, this block's range ----
     // One round of global loads: every unit's length (and every sequence's token count) is parked in the ring area,
@@ -516,6 +572,9 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
     bool use_cache = cached;
     auto len_of = [&](int v) -> int { return use_cache ? s_L[v] : len_global(v); };
     auto tokens_of = [&](int v) -> int { return (use_cache ? s_bt[v / p.Hkv] : __ldcg(p.base_tokens + v / p.Hkv)) + p.step + 1; };
+    long long T = 0, S_b = 0, S_e = 0;
+    int win_u = 0, win_P = 0;
+    if (MODE != kBalUnits) {
     if (cached)
         for (int i = tid; i < n_seq; i += NT) s_bt[i] = __ldcg(p.base_tokens + i);
     int sum = 0;
@@ -539,11 +598,10 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
     if (lane == 31) s_wsum[warp] = incl;
     __syncthreads();
     int excl = incl - sum;
-    long long T = 0;
 #pragma unroll
     for (int w = 0; w < NW; ++w) { if (w < warp) excl += s_wsum[w]; T += s_wsum[w]; }
     if (T == 0) return;
-    const long long S_b = T * blk / nblk, S_e = T * (blk + 1) / nblk;
+    S_b = T * blk / nblk; S_e = T * (blk + 1) / nblk;
     if (S_b == S_e) return;                                    // more blocks than tiles
     if (sum > 0 && excl <= S_b && S_b < (long long)excl + sum) {
         int run = excl;
@@ -554,7 +612,8 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
         }
     }
     __syncthreads();
-    int win_u = s_first_u, win_P = s_first_P;
+    win_u = s_first_u; win_P = s_first_P;
+    }
 
     const int h = lane >> 4, ci = lane & 15;
     const int key_own = 16 * h + 8 * (ci & 1) + (ci >> 1);     // tile key this lane owns after the fold of qk_tile
@@ -566,7 +625,7 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
     bool failed = false;
 
     for (;;) {   // windows of at most kBalSegCap segments (one window unless units are tiny)
-        if (warp == 0) {
+        if (MODE != kBalUnits && warp == 0) {
             // lanes look at units win_u + lane; a unit with tiles that starts before the end of the range is a segment
             const int v = win_u + lane;
             const int l = v < U ? len_of(v) : 0, tv = (l + kTileKeys - 1) / kTileKeys;
@@ -825,8 +884,10 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
             // this segment stores M = -inf, Z = 0, acc = 0), then the warp's arrival: no block-wide step here, the
             // other warps of the block stream on.
             const size_t pstride = partial_stride(128);
-            unsigned char* rec_w = p.partials + ((size_t)(blk + u) * NW + warp) * G * pstride;   // blk + u is unique: both grow along the tile list
-            if (!CORM_IN_RANGE((size_t)(blk + u) * NW + warp < bal_record_count(nblk, p.U), p.status)) continue;
+            // blk + u is unique: both grow along the tile list; a block per split numbers the records by (unit, split)
+            const size_t rec_row = MODE == kBalUnits ? (size_t)u * bal_unit_splits(p.max_splits) + blockIdx.x : (size_t)(blk + u);
+            unsigned char* rec_w = p.partials + (rec_row * NW + warp) * G * pstride;
+            if (!CORM_IN_RANGE(MODE == kBalUnits || rec_row * NW + warp < bal_record_count(nblk, p.U), p.status)) continue;
             if (lane < G) {
                 double* mz = reinterpret_cast<double*>(rec_w + (size_t)lane * pstride);
                 double Mg = M[0], Zg = Zl[0];
@@ -851,8 +912,21 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
         __syncthreads();
         if (s_failed) return;                   // a bounded wait expired: reported through the status word
         // ---- Algorithm 1 for the slots this block streamed; the ring is free now ----
-        if (FINISH) {
-            bal_finish_block<G, PAGED, NT>(p, segs, nseg, blk, T, nblk, smem, misc);
+        if (MODE == kBalUnits) {
+            // every warp's record is stored and fenced (barriers above): the split arrives; the last one finishes the unit
+            if (tid == 0) {
+                const int u = segs[0].u, n_act = segs[0].pad;
+                const unsigned prev = atomicAdd(p.ticket + u, 1u);
+                misc->last = prev == (unsigned)(n_act - 1);
+                if (misc->last) { p.ticket[u] = 0u; segs[0].tile0 = 0; segs[0].n_tiles = segs[0].n_unit; }
+                __threadfence();
+            }
+            __syncthreads();
+            if (!misc->last) return;
+            bal_finish_block<G, PAGED, NT, true>(p, segs, 1, blk, T, nblk, smem, misc);
+            return;
+        } else if (FINISH) {
+            bal_finish_block<G, PAGED, NT, false>(p, segs, nseg, blk, T, nblk, smem, misc);
             if (s_failed) return;
         } else {
             // the verdict launch may become resident now; it reads nothing of this launch before it has completed
@@ -940,7 +1014,7 @@ inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& 
                                                                                     : launch(decode_balanced_kernel<4, true, FIN>))  \
                   : (G == 1 ? launch(decode_balanced_kernel<1, false, FIN>) : G == 2 ? launch(decode_balanced_kernel<2, false, FIN>) \
                                                                                      : launch(decode_balanced_kernel<4, false, FIN>)))
-    rc = verdict_launch ? CORM_BAL(false) : CORM_BAL(true);
+    rc = verdict_launch ? CORM_BAL(kBalStream) : CORM_BAL(kBalFinish);
 #undef CORM_BAL
     if (rc != CORM_OK) return rc;
     *n_launched = 1;
@@ -970,6 +1044,65 @@ inline corm_status_t launch_decode_balanced(DecodeParams& p, const CUtensorMap& 
     rc = G == 1 ? launch_v(decode_verdict_kernel<bf16_t, 128, 1, true>) : G == 2 ? launch_v(decode_verdict_kernel<bf16_t, 128, 2, true>)
                                                                                  : launch_v(decode_verdict_kernel<bf16_t, 128, 4, true>);
     if (rc == CORM_OK) *n_launched = 2;
+    return rc;
+}
+
+// The same streaming loop with a block per split of a unit and the unit finished by its last-arriving split
+// (kBalUnits): one launch per step, no block waits for another, units leave stamps, so consecutive steps can be
+// chained (want_chain / want_trigger as for launch_decode_fast). Meant for many units of a few thousand keys at most:
+// the finishing block walks its whole unit alone.
+inline corm_status_t launch_decode_balanced_units(DecodeParams& p, const CUtensorMap& vmap, int G, int upper, int typical,
+                                                  int tune_split_len, int sm_count, size_t partial_capacity_records,
+                                                  cudaStream_t st, int* n_launched, bool want_chain, bool want_trigger) {
+    *n_launched = 0;
+    if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
+    if (p.C > kBalMaxTokens) return CORM_ERR_UNSUPPORTED;
+    const int sms = sm_count > 0 ? sm_count : 148;
+    const int grain = kBalWarps * kTileKeys;                       // a tile per warp at least
+    int split_len = tune_split_len;
+    if (!split_len) {
+        // about one and a half blocks per resident slot over the whole step, from the mean unit where the host knows it
+        // (128 units of 1660 keys, us per step: splits of 256 keys 47.4, 384 43.4, 512 42.5, 640 44.4, 896 47.8)
+        const long long keys = (long long)(typical > 0 ? typical : upper) * p.U;
+        split_len = (int)(2 * keys / (3ll * sms * kBalBlocksPerSm));
+        if (split_len > 2048) split_len = 2048;
+    }
+    const int max_unit_splits = bal_unit_splits(p.max_splits);     // records a unit has room for, in splits
+    if (split_len < (upper + max_unit_splits - 1) / max_unit_splits) split_len = (upper + max_unit_splits - 1) / max_unit_splits;
+    split_len = (split_len + grain - 1) / grain * grain;
+    if (split_len < grain) split_len = grain;
+    const int n_splits = (upper + split_len - 1) / split_len;
+    if (n_splits > max_unit_splits || (size_t)p.U * max_unit_splits * kBalWarps > partial_capacity_records) return CORM_ERR_UNSUPPORTED;
+    if ((size_t)G * n_splits * kBalWarps > 7000 || n_splits > 65535) return CORM_ERR_UNSUPPORTED;   // scale factors of a unit's records: shared memory
+    p.split_len = split_len;
+    p.chain_wait = want_chain && p.unit_stamp ? 1 : 0;
+    p.early_trigger = want_trigger ? 1 : 0;
+    constexpr int kTotal[5] = {0, bal_smem_layout(1).total, bal_smem_layout(2).total, 0, bal_smem_layout(4).total};
+    const size_t smem = (size_t)kTotal[G];
+    auto launch = [&](auto kern) -> corm_status_t {
+        cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: cudaFuncSetAttribute: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)n_splits, (unsigned)p.U);
+        cfg.blockDim = dim3(kBalThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kern, p, vmap);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { std::fprintf(stderr, "corm: decode launch: %s\n", cudaGetErrorString(e)); return CORM_ERR_CUDA; }
+        return CORM_OK;
+    };
+    const corm_status_t rc =
+        p.page_table ? (G == 1 ? launch(decode_balanced_kernel<1, true, kBalUnits>) : G == 2 ? launch(decode_balanced_kernel<2, true, kBalUnits>)
+                                                                                             : launch(decode_balanced_kernel<4, true, kBalUnits>))
+                     : (G == 1 ? launch(decode_balanced_kernel<1, false, kBalUnits>) : G == 2 ? launch(decode_balanced_kernel<2, false, kBalUnits>)
+                                                                                              : launch(decode_balanced_kernel<4, false, kBalUnits>));
+    if (rc == CORM_OK) *n_launched = 1;
     return rc;
 }
 

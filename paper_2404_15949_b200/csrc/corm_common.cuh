@@ -68,6 +68,10 @@ struct DecodeParams {
     unsigned char* partials;  // [U][max_splits][G] records {double m, double Z, float acc[D]} (scratch)
     uint32_t* keepmask;       // [U][ceil(C/32)+2] keep bits of the verdict launch (scratch)
     int2* unit_rec;           // [U] balanced kernel -> verdict launch: a unit's first record and its record count (scratch)
+    unsigned long long* unit_stamp;  // [U] (decode steps the unit has finished << 32 | its live length after the last of them),
+                                     // written by the block that finishes a unit inside the streaming launch; null = not kept
+    int32_t chain_wait;       // fast kernel: a block waits for its own unit's stamp of the previous step, not for the previous launch
+    int32_t early_trigger;    // fast kernel: the next launch on the stream may become resident once every block of this one has started
     const void* q;            // [B][Hq][D]
     const void* k_new;        // [B][Hkv][D]
     const void* v_new;        // [B][Hkv][D]
@@ -107,6 +111,16 @@ struct PromptParams {
 };
 
 __host__ __device__ inline size_t partial_stride(int D) { return 16 + 4 * (size_t)D; }
+
+// A unit's step is complete: every write of the block that finished it (row moves, registers, positions) comes before
+// the stamp, which a block of the next step's launch may be waiting for (wait_unit_stamp). Called by one thread after
+// a block barrier that follows those writes.
+__device__ __forceinline__ void publish_unit_stamp(const DecodeParams& p, int u, int new_len) {
+    if (!p.unit_stamp) return;
+    const unsigned long long v = ((unsigned long long)(uint32_t)(p.step + 1) << 32) | (uint32_t)new_len;
+    __threadfence();
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p.unit_stamp + u), "l"(v) : "memory");
+}
 
 // ---- element access: the cache dtype is only a storage format; all logits are formed in fp64 ----
 struct bf16_t { uint16_t bits; };
@@ -518,8 +532,10 @@ __device__ void finalize_unit(const DecodeParams& p, int u, int b, int l, int n_
         }
     }
     settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+    if (p.unit_stamp) __syncthreads();            // the row moves of every warp come before the stamp
     if (tid == 0) {
         p.live_out[u] = new_len;
+        publish_unit_stamp(p, u, new_len);
         publish_live(p.maxlive, p.step + 1, new_len);
         atomicAdd(p.counters + CNT_APPENDED, 1ull);
         atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);

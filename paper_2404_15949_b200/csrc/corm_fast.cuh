@@ -85,6 +85,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (clock64() - start > kWaitLimitCycles) return false;
     return true;
 }
+// Waits until the unit's stamp says that at least `steps_done` decode steps of it are complete and returns the stamp.
+// Gives up (all ones) after kWaitLimitCycles, reporting a timeout, or as soon as another block has reported a
+// failure that leaves the cache unusable anyway.
+__device__ __forceinline__ unsigned long long wait_unit_stamp(const unsigned long long* stamp, uint32_t steps_done, int32_t* status) {
+    const long long start = clock64();
+    for (;;) {
+        unsigned long long v;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(stamp) : "memory");
+        if ((uint32_t)(v >> 32) >= steps_done) return v;
+        const int32_t s = *reinterpret_cast<volatile int32_t*>(status);
+        if (s == CORM_ERR_TIMEOUT || s == CORM_ERR_INTERNAL) return ~0ull;
+        if (clock64() - start > kWaitLimitCycles) { report_status(status, CORM_ERR_TIMEOUT); return ~0ull; }
+        __nanosleep(64);
+    }
+}
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src_gmem, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst_smem), "l"(src_gmem), "r"(bytes), "r"(bar) : "memory");
@@ -260,8 +275,10 @@ __device__ void finalize_single(const DecodeParams& p, int u, int b, int l, int 
         }
     }
     if (PAGED) settle_pages<NT>(p.page_table, p.page_bits, p.page_room, p.pool_pages, p.pt_stride, p.U, u, l - 1, new_len);
+    if (p.unit_stamp) __syncthreads();            // the row moves and register writes of every warp come before the stamp
     if (tid == 0) {
         p.live_out[u] = new_len;
+        publish_unit_stamp(p, u, new_len);
         publish_live(p.maxlive, p.step + 1, new_len);
         atomicAdd(p.counters + CNT_APPENDED, 1ull);
         atomicAdd(p.counters + CNT_ATTENDED, (unsigned long long)l);
@@ -287,22 +304,50 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     // without a page for the appended row (pool exhausted) is treated like a full slab.
     __shared__ int32_t s_pt[kFastWarps][32];
     const int32_t* pt_u = PAGED ? p.page_table + (size_t)u * p.pt_stride : nullptr;
-    // launched with programmatic stream serialization: the block may start while the previous launch on the stream
-    // drains and reads nothing before that launch has completed
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Launched with programmatic stream serialization: the block may start while the previous launch on the stream
+    // drains. Ordinarily it reads nothing before that launch has completed. A chained launch (the previous launch was
+    // the previous decode step of these same units and finished every unit inside itself) waits for less: only for
+    // its own unit's previous step, whose finishing block left a stamp (steps done, live length) behind all its
+    // writes. Units are independent, so nothing else of the previous launch concerns this block, and the blocks of
+    // consecutive steps fill one another's last waves.
+    int l_old;
+    if (p.chain_wait) {
+        __shared__ unsigned long long s_stamp;
+        if (tid == 0) s_stamp = wait_unit_stamp(p.unit_stamp + u, (uint32_t)p.step, p.status);
+        __syncthreads();
+        const unsigned long long sw = s_stamp;
+        // not this step's stamp: the wait gave up (reported), or the unit is already past this step, which only a
+        // block that has no split to work on can find
+        if ((uint32_t)(sw >> 32) != (uint32_t)p.step) return;
+        l_old = (int)(uint32_t)sw;
+        asm volatile("fence.proxy.async.global;" ::: "memory");     // the bulk copies below read rows that ordinary stores wrote
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        l_old = __ldcg(p.live_in + u);
+    }
     int32_t my_page = 0, room = 1;
     if (PAGED) {
         const int idx = split * (p.split_len >> 5) + warp + lane * kFastWarps;
         if (idx < p.pt_stride) my_page = __ldcg(pt_u + idx);
         room = __ldcg(p.page_room + u);
     }
-    const int l_old = __ldcg(p.live_in + u), l = l_old + 1;
+    const int l = l_old + 1;
     if (l > p.C || !room) {
-        if (split == 0 && tid == 0) { report_status(p.status, CORM_ERR_CAPACITY); p.live_out[u] = l_old; publish_live(p.maxlive, p.step + 1, l_old); }
+        if (split == 0 && tid == 0) {
+            report_status(p.status, CORM_ERR_CAPACITY);
+            p.live_out[u] = l_old;
+            publish_unit_stamp(p, u, l_old);
+            publish_live(p.maxlive, p.step + 1, l_old);
+        }
         return;
     }
     const int n_act = (l + p.split_len - 1) / p.split_len;
     if (split >= n_act) return;
+    if (n_act > (int)gridDim.x && split == 0 && tid == 0) report_status(p.status, CORM_ERR_INTERNAL);   // the host's bound on the unit was wrong
+    // From here on the next launch may become resident (a chained one: its blocks wait for their units' stamps). Not
+    // earlier: an unchained block takes its unit's length from the double-buffered array, whose other half the next
+    // step rewrites, so every block has its length (the branch above depends on it) before a block of the next step runs.
+    if (p.early_trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const bool single = (n_act == 1 && l <= p.single_cap);
     const int t = __ldg(p.base_tokens + b) + p.step + 1;
     const int begin = split * p.split_len, end = min(l, begin + p.split_len);
@@ -508,7 +553,7 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
     // The verdict launch that may follow is allowed to become resident once every block of this grid is past its
     // tiles (it waits for this grid to complete before it reads anything written here). Allowing it from the top of
     // the kernel costs 1.4 us per step on 128 units of 1600 keys: its waiting blocks take room next to streaming ones.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!p.early_trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // fold the warp: lane-private sums of Z, the two halves of acc
     float acc[G][8];
@@ -597,9 +642,13 @@ __global__ void __launch_bounds__(kFastThreads, fast_blocks_per_sm(G)) decode_fa
 
 // Host side: split length and launch. Returns CORM_ERR_UNSUPPORTED for group sizes the kernel does not cover.
 // upper bounds every unit's live length; typical is the mean live length as far as the host knows it (0 = unknown).
+// want_chain / want_trigger: what the caller would like for p.chain_wait / p.early_trigger; granted only when this
+// launch finishes every unit inside itself (*self_finishing), which is also what lets the next launch be chained.
 inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int typical, int tune_split_len, int sm_count,
-                                        cudaStream_t st, int* n_launched, int finish_mode) {
+                                        cudaStream_t st, int* n_launched, int finish_mode, bool want_chain = false,
+                                        bool want_trigger = false, bool* self_finishing = nullptr) {
     *n_launched = 0;
+    if (self_finishing) *self_finishing = false;
     if (G != 1 && G != 2 && G != 4) return CORM_ERR_UNSUPPORTED;
     // longest unit that can finish inside one block: bounded by the verdict registers a thread carries and by the
     // shared memory that holds the unit's logits
@@ -662,6 +711,11 @@ inline corm_status_t launch_decode_fast(DecodeParams& p, int G, int upper, int t
     const bool many = finish_mode == 2 || (finish_mode != 3 && ((long long)p.U * n_splits >= 4ll * sms * fast_blocks_per_sm(G) ||
                                                                 (long long)upper * G <= 2048));
     p.inline_finalize = !all_single && many && fin <= smem;
+    const bool self = all_single || p.inline_finalize;
+    if (self_finishing) *self_finishing = self;
+    if (!self) p.unit_stamp = nullptr;            // the verdict launch finishes (some of) the units: no stamps, no chain
+    p.chain_wait = want_chain && p.unit_stamp ? 1 : 0;
+    p.early_trigger = want_trigger && self ? 1 : 0;
     const size_t fin1 = (size_t)kFastWarps * G * (16 + 512) + (size_t)2 * ((p.single_cap + 31) / 32 + 2) * 4 +
                         (size_t)2 * p.single_cap * 4;
     if (fin1 > (size_t)kFastWarps * fast_warp_bytes(G)) return CORM_ERR_UNSUPPORTED;

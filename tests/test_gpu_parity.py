@@ -329,3 +329,63 @@ def test_state_errors_on_gpu():
     assert e.value.status == 4
     with pytest.raises(CormError):
         gpu.corm_decode_step(1, x, x, x)                             # layer out of range
+
+
+CHAINED = [
+    # G, n_kv, batch, layers, prompt range, steps, w, r, split_len, tuning, pool_pages
+    (1, 32, 10, 1, (150, 500), 44, 8, 32, 0, 1, 0),        # 320 short units: one block each, every launch self-finishing
+    (1, 32, 10, 1, (150, 500), 44, 8, 32, 0, 1, 8192),     # ... on a paged cache
+    (1, 3, 2, 1, (150, 330), 40, 8, 16, 64, 2, 0),         # units of several splits, finished by the last-arriving split
+    (4, 2, 2, 1, (97, 257), 36, 4, 8, 128, 2, 0),          # grouped heads on the block-per-split kernel
+    (1, 8, 1, 4, (260, 260), 30, 8, 32, 0, 1, 0),          # four layers as one launch per step
+    (4, 2, 2, 1, (97, 257), 36, 4, 8, 0, 1, 0),            # grouped heads, automatic: a block per split inside such a call
+    (4, 1, 1, 1, (3000, 3000), 12, 8, 64, 0, 1, 0),        # one long unit: balanced kernel + verdict launch, nothing to chain
+    (4, 8, 6, 1, (150, 700), 44, 8, 32, 128, 6, 0),        # grouped heads, tensor-core loop, a block per split of 128 keys
+    (4, 8, 6, 1, (150, 700), 44, 8, 32, 0, 6, 4096),       # ... automatic split length, paged cache
+    (2, 3, 2, 1, (1, 40), 60, 8, 4, 0, 6, 0),              # tiny units (empty splits), two heads per group
+    (1, 3, 2, 1, (150, 330), 40, 8, 16, 128, 6, 0),        # one head per KV head on that kernel
+    (4, 2, 1, 3, (260, 260), 30, 8, 32, 0, 6, 0),          # three layers as one launch per step
+]
+
+
+@pytest.mark.parametrize("G,n_kv,batch,n_layers,prange,steps,w,r,split_len,tuning,pool_pages", CHAINED)
+def test_many_steps_from_one_call(G, n_kv, batch, n_layers, prange, steps, w, r, split_len, tuning, pool_pages):
+    """corm_decode_steps: several decode steps enqueued by one call, each launch chained to the previous one where
+    the kernels allow it (a block waits for its own unit's previous step only). Outputs of every step and the states
+    between calls equal the oracle's, which steps one call at a time."""
+    cfg = CONFIGS[2].with_(n_layers=n_layers, batch=batch, n_q_heads=n_kv * G, n_kv_heads=n_kv, prompt_min=prange[0],
+                           prompt_max=prange[1], steps=steps, window_w=w, recent_r=r, dense_layers=0,
+                           gqa_rho=0.7 if G > 1 else 0.0)
+    gpu = make_gpu_cache(cfg, batch, n_kv, n_layers=n_layers, pool_pages=pool_pages)
+    orc = make_oracle(cfg, batch, n_kv, n_layers=n_layers)
+    gpu.corm_cache_set_tuning(split_len, tuning)
+    datas = [generate(cfg, layer=l) for l in range(n_layers)]
+    dt = cfg.dtype
+    for l, d in enumerate(datas):
+        gpu.corm_compress_prompt(l, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+        orc.compress_prompt(l, d.k_prompt, d.v_prompt, d.q_last, d.prompt_lens)
+    q_all = torch.stack([to_dev(d.q[:steps], dt) for d in datas], dim=1).contiguous()      # [steps, layers, ...]
+    k_all = torch.stack([to_dev(d.k_new[:steps], dt) for d in datas], dim=1).contiguous()
+    v_all = torch.stack([to_dev(d.v_new[:steps], dt) for d in datas], dim=1).contiguous()
+    s0 = 0
+    for chunk in (1, 7, 16, 3, steps):                       # calls of different lengths, the last takes what is left
+        s1 = min(steps, s0 + chunk)
+        out = gpu.corm_decode_steps(0, n_layers, q_all[s0:s1], k_all[s0:s1], v_all[s0:s1]).float().cpu().numpy()
+        for s in range(s0, s1):
+            for l, d in enumerate(datas):
+                ref = orc.decode_step(l, d.q[s], d.k_new[s], d.v_new[s])
+                assert np.abs(out[s - s0, l] - ref).max() <= OUT_TOL[dt], (s, l)
+        for l in range(n_layers):
+            assert_states_equal(gpu, orc, l, batch, n_kv, f"after step {s1 - 1} layer {l}")
+        s0 = s1
+    st = gpu.corm_cache_stats()
+    assert st["device_status"] == 0 and st["evicted_keys"] == orc.counters()["evicted"] > 0
+    assert orc.counters()["near_threshold"] == 0
+    chained = gpu.corm_cache_chained_launches()
+    if G > 1 and tuning == 1 and prange[1] > 96 * batch * n_kv * n_layers:
+        assert chained == 0
+    else:     # every launch after a call's first, as long as each finished its units itself
+        assert chained >= steps // 2, chained
+    if pool_pages:
+        used, _ = gpu.corm_cache_pool_usage(0)
+        assert used == int((orc.live_lens(0) // 32 + 1).sum())
