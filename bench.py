@@ -271,17 +271,27 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
         h2d = L * (qh[0][0].numel() + 2 * kh[0][0].numel()) * oh.element_size()
         d2h = L * oh.numel() * oh.element_size()
         hviews = [[(qh[l][s], kh[l][s], vh[l][s]) for l in range(L)] for s in range(n_steps)]
+        if args.api == "steps":
+            qs, ks, vs = pin(q_all), pin(k_all), pin(v_all)
+            os_ = torch.empty_like(qs).pin_memory()
+
+        def run_host(s0, s1):
+            if s1 <= s0:
+                return
+            if args.api == "steps":
+                cache.corm_decode_steps_host(0, L, qs[s0:s1], ks[s0:s1], vs[s0:s1], os_[s0:s1])
+            else:
+                for s in range(s0, s1):
+                    for l in range(L):
+                        cache.corm_decode_step_host(l, *hviews[s][l], oh)
+
         restore()
-        for s in range(args.warmup):
-            for l in range(L):
-                cache.corm_decode_step_host(l, *hviews[s][l], oh)
+        run_host(0, args.warmup)
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         a.record()
-        for s in range(args.warmup, n_steps):
-            for l in range(L):
-                cache.corm_decode_step_host(l, *hviews[s][l], oh)
+        run_host(args.warmup, n_steps)
         b.record()
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(b)
@@ -314,7 +324,8 @@ def measure_workload(cfg, args, local, world, rank, want_e2e, want_clocks):
                                 else "decode_fast_kernel") + f" ({launches_per_step:.2f} launches per layer per step, all counted in the time)",
                      "bytes_per_launch": abytes / (args.steps * L), "us_per_launch": 1e3 * med["ms"] / (args.steps * L)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": "the same decode steps as `value`, from the same restored state"},
+                "steps": "the same decode steps as `value`, from the same restored state",
+                "api": "corm_decode_steps_host" if args.api == "steps" else "corm_decode_step_host per step and layer"},
         "gpu_launches": med["launches"], "host_issue_us_per_step": 1e3 * med["issue_ms"] / args.steps,
         "api": ("corm_decode_steps: the timed steps enqueued by one call" if args.api == "steps" else
                 "one corm_decode_step" + ("_layers" if L > 1 else "") + " call per step"),

@@ -185,6 +185,13 @@ corm_status_t corm_decode_step_layers(corm_cache_t* cache, int32_t first_layer, 
 corm_status_t corm_decode_steps(corm_cache_t* cache, int32_t first_layer, int32_t n_layers, int32_t n_steps,
                                 const void* q, const void* k_new, const void* v_new, void* out, void* stream);
 
+/* corm_decode_steps with HOST buffers of the same layout, asynchronous on `stream`. Pinned, mapped buffers are read
+ * and written in place by the kernels (as corm_decode_step_host does); any other host memory goes step by step and
+ * layer by layer through the staging buffers. Errors: as corm_decode_steps. */
+corm_status_t corm_decode_steps_host(corm_cache_t* cache, int32_t first_layer, int32_t n_layers, int32_t n_steps,
+                                     const void* q_host, const void* k_new_host, const void* v_new_host, void* out_host,
+                                     void* stream);
+
 /* Same step with HOST buffers, asynchronous on `stream` (out_host is valid once the stream has been synchronised).
  * Pinned buffers the device can address (cudaHostAlloc / cudaHostRegister, 16-byte aligned) are read and written by
  * the kernels directly across the bus, with no copies; any other host memory is copied to staging space inside the

@@ -79,6 +79,8 @@ def load_library():
     lib.corm_decode_step_layers.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.corm_decode_steps.restype = i32
     lib.corm_decode_steps.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.corm_decode_steps_host.restype = i32
+    lib.corm_decode_steps_host.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.corm_cache_chained_launches.restype = i64
     lib.corm_cache_chained_launches.argtypes = [vp]
     lib.corm_cache_stats.restype = i32
@@ -235,6 +237,18 @@ class CormCache:
             self.handle, first_layer, n_layers, n_steps, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
             _stream_ptr(stream)))
         return out.squeeze(1) if squeeze else out
+
+    def corm_decode_steps_host(self, first_layer, n_layers, q, k_new, v_new, out, stream=None):
+        """corm_decode_steps on host tensors ``[n_steps, n_layers, ...]`` (pinned ones are used in place)."""
+        n_steps = q.shape[0]
+        for t, shape in ((q, self._q_shape), (out, self._q_shape), (k_new, self._kv_shape), (v_new, self._kv_shape)):
+            if not (tuple(t.shape) == (n_steps, n_layers) + tuple(shape) and t.dtype == self.dtype and not t.is_cuda and
+                    t.is_contiguous()):
+                raise ValueError("corm_decode_steps_host: contiguous host tensors [n_steps, n_layers, ...] of the cache dtype")
+        _check("corm_decode_steps_host", self.lib.corm_decode_steps_host(
+            self.handle, first_layer, n_layers, n_steps, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+            _stream_ptr(stream)))
+        return out
 
     def corm_cache_chained_launches(self):
         return int(self.lib.corm_cache_chained_launches(self.handle))

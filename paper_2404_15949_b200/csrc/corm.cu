@@ -685,9 +685,11 @@ corm_status_t corm_decode_step_layers(corm_cache_t* c, int32_t first_layer, int3
     return CORM_OK;
 }
 
-corm_status_t corm_decode_steps(corm_cache_t* c, int32_t first_layer, int32_t n_layers, int32_t n_steps, const void* q,
+}  // extern "C"
+
+namespace {
+corm_status_t decode_steps_impl(corm_cache_t* c, int32_t first_layer, int32_t n_layers, int32_t n_steps, const void* q,
                                 const void* k_new, const void* v_new, void* out, void* stream) {
-    NvtxRange nvtx_range("corm_decode_steps");
     if (!c || n_layers < 1 || n_steps < 0 || !layer_ok(c, first_layer) || !layer_ok(c, first_layer + n_layers - 1))
         return CORM_ERR_INVALID_ARG;
     if (n_steps == 0) return CORM_OK;
@@ -729,6 +731,51 @@ corm_status_t corm_decode_steps(corm_cache_t* c, int32_t first_layer, int32_t n_
             if (rc != CORM_OK) return rc;
         }
     }
+    return CORM_OK;
+}
+}  // namespace
+
+extern "C" {
+
+corm_status_t corm_decode_steps(corm_cache_t* c, int32_t first_layer, int32_t n_layers, int32_t n_steps, const void* q,
+                                const void* k_new, const void* v_new, void* out, void* stream) {
+    NvtxRange nvtx_range("corm_decode_steps");
+    return decode_steps_impl(c, first_layer, n_layers, n_steps, q, k_new, v_new, out, stream);
+}
+
+corm_status_t corm_decode_steps_host(corm_cache_t* c, int32_t first_layer, int32_t n_layers, int32_t n_steps,
+                                     const void* q_host, const void* k_new_host, const void* v_new_host, void* out_host,
+                                     void* stream) {
+    NvtxRange nvtx_range("corm_decode_steps_host");
+    if (!c || n_layers < 1 || n_steps < 0 || !layer_ok(c, first_layer) || !layer_ok(c, first_layer + n_layers - 1))
+        return CORM_ERR_INVALID_ARG;
+    if (n_steps == 0) return CORM_OK;
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return CORM_ERR_INVALID_ARG;
+    {   // pinned, mapped buffers: the kernels read and write them in place, exactly as corm_decode_steps would
+        DeviceGuard guard(c->cfg.device);
+        if (!guard.ok) return CORM_ERR_CUDA;
+        const void* in[4] = {q_host, k_new_host, v_new_host, out_host};
+        void* dev[4] = {nullptr, nullptr, nullptr, nullptr};
+        bool mapped = true;
+        for (int i = 0; i < 4 && mapped; ++i) {
+            cudaPointerAttributes at{};
+            if (cudaPointerGetAttributes(&at, in[i]) != cudaSuccess) { (void)cudaGetLastError(); mapped = false; break; }
+            mapped = at.type == cudaMemoryTypeHost && at.devicePointer && reinterpret_cast<uintptr_t>(at.devicePointer) % 16 == 0;
+            dev[i] = at.devicePointer;
+        }
+        if (mapped) return decode_steps_impl(c, first_layer, n_layers, n_steps, dev[0], dev[1], dev[2], dev[3], stream);
+    }
+    // any other host memory: step by step and layer by layer through the staging buffers
+    const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * c->cfg.head_dim * c->e, kb = (size_t)c->U * c->cfg.head_dim * c->e;
+    for (int s = 0; s < n_steps; ++s)
+        for (int i = 0; i < n_layers; ++i) {
+            const size_t ix = (size_t)s * n_layers + i;
+            const corm_status_t rc = corm_decode_step_host(c, first_layer + i, static_cast<const unsigned char*>(q_host) + ix * qb,
+                                                           static_cast<const unsigned char*>(k_new_host) + ix * kb,
+                                                           static_cast<const unsigned char*>(v_new_host) + ix * kb,
+                                                           static_cast<unsigned char*>(out_host) + ix * qb, stream);
+            if (rc != CORM_OK) return rc;
+        }
     return CORM_OK;
 }
 

@@ -389,3 +389,30 @@ def test_many_steps_from_one_call(G, n_kv, batch, n_layers, prange, steps, w, r,
     if pool_pages:
         used, _ = gpu.corm_cache_pool_usage(0)
         assert used == int((orc.live_lens(0) // 32 + 1).sum())
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_many_steps_from_host_buffers(pinned):
+    """corm_decode_steps_host: pinned buffers are read and written in place by the (chained) launches, pageable ones
+    go through the staging buffers step by step; same results either way."""
+    G, n_kv, batch, steps = 1, 32, 10, 24
+    cfg = CONFIGS[2].with_(n_layers=1, batch=batch, n_q_heads=n_kv * G, n_kv_heads=n_kv, prompt_min=150, prompt_max=400,
+                           steps=steps, window_w=8, recent_r=32, dense_layers=0)
+    gpu, orc = make_gpu_cache(cfg, batch, n_kv), make_oracle(cfg, batch, n_kv)
+    d = generate(cfg)
+    dt = cfg.dtype
+    gpu.corm_compress_prompt(0, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+    orc.compress_prompt(0, d.k_prompt, d.v_prompt, d.q_last, d.prompt_lens)
+    host = lambda a: (lambda t: t.pin_memory() if pinned else t)(to_dev(a[:steps], dt).unsqueeze(1).contiguous().cpu())
+    q, k, v = host(d.q), host(d.k_new), host(d.v_new)
+    out = torch.empty_like(q)
+    out = out.pin_memory() if pinned else out
+    gpu.corm_decode_steps_host(0, 1, q, k, v, out)
+    torch.cuda.synchronize()
+    res = out.float().numpy()
+    for s in range(steps):
+        ref = orc.decode_step(0, d.q[s], d.k_new[s], d.v_new[s])
+        assert np.abs(res[s, 0] - ref).max() <= OUT_TOL[dt], s
+    assert_states_equal(gpu, orc, 0, batch, n_kv, "after the call")
+    assert gpu.corm_cache_stats()["device_status"] == 0
+    assert (gpu.corm_cache_chained_launches() > 0) == pinned
