@@ -3,7 +3,8 @@ the configurations' whole horizons.
 
 The CUDA library steps the whole configuration for every decode step it defines (256 / 512 / 256 / 1024); the CPU
 oracle steps a sample of its units (they are independent, and the generator yields identical slices for any subset),
-free-running from the prompt pass with no resynchronisation. Outputs of the sampled units must agree within the
+free-running from the prompt pass with no resynchronisation, once through one corm_decode_steps call per 32 steps
+(the benchmark's calls) and once through one call per step. Outputs of the sampled units must agree within the
 cache dtype's tolerance at every step; registers, positions and rows must be bit-exact every 32 steps and at the
 end, with the library enqueued far ahead of the host in between, as in the benchmark. That reaches the launch shapes
 the benchmark spends its time in: one block per unit on the batch-32 workload, the balanced kernel on the grouped
@@ -34,8 +35,12 @@ CASES = [
 CHECK_EVERY = 32
 
 
+@pytest.mark.parametrize("api", ["steps", "step"])
 @pytest.mark.parametrize("case", CASES, ids=lambda c: f"config{c[0]}")
-def test_full_size_sampled_units(case):
+def test_full_size_sampled_units(case, api):
+    """api "steps": every layer of the configuration is stepped, 32 steps per corm_decode_steps call (what bench.py
+    times: all layers of a step as one launch, launches chained); "step": one corm_decode_step call per step for the
+    sampled layers."""
     from paper_2404_15949_b200.binding import CormCache
     which, layers, seqs, heads_by_layer, expect_zero_near = case
     cfg = CONFIGS[which]
@@ -43,15 +48,19 @@ def test_full_size_sampled_units(case):
     G, dt = cfg.group, cfg.dtype
     gpu = CormCache(cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.max_tokens,
                     cfg.window_w, cfg.recent_r, cfg.alpha, dt, 0)           # default tuning = what bench.py times
-    oracles, full = {}, {}
-    for l in layers:
-        full[l] = generate(cfg, layer=l, n_steps=steps)
+    oracles, full, lens = {}, {}, {}
+    stepped = list(range(cfg.n_layers)) if api == "steps" else layers
+    for l in stepped:
+        d = generate(cfg, layer=l, n_steps=steps)
+        gpu.corm_compress_prompt(l, to_dev(d.k_prompt, dt), to_dev(d.v_prompt, dt), to_dev(d.q_last, dt), d.prompt_lens)
+        d.k_prompt = d.v_prompt = None                          # the prompts of 32 layers would not fit the host
+        full[l], lens[l] = d, d.prompt_lens
+        if l not in layers:
+            continue
         heads = heads_by_layer[l]
         sub = generate(cfg, layer=l, seqs=seqs, kv_heads=heads, n_steps=steps)
         orc = make_oracle(cfg, len(seqs), len(heads))
         orc.compress_prompt(0, sub.k_prompt, sub.v_prompt, sub.q_last, sub.prompt_lens)
-        gpu.corm_compress_prompt(l, to_dev(full[l].k_prompt, dt), to_dev(full[l].v_prompt, dt),
-                                 to_dev(full[l].q_last, dt), full[l].prompt_lens)
         oracles[l] = (orc, sub, heads)
 
     def check_states(tag):
@@ -70,14 +79,23 @@ def test_full_size_sampled_units(case):
 
     check_states("after prompt")
     worst = 0.0
-    dev_in = {l: tuple(to_dev(a, dt) for a in (full[l].q, full[l].k_new, full[l].v_new)) for l in layers}
+    if api == "steps":                                          # [step][layer][...] as corm_decode_steps takes them
+        q_all, k_all, v_all = (torch.stack([to_dev(getattr(full[l], name), dt) for l in stepped], dim=1).contiguous()
+                               for name in ("q", "k_new", "v_new"))
+    else:
+        dev_in = {l: tuple(to_dev(a, dt) for a in (full[l].q, full[l].k_new, full[l].v_new)) for l in layers}
     for s0 in range(0, steps, CHECK_EVERY):
         chunk = range(s0, min(steps, s0 + CHECK_EVERY))
-        outs = {l: [] for l in layers}
-        for s in chunk:                                        # the library runs ahead of the host for a whole chunk
-            for l in layers:
-                qd, kd, vd = dev_in[l]
-                outs[l].append(gpu.corm_decode_step(l, qd[s], kd[s], vd[s]))
+        if api == "steps":
+            s1 = chunk[-1] + 1
+            out_all = gpu.corm_decode_steps(0, cfg.n_layers, q_all[s0:s1], k_all[s0:s1], v_all[s0:s1])
+            outs = {l: list(out_all[:, l]) for l in layers}
+        else:
+            outs = {l: [] for l in layers}
+            for s in chunk:                                    # the library runs ahead of the host for a whole chunk
+                for l in layers:
+                    qd, kd, vd = dev_in[l]
+                    outs[l].append(gpu.corm_decode_step(l, qd[s], kd[s], vd[s]))
         for l in layers:
             orc, sub, heads = oracles[l]
             got = torch.stack(outs[l]).float().cpu().numpy()
@@ -96,7 +114,9 @@ def test_full_size_sampled_units(case):
     st = gpu.corm_cache_stats()
     assert st["device_status"] == 0
     # properties that hold at any size: every unit keeps at least its recent window, never more than it was given
-    for l in layers:
+    for l in stepped:
         live = gpu.corm_cache_live_lens(l)
-        seen = full[l].prompt_lens[:, None] + steps
+        seen = lens[l][:, None] + steps
         assert (live <= seen).all() and (live >= np.minimum(seen, cfg.recent_r)).all()
+    if api == "steps" and which != 5:     # the launches were chained (the long-context units keep the verdict launch)
+        assert gpu.corm_cache_chained_launches() >= steps // 2
