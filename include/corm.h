@@ -247,7 +247,9 @@ corm_status_t corm_cache_import_state(corm_cache_t* cache, int32_t layer, int32_
  * launch has many units and by a second, verdict launch when it has few, and grouped heads take the balanced
  * kernel (every block an equal share of the step's keys) followed by the verdict launch; 2 / 3 = the block-per-split
  * kernel with the first / the second way always; 4 / 5 = the balanced kernel for every group size it covers,
- * finishing inside its own launch / with the verdict launch. Errors: INVALID_ARG. */
+ * finishing inside its own launch / with the verdict launch; 6 = the balanced kernel's streaming loop with a block per
+ * split, each unit finished by its last-arriving split (what automatic picks for grouped heads inside
+ * corm_decode_steps unless units are few and long, because such launches can be chained). Errors: INVALID_ARG. */
 corm_status_t corm_cache_set_tuning(corm_cache_t* cache, int32_t split_len, int32_t allow_fast_path);
 
 /* Opt-in monitor of the method's premise (Sections 3.2-3.3: the current query resembles recent ones, which is what

@@ -712,6 +712,12 @@ corm_status_t decode_steps_impl(corm_cache_t* c, int32_t first_layer, int32_t n_
         fuse = c->steps[first_layer + i] == c->steps[first_layer] && c->parity[first_layer + i] == c->parity[first_layer];
     const auto at = [](const void* ptr, size_t off) { return static_cast<const unsigned char*>(ptr) + off; };
     const auto at_out = [](void* ptr, size_t off) { return static_cast<unsigned char*>(ptr) + off; };
+    // A call that enqueues many steps at once would size all of them from whatever the host knew on entry. If a length
+    // read-back is still in flight (typically the prompt pass's: without it the bound is the prompt length, several
+    // times the survivors), wait for it here, once: the GPU is busy with what precedes it anyway.
+    if (n_steps > 1)
+        for (int i = 0; i < n_layers; ++i)
+            if (c->readback_pending[first_layer + i]) (void)cudaEventSynchronize(c->readback_ev[first_layer + i]);
     for (int s = 0; s < n_steps; ++s) {
         // A step is chained to the one before it when that one was enqueued by this call (nothing of the caller's can
         // sit between them on the stream, and every step's inputs precede the call) and neither is the last word on

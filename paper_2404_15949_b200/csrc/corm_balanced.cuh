@@ -1065,7 +1065,12 @@ inline corm_status_t launch_decode_balanced_units(DecodeParams& p, const CUtenso
         // (128 units of 1660 keys, us per step: splits of 256 keys 47.4, 384 43.4, 512 42.5, 640 44.4, 896 47.8)
         const long long keys = (long long)(typical > 0 ? typical : upper) * p.U;
         split_len = (int)(2 * keys / (3ll * sms * kBalBlocksPerSm));
-        if (split_len > 2048) split_len = 2048;
+        // ... but at least 512 keys and at most 1024, or 2048 for long units: the grouped workload's first steps (units
+        // of 3000-4500 keys, many evictions) take 108-112 us with splits of 512 or 1024 keys and 117-120 with 1152 or
+        // 1280; 8200-key units take 132 us with splits of 2048, 142 with 1024, 162 with 512
+        const int cap = (typical > 0 ? typical : upper) < 6144 ? 1024 : 2048;
+        if (split_len > cap) split_len = cap;
+        if (split_len < 512) split_len = 512;
     }
     const int max_unit_splits = bal_unit_splits(p.max_splits);     // records a unit has room for, in splits
     if (split_len < (upper + max_unit_splits - 1) / max_unit_splits) split_len = (upper + max_unit_splits - 1) / max_unit_splits;

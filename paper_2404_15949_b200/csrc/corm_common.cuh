@@ -357,11 +357,11 @@ __device__ __forceinline__ int kept_before(const uint32_t* mask, const int* pref
 // row_of(slot) gives the slot's row in the layer's K / V storage (Kl, Vl).
 // part / n_parts: this block takes the chunks of NT / 8 rows numbered part, part + n_parts, ... (several blocks
 // sharing one unit's moves); the default is every chunk.
-template <typename T, int D, int NT, typename RowOf>
+template <typename T, int D, int NT, int KROWS = 4, typename RowOf>
 __device__ __forceinline__ void block_move_rows(T* Kl, T* Vl, RowOf row_of, uint32_t* wordu, int32_t* posu,
                                                 const int* movers, const int* holes, int n_moved, int part = 0,
                                                 int n_parts = 1, int slot_limit = 0x7fffffff, int32_t* status = nullptr) {
-    constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = 4, NW = NT / 32;
+    constexpr int kChunks = D * Elem<T>::kBytes / 16, kIter = (2 * kChunks + 31) / 32, kRows = KROWS, NW = NT / 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i0 = (part * NW + warp) * kRows; i0 < n_moved; i0 += n_parts * NW * kRows) {
         int src[kRows], dst[kRows];
