@@ -305,7 +305,8 @@ class CormCache:
     def corm_cache_set_tuning(self, split_len=0, allow_fast_path=True):
         """allow_fast_path: False/0 generic kernels, True/1 automatic, 2 / 3 block-per-split kernels that always finish
         units of several splits inside the decode launch / by the verdict launch, 4 / 5 the balanced kernel finishing
-        inside its launch / with the verdict launch."""
+        inside its launch / with the verdict launch, 6 that kernel's loop with a block per split and each unit finished
+        by its last split."""
         _check("corm_cache_set_tuning", self.lib.corm_cache_set_tuning(self.handle, split_len, int(allow_fast_path)))
 
     def corm_cache_set_similarity_monitor(self, enabled=True):

@@ -1,5 +1,6 @@
 // Host side of the C-ABI library: arena layout, argument checks, launch configuration. Every step of the hot
-// path runs in the kernels of corm_fast.cuh / corm_verdict.cuh / corm_prompt_fast.cuh / corm_generic.cuh; nothing
+// path runs in the kernels of corm_fast.cuh / corm_balanced.cuh / corm_verdict.cuh / corm_prompt_fast.cuh /
+// corm_generic.cuh; nothing
 // here touches tensor data on the CPU.
 #include <cuda_runtime.h>
 #include <nvtx3/nvToolsExt.h>

@@ -13,12 +13,14 @@
 //         being (head, hi / lo); fp32 accumulation. A group of four heads fills the 8 columns of one instruction.
 //   softmax  per head against a fixed reference (the maximum of the warp's first tile of the segment) that moves only
 //         when a logit exceeds it by more than 16; Z in fp64.
-// Per segment every warp stores one record {m, Z, acc[128]} per head and the scaled logits of its tiles and bumps the
-// unit's arrival counter; warps never meet inside the streaming loop. After its streaming a block applies
-// Algorithm 1 to the slots it streamed, once the unit's records are all in (thresholds of Definition 3.1 from the
-// records, verdicts, register update, keep bits), and the unit's last block compacts it (bal_finish_block).
+// Per segment every warp stores one record {m, Z, acc[128]} per head and the scaled logits of its tiles; warps never
+// meet inside the streaming loop. Who applies Algorithm 1 afterwards depends on the kernel's form (template
+// parameter MODE of decode_balanced_kernel): the verdict launch of corm_verdict.cuh, which reads the records through
+// a per-unit record list (the default from per-step calls); the blocks that streamed a unit, once its records are
+// all in, with the unit's last block compacting it (bal_finish_block); or, with a block per split instead of the
+// balanced partition, the unit's last-arriving split alone, which is the form whose launches can be chained.
 // Launched with programmatic stream serialization: a step's blocks set up their barriers while the previous
-// step drains and wait for it before they read anything.
+// step drains and wait for it (or, chained, for their own unit's previous step) before they read anything.
 #pragma once
 
 #include <cuda.h>
