@@ -345,6 +345,7 @@ CHAINED = [
     (2, 3, 2, 1, (1, 40), 60, 8, 4, 0, 6, 0),              # tiny units (empty splits), two heads per group
     (1, 3, 2, 1, (150, 330), 40, 8, 16, 128, 6, 0),        # one head per KV head on that kernel
     (4, 2, 1, 3, (260, 260), 30, 8, 32, 0, 6, 0),          # three layers as one launch per step
+    (1, 8, 1, 2, (260, 260), 20, 8, 32, 0, 1, 2048),       # two layers with pools of their own: a launch per layer, unchained
 ]
 
 
@@ -382,7 +383,7 @@ def test_many_steps_from_one_call(G, n_kv, batch, n_layers, prange, steps, w, r,
     assert st["device_status"] == 0 and st["evicted_keys"] == orc.counters()["evicted"] > 0
     assert orc.counters()["near_threshold"] == 0
     chained = gpu.corm_cache_chained_launches()
-    if G > 1 and tuning == 1 and prange[1] > 96 * batch * n_kv * n_layers:
+    if (G > 1 and tuning == 1 and prange[1] > 96 * batch * n_kv * n_layers) or (pool_pages and n_layers > 1):
         assert chained == 0
     else:     # every launch after a call's first, as long as each finished its units itself
         assert chained >= steps // 2, chained
