@@ -66,6 +66,18 @@ def test_create_rejects_before_any_cuda_call(lib):
     assert lib.corm_cache_destroy(None) == 1 and lib.corm_cache_kernel_launches(None) == 0
 
 
+def test_step_calls_reject_a_missing_cache_before_any_cuda_call(lib):
+    fake = ctypes.c_void_p(0x10000)
+    assert lib.corm_decode_step(None, 0, fake, fake, fake, fake, None) == 1
+    assert lib.corm_decode_step_layers(None, 0, 1, fake, fake, fake, fake, None) == 1
+    assert lib.corm_decode_steps(None, 0, 1, 4, fake, fake, fake, fake, None) == 1
+    assert lib.corm_decode_steps_host(None, 0, 1, 4, fake, fake, fake, fake, None) == 1
+    assert lib.corm_decode_step_host(None, 0, fake, fake, fake, fake, None) == 1
+    assert lib.corm_decode_step_static(None, 0, fake, fake, fake, fake, None) == 1
+    assert lib.corm_cache_chained_launches(None) == 0
+    assert len(lib.corm_status_string(8)) > 0 and lib.corm_status_string(8) != lib.corm_status_string(7)
+
+
 def test_paged_arena_holds_the_pool_not_the_slabs(lib):
     # The paper's headline is up to 70 % of the KV cache saved: a pool sized for 30 % of the slabs' rows must need
     # about 30 % of the memory (page tables, bitmap, registers, positions and scratch on top).
