@@ -542,14 +542,15 @@ decode_balanced_kernel(const __grid_constant__ DecodeParams p, const __grid_cons
             }
             return;
         }
-        const int n_unit = (l + kTileKeys - 1) / kTileKeys, tps = p.split_len / kTileKeys;
-        const int n_act = (n_unit + tps - 1) / tps;
+        const int n_unit = (l + kTileKeys - 1) / kTileKeys;
+        const int n_act = (n_unit + p.split_len / kTileKeys - 1) / (p.split_len / kTileKeys);
         if (split >= n_act) return;
+        const int tps = (n_unit + n_act - 1) / n_act;          // the unit's tiles shared out evenly over its splits
         if (n_act > (int)gridDim.x && split == 0 && tid == 0) report_status(p.status, CORM_ERR_INTERNAL);   // the host's bound on the unit was wrong
         if (p.early_trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // every block has its length by now
         if (tid == 0) {
             BalSeg sg;
-            sg.u = u; sg.l = l; sg.tile0 = split * tps; sg.n_tiles = min(tps, n_unit - split * tps); sg.gtile0 = 0;
+            sg.u = u; sg.l = l; sg.tile0 = min(n_unit, split * tps); sg.n_tiles = max(0, min(tps, n_unit - split * tps)); sg.gtile0 = 0;
             sg.t = __ldcg(p.base_tokens + u / p.Hkv) + p.step + 1; sg.n_unit = n_unit; sg.pad = n_act;
             segs[0] = sg;
             s_nseg = 1; s_more = 0;
