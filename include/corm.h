@@ -177,7 +177,8 @@ corm_status_t corm_decode_step_layers(corm_cache_t* cache, int32_t first_layer, 
  * once per step (registers, live lists and positions identical, outputs within rounding).
  * What the call adds: the units of a cache are independent (Algorithm 1 runs "on each head at every layer"), so
  * step s + 1 of a unit needs step s of that unit only. When a step's launch finishes every unit inside the streaming
- * kernel (one query head per KV head, or tuning value 2), the next step's launch is chained to it: its blocks start
+ * kernel (one query head per KV head; grouped heads inside this call, which take a block per split unless units are
+ * few and long; tuning values 2 and 6), the next step's launch is chained to it: its blocks start
  * as soon as a multiprocessor has room and each waits (bounded, like every wait here) for its own unit's previous
  * step instead of the whole previous launch, so consecutive steps fill one another's last waves. Steps that need the
  * verdict launch, and caches with the similarity monitor on, run as with the per-step calls.
